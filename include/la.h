@@ -1,0 +1,171 @@
+/*
+ * la.h -- C boundary of the linear-attention layer library (libla_b200.so, sm_100a).
+ *
+ * One causal linear-attention layer with feature map phi and the causally masked
+ * depthwise-convolution augmentation, in three modes:
+ *
+ *   prefill  (la_prefill)      grouped / chunkwise-parallel processing of T tokens,
+ *   decode   (la_decode_step)  one token per sequence against the running state,
+ *   verify   (la_verify_tree)  a draft-token tree against the committed state, which is
+ *                              left untouched, followed by
+ *   commit   (la_commit)       absorbing the accepted root-to-node path.
+ *
+ * Notation, per batch entry b and head h (d = head dimension):
+ *   a_ij = phi(q_i) . phi(k_j)
+ *   la_i = sum_{j<=i} a_ij v_j / (sum_{j<=i} a_ij + eps)
+ *   o_i  = la_i + sum_{t<W} w[h,:,t] * v_{i-t}            (elementwise over channels)
+ *   S[a][c] = sum_j phi(k_j)[a] v_j[c],  z[a] = sum_j phi(k_j)[a]
+ * W counts the live causal taps of the convolution: the current token and W-1 past ones.
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers on the device that was current at la_create,
+ *     16-byte aligned, densely packed, innermost dimension last.  Exceptions are marked
+ *     "host".  q, k, v, o and the window use the io type of the context (fp32 or bf16);
+ *     S, z and the convolution weights are always fp32.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  No entry point other than la_create / la_destroy allocates or frees
+ *     memory, and none but la_last_device_status synchronises.
+ *   - The caller owns all tensors and the state buffers.  The context owns one device
+ *     status word.
+ *   - Every entry point returns an la_status.  Problems the host can see (null or
+ *     misaligned pointers, sizes out of range, unsupported head dimension) are rejected
+ *     before anything is launched.  Problems only the device can see (a malformed tree, an
+ *     accepted node outside the tree, a bounded wait that ran out) make the kernel skip the
+ *     affected sequence, leave its outputs and state unwritten, and record a sticky code in
+ *     the status word, which la_last_device_status returns.  Nothing ever traps.
+ */
+#ifndef LA_B200_LA_H_
+#define LA_B200_LA_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  LA_OK = 0,
+  LA_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, size out of range */
+  LA_ERR_UNSUPPORTED = 2,   /* configuration the library has no kernel for */
+  LA_ERR_CUDA = 3,          /* a CUDA runtime or driver call failed */
+  LA_ERR_BAD_TREE = 4,      /* device: parent[n] not in [-1, n), path deeper than max_depth,
+                               accepted node outside [-1, N) */
+  LA_ERR_TIMEOUT = 5        /* device: a bounded wait on an asynchronous copy or MMA ran out */
+} la_status;
+
+typedef enum { LA_PHI_ELU1 = 0,   /* phi(x) = x + 1 for x > 0, exp(x) otherwise */
+               LA_PHI_RELU = 1    /* phi(x) = max(x, 0) */
+} la_phi;
+
+typedef enum { LA_F32 = 0, LA_BF16 = 1 } la_dtype;
+
+/* Limits of this build. */
+#define LA_MAX_TAPS   32   /* W */
+#define LA_MAX_NODES  64   /* N, one 64-bit ancestor mask per node */
+
+typedef struct {
+  int32_t  H;           /* heads */
+  int32_t  d;           /* head dimension: 64 or 128 */
+  int32_t  conv_taps;   /* W, 1..LA_MAX_TAPS */
+  int32_t  chunk;       /* group size C of the grouped prefill; 0 = library default.  The
+                           result does not depend on it; it only selects the tiling. */
+  la_phi   phi;
+  float    eps;         /* added to the denominator */
+  la_dtype io_dtype;    /* type of q, k, v, o and the window */
+  int32_t  max_nodes;   /* largest N passed to verify / commit, 1..LA_MAX_NODES */
+  int32_t  max_depth;   /* longest accepted path; row length of path_out */
+} la_config;
+
+/* Running state of B sequences (caller-owned device buffers). */
+typedef struct {
+  float*   S;     /* [B, H, d, d]   S[a][c], c innermost */
+  float*   z;     /* [B, H, d] */
+  void*    win;   /* [B, H, W-1, d] io type, the last W-1 values of v, oldest first;
+                     may be NULL when W == 1 */
+  int64_t* pos;   /* [B] tokens absorbed so far */
+} la_state;
+
+typedef struct la_ctx la_ctx;
+
+/* Library set-up.  la_create validates the configuration, allocates the device status word
+ * on the current device and returns a context; la_destroy frees it.  Neither is
+ * asynchronous. */
+la_status la_create(const la_config* cfg /*host*/, la_ctx** out /*host*/);
+la_status la_destroy(la_ctx* ctx);
+
+/* Name of a status code (static string, never NULL). */
+const char* la_status_str(la_status s);
+
+/* Prefill: the grouped processing of Sec. 4.1 ("LA Augmentation for Autoregressive LLMs").
+ * The sequence is cut into non-overlapping groups; inside a group the causally masked
+ * product phi(Q) phi(K)^T V is formed in parallel, between groups only the group-level
+ * cumulative sums S and z of the phi(K)^T V products are carried (Sec. 3 "Linear
+ * Attentions" for the reordering phi(Q)(phi(K)^T V)); the masked depthwise convolution of
+ * V (Sec. 4.1 "Revised LA Augmentation") is added to the output.
+ *
+ *   q, k, v     [B, H, T, d] io type, T >= 1
+ *   conv_w      [H, d, W] fp32, tap 0 multiplies the current token
+ *   init_state  0: start from an empty state (st is output only); 1: continue from st
+ *   st          in-out; on return holds S, z, the window and pos after the T tokens
+ *   o           [B, H, T, d] io type
+ */
+la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
+                     const float* conv_w, int32_t init_state, la_state* st /*host struct*/, void* o,
+                     void* stream);
+
+/* Decode: one token per sequence.  The cumulative sum of Sec. 4.1 (query t meets
+ * sum_{i<=t} K_i V_i) as a recurrence: S += phi(k) v^T, z += phi(k), then
+ * o = phi(q)^T S / (phi(q).z + eps) + conv, with the convolution reading the carried
+ * window, which is then advanced by one token.
+ *
+ *   q, k, v  [B, H, d] io type;  st in-out;  o [B, H, d] io type
+ */
+la_status la_decode_step(la_ctx* ctx, int32_t B, const void* q, const void* k, const void* v,
+                         const float* conv_w, la_state* st /*host struct*/, void* o, void* stream);
+
+/* Verify: outputs for all N nodes of a per-sequence draft tree against the committed
+ * state, which is read once and not modified (Sec. 4.2 "Proposed Solution"; the shared
+ * cumulative-sum state of Sec. 5.3 "Comparison with Direct Integration").  Node n sees the
+ * committed prefix, its ancestors and itself; tap t of the unfolded convolution reads the
+ * t-th ancestor while one exists and the committed window behind the tree otherwise,
+ * never a sibling.
+ *
+ *   q, k, v  [B, H, N, d] io type, 1 <= N <= max_nodes
+ *   parent   [B, N] int32; -1 = child of the committed prefix; parent[n] < n
+ *   st       read-only;  o [B, H, N, d] io type
+ */
+la_status la_verify_tree(la_ctx* ctx, int32_t B, int32_t N, const void* q, const void* k, const void* v,
+                         const int32_t* parent, const float* conv_w, const la_state* st /*host struct*/,
+                         void* o, void* stream);
+
+/* Commit: absorb the accepted root-to-node path of each sequence exactly as if its tokens
+ * had been decoded one by one (Sec. 4.2: later groups interact with the verified tokens of
+ * earlier ones).  k, v and parent are the buffers given to la_verify_tree.
+ *
+ *   accept_node  [B] int32: deepest accepted node, -1 = nothing accepted (a no-op)
+ *   st           in-out: S, z, window and pos advance by the path
+ *   path_out     [B, max_depth] int32: the path root first, padded with -1
+ *   commit_len   [B] int32: its length
+ */
+la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void* v, const int32_t* parent,
+                    const int32_t* accept_node, la_state* st /*host struct*/, int32_t* path_out,
+                    int32_t* commit_len, void* stream);
+
+/* Waits for `stream`, then returns the sticky device status (LA_OK if no kernel reported a
+ * problem since the last la_clear_device_status). */
+la_status la_last_device_status(la_ctx* ctx, void* stream);
+
+/* Resets the device status word to LA_OK (asynchronous on `stream`). */
+la_status la_clear_device_status(la_ctx* ctx, void* stream);
+
+/* Selects the prefill kernel: 0 = automatic (tensor-core kernel where it applies),
+ * 1 = always the fp32 CUDA-core kernel.  For testing one kernel against the other. */
+la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which);
+
+/* Number of kernels the library has launched through this context since creation. */
+int64_t la_launch_count(const la_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* LA_B200_LA_H_ */

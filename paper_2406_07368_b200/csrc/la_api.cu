@@ -1,0 +1,169 @@
+// C boundary: argument validation, dispatch to the kernel launchers, status handling.
+#include <cmath>
+#include <cstdlib>
+#include <new>
+
+#include "la_common.cuh"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool good(const void* p) { return p != nullptr && aligned16(p); }
+
+bool state_ok(const la_ctx* ctx, const la_state* st) {
+  if (!st || !good(st->S) || !good(st->z) || st->pos == nullptr) return false;
+  if (ctx->cfg.conv_taps > 1 && !good(st->win)) return false;
+  return true;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* la_status_str(la_status s) {
+  switch (s) {
+    case LA_OK: return "LA_OK";
+    case LA_ERR_INVALID_ARG: return "LA_ERR_INVALID_ARG";
+    case LA_ERR_UNSUPPORTED: return "LA_ERR_UNSUPPORTED";
+    case LA_ERR_CUDA: return "LA_ERR_CUDA";
+    case LA_ERR_BAD_TREE: return "LA_ERR_BAD_TREE";
+    case LA_ERR_TIMEOUT: return "LA_ERR_TIMEOUT";
+  }
+  return "LA_ERR_UNKNOWN";
+}
+
+la_status la_create(const la_config* cfg, la_ctx** out) {
+  if (!cfg || !out) return LA_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->H < 1 || cfg->conv_taps < 1 || cfg->conv_taps > LA_MAX_TAPS || cfg->chunk < 0) return LA_ERR_INVALID_ARG;
+  if (cfg->phi != LA_PHI_ELU1 && cfg->phi != LA_PHI_RELU) return LA_ERR_INVALID_ARG;
+  if (cfg->io_dtype != LA_F32 && cfg->io_dtype != LA_BF16) return LA_ERR_INVALID_ARG;
+  if (!(cfg->eps >= 0.f) || !std::isfinite(cfg->eps)) return LA_ERR_INVALID_ARG;
+  if (cfg->max_nodes < 1 || cfg->max_nodes > LA_MAX_NODES) return LA_ERR_INVALID_ARG;
+  if (cfg->max_depth < 1 || cfg->max_depth > LA_MAX_NODES) return LA_ERR_INVALID_ARG;
+  if (cfg->d != 64 && cfg->d != 128) return LA_ERR_UNSUPPORTED;
+
+  la_ctx* ctx = new (std::nothrow) la_ctx();
+  if (!ctx) return LA_ERR_CUDA;
+  ctx->cfg = *cfg;
+  ctx->prefill_kernel = 0;
+  ctx->launches = 0;
+  ctx->d_status = nullptr;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
+      cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess ||
+      cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) {
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+    cudaGetLastError();
+    return LA_ERR_CUDA;
+  }
+  *out = ctx;
+  return LA_OK;
+}
+
+la_status la_destroy(la_ctx* ctx) {
+  if (!ctx) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = cudaFree(ctx->d_status);
+  delete ctx;
+  return e == cudaSuccess ? LA_OK : LA_ERR_CUDA;
+}
+
+la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which) {
+  if (!ctx || which < 0 || which > 1) return LA_ERR_INVALID_ARG;
+  ctx->prefill_kernel = which;
+  return LA_OK;
+}
+
+int64_t la_launch_count(const la_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
+                     const float* conv_w, int32_t init_state, la_state* st, void* o, void* stream) {
+  if (!ctx || B < 1 || T < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o)) return LA_ERR_INVALID_ARG;
+  if (!state_ok(ctx, st) || (init_state != 0 && init_state != 1)) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->prefill_kernel == 0) {
+    bool handled = false;
+    cudaError_t e = la::launch_prefill_tc(ctx, B, T, q, k, v, conv_w, init_state, *st, o, s, &handled);
+    if (e != cudaSuccess) return LA_ERR_CUDA;
+    if (handled) return LA_OK;
+  }
+  return la::launch_prefill_simt(ctx, B, T, q, k, v, conv_w, init_state, *st, o, s) == cudaSuccess ? LA_OK
+                                                                                                   : LA_ERR_CUDA;
+}
+
+la_status la_decode_step(la_ctx* ctx, int32_t B, const void* q, const void* k, const void* v, const float* conv_w,
+                         la_state* st, void* o, void* stream) {
+  if (!ctx || B < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o)) return LA_ERR_INVALID_ARG;
+  if (!state_ok(ctx, st)) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return la::launch_decode(ctx, B, q, k, v, conv_w, *st, o, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
+la_status la_verify_tree(la_ctx* ctx, int32_t B, int32_t N, const void* q, const void* k, const void* v,
+                         const int32_t* parent, const float* conv_w, const la_state* st, void* o, void* stream) {
+  if (!ctx || B < 1 || N < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o) || !parent)
+    return LA_ERR_INVALID_ARG;
+  if (N > ctx->cfg.max_nodes) return LA_ERR_INVALID_ARG;
+  if (!state_ok(ctx, st)) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return la::launch_verify(ctx, B, N, q, k, v, parent, conv_w, *st, o, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
+la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void* v, const int32_t* parent,
+                    const int32_t* accept_node, la_state* st, int32_t* path_out, int32_t* commit_len, void* stream) {
+  if (!ctx || B < 1 || N < 1 || !good(k) || !good(v) || !parent || !accept_node || !path_out || !commit_len)
+    return LA_ERR_INVALID_ARG;
+  if (N > ctx->cfg.max_nodes) return LA_ERR_INVALID_ARG;
+  if (!state_ok(ctx, st)) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return la::launch_commit(ctx, B, N, k, v, parent, accept_node, *st, path_out, commit_len,
+                           static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
+la_status la_last_device_status(la_ctx* ctx, void* stream) {
+  if (!ctx) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  int code = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&code, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return LA_ERR_CUDA;
+  return static_cast<la_status>(code);
+}
+
+la_status la_clear_device_status(la_ctx* ctx, void* stream) {
+  if (!ctx) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return cudaMemsetAsync(ctx->d_status, 0, sizeof(int), static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
+}  // extern "C"

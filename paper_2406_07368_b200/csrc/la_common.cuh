@@ -1,0 +1,76 @@
+// Shared device helpers: io-type loads and stores, the feature map, the sticky status word.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "la.h"
+
+namespace la {
+
+// ---- io type ---------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// ---- feature map (Sec. 3: Sim(Q,K) ~ phi(Q) phi(K)^T) ------------------------------------
+template <int PHI> __device__ __forceinline__ float phi(float x) {
+  if (PHI == LA_PHI_ELU1) return x > 0.f ? x + 1.f : expf(x);
+  return fmaxf(x, 0.f);
+}
+
+// ---- sticky device status ---------------------------------------------------------------
+__device__ __forceinline__ void report(int* status, int code) { atomicCAS(status, 0, code); }
+
+// Block-wide sum of one float per thread; result valid in every thread.  `scratch` holds
+// at least 33 floats.
+__device__ __forceinline__ float block_sum(float x, float* scratch) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  if (lane == 0) scratch[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    float y = lane < nwarp ? scratch[lane] : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) y += __shfl_xor_sync(0xffffffffu, y, o);
+    if (lane == 0) scratch[32] = y;
+  }
+  __syncthreads();
+  float r = scratch[32];
+  __syncthreads();
+  return r;
+}
+
+}  // namespace la
+
+// ---- host side --------------------------------------------------------------------------
+struct la_ctx {
+  la_config cfg;
+  int device;
+  int* d_status;          // device status word
+  int prefill_kernel;     // 0 auto, 1 CUDA-core kernel
+  int64_t launches;
+  int sm_count;
+};
+
+// Kernel launchers (one per translation unit).  All return the cudaError_t of the launch.
+namespace la {
+cudaError_t launch_decode(la_ctx* ctx, int B, const void* q, const void* k, const void* v, const float* w,
+                          const la_state& st, void* o, cudaStream_t s);
+cudaError_t launch_prefill_simt(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v,
+                                const float* w, int init_state, const la_state& st, void* o, cudaStream_t s);
+cudaError_t launch_verify(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
+                          const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s);
+cudaError_t launch_commit(la_ctx* ctx, int B, int N, const void* k, const void* v, const int32_t* parent,
+                          const int32_t* accept, const la_state& st, int32_t* path_out, int32_t* commit_len,
+                          cudaStream_t s);
+// Tensor-core prefill (bf16, d = 128).  Sets *handled to false when the shape is not covered.
+cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v,
+                              const float* w, int init_state, const la_state& st, void* o, cudaStream_t s,
+                              bool* handled);
+}  // namespace la
