@@ -1,0 +1,291 @@
+"""Parity of the CUDA path (through the C boundary) with the float64 oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import la_oracle as orc
+from paper_2406_07368_b200 import binding, workloads as wl
+from tests._util import TOL, rel_err
+
+pytestmark = pytest.mark.gpu
+
+
+def dev(x, io):
+    return torch.from_numpy(np.ascontiguousarray(x)).to(binding.TORCH_DTYPE[io]).cuda()
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64) if t.is_floating_point() else t.cpu().numpy()
+
+
+def oracle_state_to_dev(st, io):
+    return binding.State(torch.from_numpy(st.S).float().cuda(), torch.from_numpy(st.z).float().cuda(),
+                         dev(st.win.astype(np.float32), io), torch.from_numpy(st.pos).cuda())
+
+
+def check_state(got: binding.State, want: orc.State, tol, exact_window=True):
+    assert rel_err(host(got.S), want.S) < tol
+    assert rel_err(host(got.z), want.z) < tol
+    if exact_window:
+        np.testing.assert_array_equal(host(got.win), want.win)
+    np.testing.assert_array_equal(host(got.pos), want.pos)
+
+
+def make(io, B, H, d, T, W, seed, scale=1.0):
+    q, k, v = wl.qkv(seed, (B, H, T, d), scale, io)
+    w = wl.conv_weights(seed, H, d, W)
+    return q, k, v, w
+
+
+# ------------------------------------------------------------------ prefill
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("io,d,phi,eps,W,T", [
+    ("f32", 64, "elu1", 0.0, 3, 256),
+    ("f32", 128, "relu", 1e-6, 5, 70),
+    ("bf16", 128, "elu1", 0.0, 3, 1),
+    ("bf16", 128, "elu1", 0.0, 3, 127),
+    ("bf16", 128, "elu1", 0.0, 3, 128),
+    ("bf16", 128, "elu1", 0.0, 3, 129),
+    ("bf16", 128, "elu1", 0.0, 3, 700),
+    ("bf16", 128, "relu", 1e-6, 5, 333),
+    ("bf16", 64, "elu1", 0.0, 3, 200),
+    ("bf16", 128, "elu1", 0.0, 32, 150),
+    ("bf16", 128, "elu1", 0.0, 1, 150),
+])
+def test_prefill_matches_oracle(kernel, io, d, phi, eps, W, T):
+    B, H = 2, 3
+    scale = 1.0 if io == "f32" else d ** -0.5
+    q, k, v, w = make(io, B, H, d, T, W, seed=T + W, scale=scale)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    st.S.fill_(7.0)          # a fresh prefill must ignore whatever the buffers hold
+    st.pos.fill_(99)
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st, init_state=False)
+    want, wst = orc.prefill_quadratic(q, k, v, w, phi, eps)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    assert rel_err(host(o), want) < TOL[io]
+    check_state(st, wst, TOL[io])
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("io,T1,T2", [("f32", 50, 77), ("bf16", 1, 200), ("bf16", 130, 129), ("bf16", 255, 2)])
+def test_prefill_continuation(kernel, io, T1, T2):
+    B, H, d, W = 1, 2, 128, 4
+    q, k, v, w = make(io, B, H, d, T1 + T2, W, seed=5, scale=0.5)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    cut = lambda x, a, b: dev(x[:, :, a:b], io)
+    o1 = ctx.la_prefill(cut(q, 0, T1), cut(k, 0, T1), cut(v, 0, T1), dev(w, "f32"), st, init_state=False)
+    o2 = ctx.la_prefill(cut(q, T1, T1 + T2), cut(k, T1, T1 + T2), cut(v, T1, T1 + T2), dev(w, "f32"), st,
+                        init_state=True)
+    want, wst = orc.prefill_quadratic(q, k, v, w, "elu1", 0.0)
+    assert rel_err(np.concatenate([host(o1), host(o2)], axis=2), want) < TOL[io]
+    check_state(st, wst, TOL[io])
+
+
+def test_prefill_is_causal_bitwise():
+    """Perturbing token j leaves every earlier output bit-identical (no leakage through the conv)."""
+    io, B, H, d, T, W = "bf16", 1, 2, 128, 300, 8
+    q, k, v, w = make(io, B, H, d, T, W, seed=11, scale=0.3)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    for kernel in (0, 1):
+        ctx.la_set_prefill_kernel(kernel)
+        o1 = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), ctx.new_state(B))
+        j = 200
+        q2, k2, v2 = q.copy(), k.copy(), v.copy()
+        q2[:, :, j] = wl.round_to_bf16(q2[:, :, j] + 1)
+        k2[:, :, j] = wl.round_to_bf16(k2[:, :, j] - 1)
+        v2[:, :, j] = wl.round_to_bf16(v2[:, :, j] * 3)
+        o2 = ctx.la_prefill(dev(q2, io), dev(k2, io), dev(v2, io), dev(w, "f32"), ctx.new_state(B))
+        assert torch.equal(o1[:, :, :j], o2[:, :, :j])
+        assert not torch.equal(o1[:, :, j], o2[:, :, j])
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("io,d,phi,eps,W", [("f32", 64, "elu1", 0.0, 3), ("bf16", 128, "elu1", 0.0, 3),
+                                            ("bf16", 128, "relu", 1e-6, 5), ("bf16", 64, "elu1", 0.0, 1),
+                                            ("f32", 128, "elu1", 0.0, 32)])
+def test_decode_matches_oracle(io, d, phi, eps, W):
+    B, H, T0, steps = 3, 2, 40, 12
+    q, k, v, w = make(io, B, H, d, T0, W, seed=21 + W, scale=0.7)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    _, ost = orc.prefill_quadratic(q, k, v, w, phi, eps)
+    st = oracle_state_to_dev(ost, io)
+    for s in range(steps):
+        qs, ks, vs = wl.qkv(100 + s, (B, H, d), 0.7, io)
+        o = ctx.la_decode_step(dev(qs, io), dev(ks, io), dev(vs, io), dev(w, "f32"), st)
+        want, ost = orc.decode_step(qs, ks, vs, w, phi, eps, ost)
+        assert rel_err(host(o), want) < TOL[io], s
+    check_state(st, ost, TOL[io])
+
+
+def test_prefill_then_decode_equals_longer_prefill():
+    io, B, H, d, W, T, extra = "bf16", 1, 2, 128, 3, 140, 5
+    q, k, v, w = make(io, B, H, d, T + extra, W, seed=31, scale=0.5)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    st = ctx.new_state(B)
+    ctx.la_prefill(dev(q[:, :, :T], io), dev(k[:, :, :T], io), dev(v[:, :, :T], io), dev(w, "f32"), st)
+    outs = [ctx.la_decode_step(dev(q[:, :, T + i], io), dev(k[:, :, T + i], io), dev(v[:, :, T + i], io),
+                               dev(w, "f32"), st) for i in range(extra)]
+    want, wst = orc.prefill_quadratic(q, k, v, w, "elu1", 0.0)
+    got = np.stack([host(o) for o in outs], axis=2)
+    assert rel_err(got, want[:, :, T:]) < TOL[io]
+    check_state(st, wst, TOL[io])
+
+
+# ------------------------------------------------------------------ verify + commit
+def tree_case(io, B, H, d, N, W, seed, phi="elu1", eps=0.0, chain=False):
+    q0, k0, v0, w = make(io, B, H, d, 30, W, seed=seed, scale=0.7)
+    _, ost = orc.prefill_quadratic(q0, k0, v0, w, phi, eps)
+    q, k, v = wl.qkv(seed + 1, (B, H, N, d), 0.7, io)
+    if chain:
+        parent = np.stack([wl.chain_tree(N)] * B)
+    else:
+        parent = np.stack([wl.random_tree(wl.rng(seed, 4, 0, b), N, 5, 4) for b in range(B)]).astype(np.int32)
+    return ost, q, k, v, parent, w
+
+
+@pytest.mark.parametrize("io,d,N,W,phi,eps,chain", [
+    ("bf16", 128, 64, 3, "elu1", 0.0, False), ("bf16", 128, 37, 5, "relu", 1e-6, False),
+    ("f32", 64, 4, 3, "elu1", 0.0, True), ("bf16", 64, 64, 3, "elu1", 0.0, False),
+    ("bf16", 128, 1, 3, "elu1", 0.0, False), ("f32", 128, 64, 9, "elu1", 0.0, False),
+    ("bf16", 128, 20, 32, "elu1", 0.0, True), ("bf16", 128, 16, 1, "elu1", 0.0, False)])
+def test_verify_matches_oracle_and_leaves_state_untouched(io, d, N, W, phi, eps, chain):
+    B, H = 3, 2
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=41 + N, phi=phi, eps=eps, chain=chain)
+    ctx = binding.Context(H, d, W, phi, eps, io, max_nodes=64, max_depth=64)
+    st = oracle_state_to_dev(ost, io)
+    before = st.clone()
+    o = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want = orc.verify_tree(q, k, v, parent, w, phi, eps, ost)
+    assert rel_err(host(o), want) < TOL[io]
+    for a, b in ((st.S, before.S), (st.z, before.z), (st.win, before.win), (st.pos, before.pos)):
+        assert torch.equal(a, b)
+
+
+def test_verify_siblings_are_independent_bitwise():
+    io, B, H, d, W = "bf16", 1, 2, 128, 3
+    ost, q, k, v, _, w = tree_case(io, B, H, d, 4, W, seed=51)
+    parent = np.array([[-1, 0, 0, 2]], dtype=np.int32)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    st = oracle_state_to_dev(ost, io)
+    o1 = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    q2, k2, v2 = q.copy(), k.copy(), v.copy()
+    q2[:, :, 1] = wl.round_to_bf16(q2[:, :, 1] + 2)
+    k2[:, :, 1] = wl.round_to_bf16(k2[:, :, 1] - 1)
+    v2[:, :, 1] = wl.round_to_bf16(v2[:, :, 1] * -4)
+    o2 = ctx.la_verify_tree(dev(q2, io), dev(k2, io), dev(v2, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    for n in (0, 2, 3):
+        assert torch.equal(o1[:, :, n], o2[:, :, n])
+    assert not torch.equal(o1[:, :, 1], o2[:, :, 1])
+
+
+@pytest.mark.parametrize("io,d,N,W", [("bf16", 128, 64, 3), ("f32", 64, 10, 5), ("bf16", 128, 64, 8)])
+def test_commit_matches_oracle_and_paths_are_exact(io, d, N, W):
+    B, H = 4, 2
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=61 + N)
+    accept = np.array([wl.random_accept(wl.rng(7, 6, 0, b), parent[b]) for b in range(B)], dtype=np.int32)
+    accept[1] = -1                                     # nothing accepted: a no-op
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=64, max_depth=6)
+    st = oracle_state_to_dev(ost, io)
+    path, clen = ctx.la_commit(dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(),
+                               torch.from_numpy(accept).cuda(), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    wst, wpath, wlen = orc.commit(k, v, parent, accept, "elu1", ost, max_depth=6)
+    np.testing.assert_array_equal(host(path), wpath)
+    np.testing.assert_array_equal(host(clen), wlen)
+    check_state(st, wst, TOL[io])
+    # and it equals decoding the path token by token on the GPU
+    st2 = oracle_state_to_dev(ost, io)
+    for b in range(B):
+        pass
+    ctx1 = binding.Context(H, d, W, "elu1", 0.0, io)
+    for b in range(B):
+        sb = binding.State(st2.S[b:b + 1].clone(), st2.z[b:b + 1].clone(), st2.win[b:b + 1].clone(),
+                           st2.pos[b:b + 1].clone())
+        for n in wpath[b][:wlen[b]]:
+            ctx1.la_decode_step(dev(q[b:b + 1, :, n], io), dev(k[b:b + 1, :, n], io), dev(v[b:b + 1, :, n], io),
+                                dev(w, "f32"), sb)
+        assert rel_err(host(sb.S), host(st.S[b:b + 1])) < 1e-5
+        assert torch.equal(sb.win, st.win[b:b + 1]) and torch.equal(sb.pos, st.pos[b:b + 1])
+
+
+def test_bad_trees_set_the_status_word_and_write_nothing():
+    io, B, H, d, N, W = "bf16", 2, 2, 128, 8, 3
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=71)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=16, max_depth=2)
+    st = oracle_state_to_dev(ost, io)
+    bad = parent.copy()
+    bad[1, 3] = 5                                      # parent after child in sequence 1
+    out = torch.full((B, H, N, d), 123.0, dtype=torch.bfloat16, device="cuda")
+    ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(bad).cuda(), dev(w, "f32"), st, out=out)
+    assert ctx.la_last_device_status() == binding.LA_ERR_BAD_TREE
+    assert torch.all(out[1] == 123.0) and not torch.any(out[0] == 123.0)
+    ctx.la_clear_device_status()
+    assert ctx.la_last_device_status() == binding.LA_OK
+    # accepted node outside the tree, and a path longer than max_depth
+    chain = np.stack([wl.chain_tree(N)] * B)
+    before = st.clone()
+    for accept in ([N, 0], [0, 5]):
+        path, clen = ctx.la_commit(dev(k, io), dev(v, io), torch.from_numpy(chain).cuda(),
+                                   torch.tensor(accept, dtype=torch.int32).cuda(), st)
+        assert ctx.la_last_device_status() == binding.LA_ERR_BAD_TREE
+        ctx.la_clear_device_status()
+        bad_b = 0 if accept[0] == N else 1
+        assert torch.equal(st.S[bad_b], before.S[bad_b]) and torch.equal(st.pos[bad_b:bad_b + 1], before.pos[bad_b:bad_b + 1])
+        st = before.clone()
+
+
+def test_host_side_rejections():
+    ctx = binding.Context(2, 128, 3, "elu1", 0.0, "bf16", max_nodes=8)
+    st = ctx.new_state(1)
+    x = torch.zeros(1, 2, 9, 128, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(2, 128, 3, device="cuda")
+    par = torch.full((1, 9), -1, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.LaError) as e:
+        ctx.la_verify_tree(x, x, x, par, w, st)        # N > max_nodes
+    assert e.value.code == binding.LA_ERR_INVALID_ARG
+    L = binding.lib()
+    cs = st.c()
+    import ctypes
+    rc = L.la_prefill(ctx._h, 1, 9, x.data_ptr() + 2, x.data_ptr(), x.data_ptr(), w.data_ptr(), 0, ctypes.byref(cs),
+                      x.data_ptr(), None)              # misaligned q
+    assert rc == binding.LA_ERR_INVALID_ARG
+    rc = L.la_prefill(ctx._h, 1, 0, x.data_ptr(), x.data_ptr(), x.data_ptr(), w.data_ptr(), 0, ctypes.byref(cs),
+                      x.data_ptr(), None)              # T = 0
+    assert rc == binding.LA_ERR_INVALID_ARG
+    assert ctx.la_launch_count() == 0
+
+
+# ------------------------------------------------------------------ the small end-to-end workload
+def test_tiny_fp32_workload_end_to_end():
+    """B=1, H=2, d=64, T=256 fp32: prefill, 16 decode steps, a 4-node chain verify, commit of 2."""
+    W = wl.tiny_fp32()
+    io = W.io
+    q, k, v = W.prefill_inputs()
+    w = W.weights()
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io, chunk=W.chunk)
+    st = ctx.new_state(W.B)
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st)
+    want, ost = orc.prefill_quadratic(q, k, v, w, W.phi, W.eps)
+    assert rel_err(host(o), want) < TOL[io]
+    for s in range(W.decode_steps):
+        qs, ks, vs = W.decode_inputs(s)
+        o = ctx.la_decode_step(dev(qs, io), dev(ks, io), dev(vs, io), dev(w, "f32"), st)
+        want, ost = orc.decode_step(qs, ks, vs, w, W.phi, W.eps, ost)
+        assert rel_err(host(o), want) < TOL[io]
+    qd, kd, vd = W.draft_inputs(0)
+    parent = np.stack([wl.chain_tree(W.tree_nodes)] * W.B)
+    o = ctx.la_verify_tree(dev(qd, io), dev(kd, io), dev(vd, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    assert rel_err(host(o), orc.verify_tree(qd, kd, vd, parent, w, W.phi, W.eps, ost)) < TOL[io]
+    accept = np.full((W.B,), W.extra["accept_node"], dtype=np.int32)
+    path, clen = ctx.la_commit(dev(kd, io), dev(vd, io), torch.from_numpy(parent).cuda(),
+                               torch.from_numpy(accept).cuda(), st)
+    ost, wpath, wlen = orc.commit(kd, vd, parent, accept, W.phi, ost, max_depth=ctx.max_depth)
+    assert host(clen).tolist() == [2] and host(path)[0, :2].tolist() == [0, 1]
+    np.testing.assert_array_equal(host(path), wpath)
+    check_state(st, ost, TOL[io])
+    assert int(st.pos[0]) == 256 + 16 + 2
