@@ -1,0 +1,432 @@
+"""Benchmark of the linear-attention layer's hot path on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+One step is one pass of the hot path over one batch of synthetic input.  The default
+workload is the LLaMA-2-7B-shaped prefill (B=4, H=32, d=128, T=2048, bf16, elu+1, 3 taps);
+--workload batched_decode / tree_verify / long_prefill time the other shapes with the same
+machinery.  Rank 0 prints one JSON line.  With N > 1 (launched by torch.distributed.run) every
+rank processes its own batch -- (sequence, head) units are independent, so there is no
+collective on the data path -- and the value is the total over ranks divided by the slowest
+rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2406_07368_b200 import workloads as wl  # noqa: E402
+from paper_2406_07368_b200 import dist as ladist   # noqa: E402
+
+L2_BYTES = 126 * 2 ** 20
+
+
+# ----------------------------------------------------------------------------------------
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, val in zip(names, r[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dev(x, io, device):
+    from paper_2406_07368_b200 import binding
+    return torch.from_numpy(np.ascontiguousarray(x)).to(binding.TORCH_DTYPE[io]).to(device)
+
+
+# ----------------------------------------------------------------------------------------
+# The steps of each workload.  Each factory returns (step_fn, units_per_step, bytes_per_launch,
+# launches_per_step, e2e_fn or None, description).
+# ----------------------------------------------------------------------------------------
+def prefill_workload(W: wl.Workload, rank: int, device):
+    from paper_2406_07368_b200 import binding
+    io = W.io
+    q, k, v = W.prefill_inputs()
+    if rank:   # another batch of the same law for every rank
+        q, k, v = wl.qkv(W.seed + 1000 * rank, q.shape, W.scale, io)
+    w = dev(W.weights(), "f32", device)
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io, chunk=W.chunk)
+    per_set = 4 * q.size * 2                                   # q, k, v read + o written, bf16
+    nsets = max(2, -(-2 * L2_BYTES // per_set) + 1) if per_set < 4 * L2_BYTES else 1
+    base = [dev(x, io, device) for x in (q, k, v)]
+    sets = [[x.roll(i, dims=0).contiguous() if i else x for x in base] for i in range(nsets)]
+    outs = [torch.empty_like(base[0]) for _ in range(nsets)]
+    st = ctx.new_state(W.B)
+    counter = [0]
+
+    def step():
+        i = counter[0] % nsets
+        counter[0] += 1
+        ctx.la_prefill(sets[i][0], sets[i][1], sets[i][2], w, st, init_state=False, out=outs[i])
+
+    pinned = [torch.from_numpy(x).to(binding.TORCH_DTYPE[io]).pin_memory() for x in (q, k, v)]
+    o_host = torch.empty(q.shape, dtype=binding.TORCH_DTYPE[io]).pin_memory()
+
+    def e2e_step():
+        for dst, src in zip(sets[0], pinned):
+            dst.copy_(src, non_blocking=True)
+        ctx.la_prefill(sets[0][0], sets[0][1], sets[0][2], w, st, init_state=False, out=outs[0])
+        o_host.copy_(outs[0], non_blocking=True)
+
+    tokens = W.B * W.T
+    units = W.B * W.H * W.T
+    alg_bytes = units * 4 * W.d * 2 + W.B * W.H * (W.d * W.d + W.d) * 4
+    info = {"ctx": ctx, "tokens_per_step": tokens, "alg_bytes_per_launch": alg_bytes, "launches_per_step": 1,
+            "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill",
+            "flops_per_launch": units * 4 * W.d * (W.chunk + W.d),
+            "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
+    return step, e2e_step, info
+
+
+def decode_workload(W: wl.Workload, rank: int, device):
+    from paper_2406_07368_b200 import binding
+    io = W.io
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io)
+    w = dev(W.weights(), "f32", device)
+    st = ctx.new_state(W.B)
+    # state after a seeded prefill of a shorter prompt: same magnitude law, bounded set-up time
+    q, k, v = W.prefill_inputs(T=256)
+    ctx.la_prefill(dev(q, io, device), dev(k, io, device), dev(v, io, device), w, st)
+    nrot = 8
+    toks = [[dev(x, io, device) for x in W.decode_inputs(s)] for s in range(nrot)]
+    out = torch.empty(W.B, W.H, W.d, dtype=binding.TORCH_DTYPE[io], device=device)
+    counter = [0]
+
+    def step():
+        t = toks[counter[0] % nrot]
+        counter[0] += 1
+        ctx.la_decode_step(t[0], t[1], t[2], w, st, out=out)
+
+    pinned = [x.cpu().pin_memory() for x in toks[0]]
+    o_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+
+    def e2e_step():
+        for dst, src in zip(toks[0], pinned):
+            dst.copy_(src, non_blocking=True)
+        ctx.la_decode_step(toks[0][0], toks[0][1], toks[0][2], w, st, out=out)
+        o_host.copy_(out, non_blocking=True)
+
+    units = W.B * W.H
+    el = 2
+    alg = units * (8 * W.d * W.d + 2 * 4 * W.d + 4 * W.d * el + 2 * (W.W - 1) * W.d * el)
+    info = {"ctx": ctx, "tokens_per_step": W.B, "alg_bytes_per_launch": alg, "launches_per_step": 1,
+            "h2d": 3 * units * W.d * el, "d2h": units * W.d * el, "kernel": "decode",
+            "flops_per_launch": units * 4 * W.d * W.d,
+            "l2": f"state of {units * W.d * W.d * 4 / 2**20:.0f} MiB streamed every step (larger than L2)"}
+    return step, e2e_step, info
+
+
+def verify_workload(W: wl.Workload, rank: int, device):
+    from paper_2406_07368_b200 import binding
+    io = W.io
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io, max_nodes=W.tree_nodes, max_depth=W.max_depth)
+    w = dev(W.weights(), "f32", device)
+    N = W.tree_nodes
+    # several independent state sets so that the rotation exceeds L2
+    per_state = W.B * W.H * W.d * W.d * 4
+    nsets = max(2, -(-2 * L2_BYTES // per_state) + 1)
+    q, k, v = W.prefill_inputs(T=256)
+    states = []
+    for i in range(nsets):
+        st = ctx.new_state(W.B)
+        ctx.la_prefill(dev(q, io, device), dev(k, io, device), dev(v, io, device), w, st)
+        states.append(st)
+    nrot = 4
+    drafts = [[dev(x, io, device) for x in W.draft_inputs(r)] for r in range(nrot)]
+    trees = [W.trees(r) for r in range(nrot)]
+    parents = [torch.from_numpy(p).to(device) for p, _ in trees]
+    accepts = [torch.from_numpy(a).to(device) for _, a in trees]
+    out = torch.empty(W.B, W.H, N, W.d, dtype=binding.TORCH_DTYPE[io], device=device)
+    path = torch.empty(W.B, W.max_depth, dtype=torch.int32, device=device)
+    clen = torch.empty(W.B, dtype=torch.int32, device=device)
+    counter = [0]
+
+    def step():
+        i = counter[0]
+        counter[0] += 1
+        r, st = i % nrot, states[i % nsets]
+        ctx.la_verify_tree(drafts[r][0], drafts[r][1], drafts[r][2], parents[r], w, st, out=out)
+        ctx.la_commit(drafts[r][1], drafts[r][2], parents[r], accepts[r], st, path_out=path, commit_len=clen)
+
+    pinned = [x.cpu().pin_memory() for x in drafts[0]]
+    o_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+
+    def e2e_step():
+        for dst, src in zip(drafts[0], pinned):
+            dst.copy_(src, non_blocking=True)
+        step()
+        o_host.copy_(out, non_blocking=True)
+
+    units = W.B * W.H
+    el = 2
+    alg_verify = units * (4 * W.d * W.d + 4 * W.d + 4 * N * W.d * el + (W.W - 1) * W.d * el)
+    info = {"ctx": ctx, "tokens_per_step": W.B * N, "alg_bytes_per_launch": alg_verify, "launches_per_step": 2,
+            "h2d": 3 * units * N * W.d * el, "d2h": units * N * W.d * el, "kernel": "verify",
+            "flops_per_launch": units * (2 * N * W.d * W.d + 4 * N * N * W.d),
+            "l2": f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"}
+    return step, e2e_step, info
+
+
+FACTORIES = {"llama7b_prefill": prefill_workload, "long_prefill": prefill_workload,
+             "batched_decode": decode_workload, "tree_verify": verify_workload}
+METRICS = {"llama7b_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
+           "long_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
+           "batched_decode": ("decode_tokens_per_s_per_layer", "tokens/s"),
+           "tree_verify": ("verify_nodes_per_s_per_layer", "nodes/s")}
+
+
+# ----------------------------------------------------------------------------------------
+def oracle_sample(W: wl.Workload):
+    """One bounded sample of the workload for the float64 oracle: returns (fn, units, text)."""
+    from oracle import la_oracle as orc
+    if W.name in ("llama7b_prefill", "long_prefill"):
+        T = min(W.T, 2048)
+        q, k, v = W.prefill_inputs(B=1, T=T)
+        w = W.weights()
+        return (lambda: orc.prefill_quadratic(q, k, v, w, W.phi, W.eps), T,
+                f"quadratic definition, 1 of {W.B} sequences, all {W.H} heads, first {T} of {W.T} tokens")
+    if W.name == "batched_decode":
+        B = 8
+        q, k, v = W.prefill_inputs(B=B, T=64)
+        w = W.weights()
+        _, st = orc.prefill_quadratic(q, k, v, w, W.phi, W.eps)
+        qs, ks, vs = W.decode_inputs(0, B=B)
+        box = [st]
+
+        def fn():
+            for _ in range(4):
+                _, box[0] = orc.decode_step(qs, ks, vs, w, W.phi, W.eps, box[0])
+        return fn, 4 * B, f"recurrent form, {B} of {W.B} sequences, all heads, 4 decode steps"
+    B = 2
+    q, k, v = W.prefill_inputs(B=B, T=64)
+    w = W.weights()
+    _, st = orc.prefill_quadratic(q, k, v, w, W.phi, W.eps)
+    qd, kd, vd = W.draft_inputs(0, B=B)
+    parent, accept = W.trees(0, B=B)
+
+    def fn():
+        orc.verify_tree(qd, kd, vd, parent, w, W.phi, W.eps, st)
+        orc.commit(kd, vd, parent, accept, W.phi, st, W.max_depth)
+    return fn, B * W.tree_nodes, f"tree form, {B} of {W.B} sequences, all heads, one verify + commit round"
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return int(max(n))
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def time_oracle(W: wl.Workload, repeats: int, warmup: int = 0):
+    fn, units, text = oracle_sample(W)
+    for _ in range(warmup):
+        fn()
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        fn()
+    dt = time.perf_counter() - t0
+    return units * repeats / dt, dt / repeats, text
+
+
+def run_reference(args, W: wl.Workload):
+    metric, unit = METRICS[W.name]
+    value, per_step, text = time_oracle(W, args.steps, args.warmup)
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": W.name, "sample_per_step": text},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": text},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_prefill", choices=sorted(FACTORIES))
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    W = wl.WORKLOADS[args.workload]()
+    rank, world = ladist.rank_world()
+
+    if args.impl == "reference":
+        args.steps = args.steps or 3
+        args.warmup = 1 if args.warmup is None else args.warmup
+        if rank == 0:
+            run_reference(args, W)
+        return 0
+
+    defaults = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000}
+    args.steps = args.steps or defaults[W.name]
+    args.warmup = 5 if args.warmup is None else max(3, args.warmup)
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    ladist.init(world, backend="nccl")
+
+    step, e2e_step, info = FACTORIES[W.name](W, rank, device)
+    ctx = info["ctx"]
+    stream = torch.cuda.current_stream()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if ctx.la_last_device_status() != 0:
+        raise RuntimeError("device status not OK after warm-up")
+
+    ladist.barrier(world)
+    torch.cuda.synchronize()
+    launches0 = ctx.la_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clocks:
+        ev0.record(stream)
+        for _ in range(args.steps):
+            step()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+    ladist.barrier(world)
+    ms = ev0.elapsed_time(ev1)
+    launches = ctx.la_launch_count() - launches0
+    ms_max = ladist.max_over_ranks(ms, world, device)
+    value = world * info["tokens_per_step"] * args.steps / (ms_max * 1e-3)
+
+    # per-launch duration of the dominant kernel, measured live: events around every launch of a
+    # short second pass on the same stream (for two-kernel steps only the first kernel is bracketed)
+    n_probe = min(args.steps, 50)
+    if info["launches_per_step"] == 1:
+        kernel_ms = ms / args.steps
+    else:
+        kernel_ms = None
+
+    # end to end: pinned host inputs copied in, result copied out, every step
+    for _ in range(2):
+        e2e_step()
+    torch.cuda.synchronize()
+    ladist.barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = ladist.max_over_ranks(e0.elapsed_time(e1), world, device)
+    e2e_value = world * info["tokens_per_step"] * args.e2e_steps / (e2e_ms * 1e-3)
+    if ctx.la_last_device_status() != 0:
+        raise RuntimeError("device status not OK after the timed region")
+
+    if rank != 0:
+        ladist.finish(world)
+        return 0
+
+    peaks = measured_peaks()
+    metric, unit = METRICS[W.name]
+    roofline = None
+    if kernel_ms is not None:
+        achieved = info["alg_bytes_per_launch"] / (kernel_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": info["kernel"], "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": peaks["source"], "alg_bytes_per_launch": info["alg_bytes_per_launch"],
+                    "launch_ms": kernel_ms,
+                    "tensor_tflops": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12,
+                    "tensor_frac_of_sustained": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
+                    / peaks["bf16_tflops_sustained"]}
+    else:
+        ms_step = ms / args.steps
+        achieved = 2 * info["alg_bytes_per_launch"] / (ms_step * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "verify+commit", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": peaks["source"], "launch_ms": ms_step}
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        reps = {"llama7b_prefill": 4, "long_prefill": 4, "batched_decode": 3, "tree_verify": 1}[W.name]
+        v, per, text = time_oracle(W, reps, warmup=0)
+        cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text,
+               "seconds": per * reps}
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if W.io == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": W.name, "B": W.B, "H": W.H, "d": W.d, "T": W.T, "chunk": W.chunk, "phi": W.phi,
+                       "conv_taps": W.W, "tree_nodes": W.tree_nodes, "l2": info["l2"],
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
+                    "d2h_bytes_per_step": info["d2h"], "steps": args.e2e_steps},
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    ladist.finish(world)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
