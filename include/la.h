@@ -50,7 +50,8 @@ typedef enum {
   LA_ERR_CUDA = 3,          /* a CUDA runtime or driver call failed */
   LA_ERR_BAD_TREE = 4,      /* device: parent[n] not in [-1, n), path deeper than max_depth,
                                accepted node outside [-1, N) */
-  LA_ERR_TIMEOUT = 5        /* device: a bounded wait on an asynchronous copy or MMA ran out */
+  LA_ERR_TIMEOUT = 5,       /* device: a bounded wait on an asynchronous copy or MMA ran out */
+  LA_ERR_TOO_LARGE = 6      /* a size exceeds the fixed capacity of an entry point that cannot allocate */
 } la_status;
 
 typedef enum { LA_PHI_ELU1 = 0,   /* phi(x) = x + 1 for x > 0, exp(x) otherwise */
@@ -62,6 +63,7 @@ typedef enum { LA_F32 = 0, LA_BF16 = 1 } la_dtype;
 /* Limits of this build. */
 #define LA_MAX_TAPS   32   /* W */
 #define LA_MAX_NODES  64   /* N, one 64-bit ancestor mask per node */
+#define LA_NOALLOC_MAX_SEQ 1024   /* largest B of la_verify_tree_noalloc */
 
 typedef struct {
   int32_t  H;           /* heads */
@@ -150,6 +152,39 @@ la_status la_verify_tree(la_ctx* ctx, int32_t B, int32_t N, const void* q, const
 la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void* v, const int32_t* parent,
                     const int32_t* accept_node, la_state* st /*host struct*/, int32_t* path_out,
                     int32_t* commit_len, void* stream);
+
+/* Tree verification for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for the way the library is embedded.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a serving loop
+ * whose memory was handed out up front by a pool that owns the whole device, in a plug-in
+ * that is given a fixed workspace and a stream and nothing else, or at a point where an
+ * allocation's implicit synchronisation would stall other streams.  Such a caller cannot
+ * use la_create, because the context allocates its status word.
+ *
+ * It computes exactly what la_verify_tree computes, from the same arguments, with the
+ * configuration passed directly instead of a context, on the device that is current at the
+ * call.  It calls no allocating routine.  Its only scratch memory, one status word per
+ * sequence, is a fixed array inside the library image; each GPU that loads the library
+ * carries those LA_NOALLOC_MAX_SEQ * 4 bytes until the process ends.
+ *
+ *   B           1 .. LA_NOALLOC_MAX_SEQ; a larger batch is refused with LA_ERR_TOO_LARGE
+ *               before anything is launched (split the batch instead)
+ *   seq_status  [B] int32 device buffer or NULL.  If given, after the kernel it receives,
+ *               per sequence, LA_OK or LA_ERR_BAD_TREE (that sequence's outputs were then
+ *               left unwritten).
+ *   other arguments as for la_verify_tree; cfg->max_nodes, max_depth and chunk are ignored
+ *   (N is limited by LA_MAX_NODES).
+ *
+ * The first call on each device looks up the device address of the fixed array; make that
+ * first call outside any stream capture.  All calls share the array, which still holds the
+ * previous call's codes on entry, so every call first clears the B words it uses, on
+ * `stream`.  Two calls that overlap on the GPU (different streams, no ordering between
+ * them) race on those words: keep calls to this entry point ordered on one device. */
+la_status la_verify_tree_noalloc(const la_config* cfg /*host*/, int32_t B, int32_t N, const void* q,
+                                 const void* k, const void* v, const int32_t* parent, const float* conv_w,
+                                 const la_state* st /*host struct*/, void* o, int32_t* seq_status,
+                                 void* stream);
 
 /* Waits for `stream`, then returns the sticky device status (LA_OK if no kernel reported a
  * problem since the last la_clear_device_status). */

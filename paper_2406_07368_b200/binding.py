@@ -16,15 +16,15 @@ import torch
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libla_b200.so")
 _lib = None
 
-LA_OK, LA_ERR_INVALID_ARG, LA_ERR_UNSUPPORTED, LA_ERR_CUDA, LA_ERR_BAD_TREE, LA_ERR_TIMEOUT = range(6)
+LA_OK, LA_ERR_INVALID_ARG, LA_ERR_UNSUPPORTED, LA_ERR_CUDA, LA_ERR_BAD_TREE, LA_ERR_TIMEOUT, LA_ERR_TOO_LARGE = range(7)
 LA_PHI = {"elu1": 0, "relu": 1}
 LA_DTYPE = {"f32": 0, "bf16": 1}
 TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
-LA_MAX_TAPS, LA_MAX_NODES = 32, 64
+LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
-           "la_launch_count"]
+           "la_launch_count", "la_verify_tree_noalloc"]
 
 
 class LaError(RuntimeError):
@@ -60,6 +60,8 @@ def lib() -> C.CDLL:
         L.la_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
+        L.la_verify_tree_noalloc.argtypes = [C.POINTER(la_config), i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state),
+                                             vp, vp, vp]
         L.la_last_device_status.argtypes = [vp, vp]
         L.la_clear_device_status.argtypes = [vp, vp]
         L.la_set_prefill_kernel.argtypes = [vp, i32]
@@ -219,3 +221,23 @@ class Context:
 
     def la_launch_count(self) -> int:
         return int(lib().la_launch_count(self._h))
+
+
+def la_verify_tree_noalloc(H: int, d: int, conv_taps: int, phi: str, eps: float, io: str, q, k, v, parent, conv_w,
+                           state: State, out, seq_status=None, stream=None) -> None:
+    """Tree verification without a context, for callers that are not allowed to allocate.
+
+    Every buffer, including `out` ([B, H, N, d]) and the optional per-sequence status
+    `seq_status` ([B] int32), is supplied by the caller; neither this wrapper nor the C entry
+    point behind it allocates device memory.  See la_verify_tree_noalloc in include/la.h for
+    the batch limit and the rule about overlapping calls.
+    """
+    B, _, N, _ = q.shape
+    dt = TORCH_DTYPE[io]
+    shp = (B, H, N, d)
+    cfg = la_config(H, d, conv_taps, 0, LA_PHI[phi], eps, LA_DTYPE[io], LA_MAX_NODES, LA_MAX_NODES)
+    cs = state.c()
+    _check("la_verify_tree_noalloc", lib().la_verify_tree_noalloc(
+        C.byref(cfg), B, N, _ptr(q, dt, shp, "q"), _ptr(k, dt, shp, "k"), _ptr(v, dt, shp, "v"),
+        _ptr(parent, torch.int32, (B, N), "parent"), _ptr(conv_w, torch.float32, (H, d, conv_taps), "conv_w"),
+        C.byref(cs), _ptr(out, dt, shp, "o"), _ptr(seq_status, torch.int32, (B,), "seq_status"), _stream(stream)))

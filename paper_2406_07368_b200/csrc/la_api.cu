@@ -39,6 +39,7 @@ const char* la_status_str(la_status s) {
     case LA_ERR_CUDA: return "LA_ERR_CUDA";
     case LA_ERR_BAD_TREE: return "LA_ERR_BAD_TREE";
     case LA_ERR_TIMEOUT: return "LA_ERR_TIMEOUT";
+    case LA_ERR_TOO_LARGE: return "LA_ERR_TOO_LARGE";
   }
   return "LA_ERR_UNKNOWN";
 }

@@ -24,7 +24,8 @@ template <int D> struct VerifySmem {
   int bad;
 };
 
-template <typename T, int D, int PHI>
+// PER_SEQ = false: `status` is one sticky word.  PER_SEQ = true: `status` has one word per sequence.
+template <typename T, int D, int PHI, bool PER_SEQ = false>
 __global__ void __launch_bounds__(256)
 verify_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
               const int32_t* __restrict__ parent, const float* __restrict__ w, const float* __restrict__ S,
@@ -58,7 +59,7 @@ verify_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restr
   }
   __syncthreads();
   if (sm.bad) {
-    if (t == 0) report(status, LA_ERR_BAD_TREE);
+    if (t == 0) report(PER_SEQ ? status + b : status, LA_ERR_BAD_TREE);
     return;
   }
 
@@ -167,11 +168,11 @@ verify_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restr
   }
 }
 
-template <typename T, int D, int PHI>
+template <typename T, int D, int PHI, bool PER_SEQ = false>
 static cudaError_t launch_t(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
                             const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s) {
   const la_config& c = ctx->cfg;
-  auto kern = verify_kernel<T, D, PHI>;
+  auto kern = verify_kernel<T, D, PHI, PER_SEQ>;
   const size_t smem = sizeof(VerifySmem<D>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
@@ -198,4 +199,97 @@ cudaError_t launch_verify(la_ctx* ctx, int B, int N, const void* q, const void* 
                    : launch_phi<__nv_bfloat16, 128>(ctx, B, N, q, k, v, parent, w, st, o, s);
 }
 
+// ---- the same kernel with one status word per sequence (used by la_verify_tree_noalloc) ----
+template <typename T, int D>
+static cudaError_t launch_phi_per_seq(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
+                                      const int32_t* parent, const float* w, const la_state& st, void* o,
+                                      cudaStream_t s) {
+  return ctx->cfg.phi == LA_PHI_ELU1
+             ? launch_t<T, D, LA_PHI_ELU1, true>(ctx, B, N, q, k, v, parent, w, st, o, s)
+             : launch_t<T, D, LA_PHI_RELU, true>(ctx, B, N, q, k, v, parent, w, st, o, s);
+}
+
+static cudaError_t launch_verify_per_seq(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
+                                         const int32_t* parent, const float* w, const la_state& st, void* o,
+                                         cudaStream_t s) {
+  const la_config& c = ctx->cfg;
+  if (c.io_dtype == LA_F32)
+    return c.d == 64 ? launch_phi_per_seq<float, 64>(ctx, B, N, q, k, v, parent, w, st, o, s)
+                     : launch_phi_per_seq<float, 128>(ctx, B, N, q, k, v, parent, w, st, o, s);
+  return c.d == 64 ? launch_phi_per_seq<__nv_bfloat16, 64>(ctx, B, N, q, k, v, parent, w, st, o, s)
+                   : launch_phi_per_seq<__nv_bfloat16, 128>(ctx, B, N, q, k, v, parent, w, st, o, s);
+}
+
 }  // namespace la
+
+// =========================================================================================
+// la_verify_tree_noalloc: tree verification for callers that must not allocate.
+//
+// The regular path reports device-side problems through a status word that la_create
+// allocates with cudaMalloc.  Here that scratch lives in the library image instead: one
+// status word per sequence in a fixed array that every GPU loading the library carries
+// until the process exits (LA_NOALLOC_MAX_SEQ words = 4 KiB).
+//
+// In host code the name of a __device__ array is only a host-side handle, not an address
+// the GPU can use, so the device address is looked up once per device with
+// cudaGetSymbolAddress (with that device current) and then handed to the kernel.
+// =========================================================================================
+#include <mutex>
+
+static __device__ __align__(256) int g_noalloc_seq_status[LA_NOALLOC_MAX_SEQ];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+
+// Device address of g_noalloc_seq_status on the current device `dev`; looked up on first use.
+int* noalloc_scratch(int dev, cudaError_t* err) {
+  static std::mutex mu;
+  static int* addr[kMaxDevices] = {};
+  std::lock_guard<std::mutex> lock(mu);
+  *err = cudaSuccess;
+  if (addr[dev] == nullptr) {
+    void* p = nullptr;
+    *err = cudaGetSymbolAddress(&p, g_noalloc_seq_status);
+    if (*err != cudaSuccess) return nullptr;
+    addr[dev] = static_cast<int*>(p);
+  }
+  return addr[dev];
+}
+
+inline bool ok16(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" la_status la_verify_tree_noalloc(const la_config* cfg, int32_t B, int32_t N, const void* q, const void* k,
+                                            const void* v, const int32_t* parent, const float* conv_w,
+                                            const la_state* st, void* o, int32_t* seq_status, void* stream) {
+  if (!cfg || cfg->H < 1 || cfg->conv_taps < 1 || cfg->conv_taps > LA_MAX_TAPS) return LA_ERR_INVALID_ARG;
+  if (cfg->phi != LA_PHI_ELU1 && cfg->phi != LA_PHI_RELU) return LA_ERR_INVALID_ARG;
+  if (cfg->io_dtype != LA_F32 && cfg->io_dtype != LA_BF16) return LA_ERR_INVALID_ARG;
+  if (!(cfg->eps >= 0.f) || cfg->eps > 3.0e38f) return LA_ERR_INVALID_ARG;
+  if (cfg->d != 64 && cfg->d != 128) return LA_ERR_UNSUPPORTED;
+  if (B < 1 || N < 1 || N > LA_MAX_NODES) return LA_ERR_INVALID_ARG;
+  if (B > LA_NOALLOC_MAX_SEQ) return LA_ERR_TOO_LARGE;       // the fixed scratch has one word per sequence
+  if (!ok16(q) || !ok16(k) || !ok16(v) || !ok16(conv_w) || !ok16(o) || !parent) return LA_ERR_INVALID_ARG;
+  if (!st || !ok16(st->S) || !ok16(st->z) || (cfg->conv_taps > 1 && !ok16(st->win))) return LA_ERR_INVALID_ARG;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LA_ERR_CUDA;
+  cudaError_t e;
+  int* scratch = noalloc_scratch(dev, &e);
+  if (!scratch) return LA_ERR_CUDA;
+
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // The array keeps what the previous call left in it: clear the words this call uses.
+  if (cudaMemsetAsync(scratch, 0, sizeof(int) * B, s) != cudaSuccess) return LA_ERR_CUDA;
+  la_ctx tmp{};
+  tmp.cfg = *cfg;
+  tmp.device = dev;
+  tmp.d_status = scratch;
+  if (la::launch_verify_per_seq(&tmp, B, N, q, k, v, parent, conv_w, *st, o, s) != cudaSuccess) return LA_ERR_CUDA;
+  if (seq_status &&
+      cudaMemcpyAsync(seq_status, scratch, sizeof(int) * B, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+    return LA_ERR_CUDA;
+  return LA_OK;
+}
