@@ -3,20 +3,24 @@
 // Sec. 4.1: the sequence is cut into non-overlapping groups; inside a group the causally
 // masked product phi(Q) phi(K)^T V is formed in parallel, between groups only the cumulative
 // sums S = sum phi(k) v^T and z = sum phi(k) are carried.  One CTA walks one (batch, head)
-// chain in tiles of 128 tokens.  Per tile:
+// chain in tiles of 128 tokens.  The normaliser rides along on the tensor cores: V is
+// extended by a column of ones and S by the column z, so that
+//     [O | den] = phi(Q) [S | z]_prev + (P o M) [V | 1],     [S | z] += phi(K)^T [V | 1].
+// Per tile n:
 //
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
-//   CUDA     phi applied in place on Q and K; den_inter = phi(Q) z; z += colsum phi(K)
-//   tcgen05  P = phi(Q) phi(K)^T          (TMEM columns   0..127)
-//            O = phi(Q) S_prev            (TMEM columns 128..255; S_prev as a bf16 copy in smem)
-//   CUDA     P -> causal mask, row sums, bf16 -> smem
-//   tcgen05  O += P V ;  S += phi(K)^T V  (S fp32 in TMEM columns 256..383 for the whole chain)
-//   CUDA     o = O / den + conv(V)  -> smem -> TMA store;  S -> bf16 copy for the next tile
+//   group A  phi applied in place on Q and K (packed bf16x2 arithmetic, fp32 exp)
+//   tcgen05  P = phi(Q) phi(K)^T            -> TMEM buffer (n+1)&1 (idle until tile n+1 needs it)
+//            [O | den] = phi(Q) [S | z]_prev -> TMEM buffer n&1; [S | z]_prev is a bf16 copy in smem
+//            [S | z] += phi(K)^T [V | 1]     -> fp32 in TMEM for the whole chain
+//   group A  P -> causal mask, bf16 -> shared memory;  [S | z] -> bf16 copy for tile n+1
+//   tcgen05  [O | den] += (P o M) [V | 1]
+//   group B  o = O / (den + eps) + conv(V) -> global memory
 //
-// Warps 0-7 do the CUDA-core work (thread = one tile row / TMEM lane, two column halves),
-// warp 8 issues all TMA loads and all MMAs from one elected lane.  Every wait on an mbarrier
-// is bounded; when one runs out the CTA records LA_ERR_TIMEOUT, stops issuing work, frees its
-// TMEM and returns.
+// Three roles run concurrently: group A (warps 8-15), group B (warps 0-7) and warp 16, whose
+// elected lane issues every TMA load and every MMA.  While group B finishes tile n, group A
+// already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
+// records LA_ERR_TIMEOUT, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
 #include "la_common.cuh"
@@ -26,28 +30,35 @@ namespace tc {
 
 constexpr int D = 128;
 constexpr int TILE = 128;
-constexpr int kComputeThreads = 256;
-constexpr int kThreads = 288;
+constexpr int kThreadsB = 256;                     // group B: warps 0-7
+constexpr int kThreadsA = 256;                     // group A: warps 8-15
+constexpr int kCtrlWarp = 16;
+constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, TMEM_COLS = 512;
+// TMEM columns: two 128-column buffers that hold O of tile n (buffer n&1) and P of tile n (buffer (n+1)&1),
+// S, and three 16-column blocks whose first column is den (per O buffer) and z.
+constexpr uint32_t X_COL = 0, S_COL = 256, DEN_COL = 384, Z_COL = 416, TMEM_COLS = 512;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
-                   OFF_P = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES, OFF_SMALL = 6 * TILE_BYTES;
+                   OFF_P = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
+                   OFF_ONES = 6 * TILE_BYTES,      // [128 x 16] bf16, column 0 = 1: the extension of V
+                   OFF_SZ = OFF_ONES + 4096,       // [128 x 16] bf16, column 0 = z: the extension of the S copy
+                   OFF_SMALL = OFF_SZ + 4096;
 
 struct Small {
-  float zs[D];
-  float zpart[8][D];
-  float den_inter[2][TILE];
-  float den_intra[2][TILE];
-  unsigned long long bars[8];
+  unsigned long long bars[12];
   uint32_t tmem_base;
   int abort;
   int pad[2];
 };
-enum { B_FULL_QK = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA1 = 3, B_MMA2 = 4, B_PHI = 5, B_P = 6, B_EPI = 7 };
+// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B.
+// MMA_P / MMA_S / MMA_O: tcgen05.commit after P; after [O|den] = phi(Q)[S|z] and [S|z] += phi(K)^T[V|1];
+// after [O|den] += P[V|1].
+enum { B_FULL_QK = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
+       B_SB = 8, B_EPI = 9, kNumBars = 10 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
@@ -100,7 +111,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void compute_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void sync_group_b() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -152,29 +163,45 @@ __device__ __forceinline__ void mma_commit(uint32_t bar) {
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])           \
       : "memory")
 
+__device__ __forceinline__ uint32_t tmem_ld1(uint32_t taddr) {
+  uint32_t v;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(v) : "r"(taddr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t v) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(v) : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---- descriptors ----------------------------------------------------------------------------
-// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride byte offsets
-// (all in 16-byte units), descriptor version 1, layout type 2.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+// Shared-memory matrix descriptor: start address, leading and stride byte offsets (16-byte units),
+// descriptor version 1, layout type (2 = 128-byte swizzle, 0 = no swizzle).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
 }
 // Operand whose contraction index runs along the 128-byte rows (rows = M or N): step ks covers 16 elements.
 __device__ __forceinline__ uint64_t desc_kmajor(uint32_t tile, int ks) {
-  return smem_desc(tile + (uint32_t)(ks >> 2) * BOX_BYTES + (uint32_t)(ks & 3) * 32u, 16u, 1024u);
+  return smem_desc(tile + (uint32_t)(ks >> 2) * BOX_BYTES + (uint32_t)(ks & 3) * 32u, 16u, 1024u, 2u);
 }
 // Operand whose contraction index runs along the tile rows (rows = K, 128-byte rows hold M or N): step ks
 // covers 16 rows; the two 64-element column boxes are BOX_BYTES apart.
 __device__ __forceinline__ uint64_t desc_mnmajor(uint32_t tile, int ks) {
-  return smem_desc(tile + (uint32_t)ks * 2048u, BOX_BYTES, 1024u);
+  return smem_desc(tile + (uint32_t)ks * 2048u, BOX_BYTES, 1024u, 2u);
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128.
-__host__ __device__ constexpr uint32_t idesc(bool a_mn, bool b_mn) {
+// The 16-column extensions ([128 rows = K] x [16 = N], no swizzle): 8 x 8 cores of 128 bytes, the two cores of
+// one 8-row group side by side (stride 128 B along N), 8-row groups 256 B apart (stride along K).
+__device__ __forceinline__ uint64_t desc_ext(uint32_t tile, int ks) {
+  return smem_desc(tile + (uint32_t)ks * 512u, 256u, 128u, 0u);
+}
+__device__ __forceinline__ uint32_t ext_offset(int k, int n) {   // byte offset of element (k, n) in such a block
+  return (uint32_t)(k >> 3) * 256u + (uint32_t)(n >> 3) * 128u + (uint32_t)(k & 7) * 16u + (uint32_t)(n & 7) * 2u;
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n.
+__host__ __device__ constexpr uint32_t idesc(bool a_mn, bool b_mn, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-         ((128u >> 3) << 17) | ((128u >> 4) << 24);
+         ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // ---- bf16 packing ------------------------------------------------------------------------------
@@ -185,34 +212,62 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 __device__ __forceinline__ float lo_f(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float hi_f(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-template <int PHI> __device__ __forceinline__ float phi_fast(float x) {
-  if (PHI == LA_PHI_ELU1) return x > 0.f ? x + 1.f : __expf(x);
-  return fmaxf(x, 0.f);
-}
-
-// phi on 8 packed bf16 values; returns the rounded results packed, and their fp32 values in f[8].
-template <int PHI> __device__ __forceinline__ uint4 phi8(uint4 u, float* f) {
-  uint4 r;
-  r.x = pack2(phi_fast<PHI>(lo_f(u.x)), phi_fast<PHI>(hi_f(u.x)));
-  r.y = pack2(phi_fast<PHI>(lo_f(u.y)), phi_fast<PHI>(hi_f(u.y)));
-  r.z = pack2(phi_fast<PHI>(lo_f(u.z)), phi_fast<PHI>(hi_f(u.z)));
-  r.w = pack2(phi_fast<PHI>(lo_f(u.w)), phi_fast<PHI>(hi_f(u.w)));
-  f[0] = lo_f(r.x); f[1] = hi_f(r.x); f[2] = lo_f(r.y); f[3] = hi_f(r.y);
-  f[4] = lo_f(r.z); f[5] = hi_f(r.z); f[6] = lo_f(r.w); f[7] = hi_f(r.w);
+// phi on two packed bf16 values.  elu+1: x + 1 where x > 0 (one correctly rounded bf16 addition), exp(x)
+// elsewhere (fp32 exp2, rounded once to bf16); the two are merged with a lane mask.  ReLU: packed max.
+template <int PHI> __device__ __forceinline__ uint32_t phi2(uint32_t u) {
+  if (PHI == LA_PHI_ELU1) {
+    float e0, e1;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(lo_f(u) * 1.4426950408889634f));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(hi_f(u) * 1.4426950408889634f));
+    const uint32_t e = pack2(e0, e1);
+    uint32_t xp1, mask;
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(xp1) : "r"(u), "r"(0x3f803f80u));
+    asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(mask) : "r"(u), "r"(0u));
+    return (xp1 & mask) | (e & ~mask);
+  }
+  uint32_t r;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(u), "r"(0u));
   return r;
+}
+template <int PHI> __device__ __forceinline__ uint4 phi8(uint4 u) {
+  return make_uint4(phi2<PHI>(u.x), phi2<PHI>(u.y), phi2<PHI>(u.z), phi2<PHI>(u.w));
 }
 
 // Byte offset of 16-byte chunk `cc` (0..7) of row `row` inside one 128-byte-swizzled box.
 __device__ __forceinline__ uint32_t swz(int row, int cc) { return (uint32_t)row * 128u + (uint32_t)((cc ^ (row & 7)) << 4); }
 
 // ---- the kernel ------------------------------------------------------------------------------------
-template <int PHI>
+// Convolution part of the epilogue for one 8-channel chunk: acc[e] += sum_t w[t][ch] v_{row-t}[ch].
+template <int WT>
+__device__ __forceinline__ void conv8(float* acc, int W, int r, int cc, int ch0, const unsigned char* Vbox,
+                                      const __nv_bfloat16* halo, const float* wsm) {
+  const int taps = WT > 0 ? WT : W;
+#pragma unroll
+  for (int t = 0; t < taps; ++t) {
+    const int row = r - t;
+    uint4 u;
+    if (row >= 0) u = *reinterpret_cast<const uint4*>(Vbox + swz(row, cc));
+    else u = *reinterpret_cast<const uint4*>(halo + (W - 1 + row) * D + ch0);
+    const float4 w0 = *reinterpret_cast<const float4*>(wsm + t * D + ch0);
+    const float4 w1 = *reinterpret_cast<const float4*>(wsm + t * D + ch0 + 4);
+    acc[0] = fmaf(w0.x, lo_f(u.x), acc[0]); acc[1] = fmaf(w0.y, hi_f(u.x), acc[1]);
+    acc[2] = fmaf(w0.z, lo_f(u.y), acc[2]); acc[3] = fmaf(w0.w, hi_f(u.y), acc[3]);
+    acc[4] = fmaf(w1.x, lo_f(u.z), acc[4]); acc[5] = fmaf(w1.y, hi_f(u.z), acc[5]);
+    acc[6] = fmaf(w1.z, lo_f(u.w), acc[6]); acc[7] = fmaf(w1.w, hi_f(u.w), acc[7]);
+  }
+}
+
+__device__ __forceinline__ uint4 pack8(const uint32_t* v) {
+  return make_uint4(pack2(__uint_as_float(v[0]), __uint_as_float(v[1])), pack2(__uint_as_float(v[2]), __uint_as_float(v[3])),
+                    pack2(__uint_as_float(v[4]), __uint_as_float(v[5])), pack2(__uint_as_float(v[6]), __uint_as_float(v[7])));
+}
+
+template <int PHI, int WT>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
-                  const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
-                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int* status, int H, int T, int W,
-                  float eps, int init) {
+                  const __grid_constant__ CUtensorMap mv, const float* __restrict__ w, float* __restrict__ S,
+                  float* __restrict__ z, __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos,
+                  __nv_bfloat16* __restrict__ o, int* status, int H, int T, int W, float eps, int init) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -224,25 +279,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bh = blockIdx.x, h = bh % H;
   const int nchunks = (T + TILE - 1) / TILE;
-  uint32_t bar[8];
+  uint32_t bar[kNumBars];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) bar[i] = smem_u32(&sm.bars[i]);
+  for (int i = 0; i < kNumBars; ++i) bar[i] = smem_u32(&sm.bars[i]);
 
   // ---- set-up ----
   if (tid == 0) {
     mbar_init(bar[B_FULL_QK], 1);
     mbar_init(bar[B_FULL_V0], 1);
     mbar_init(bar[B_FULL_V1], 1);
-    mbar_init(bar[B_MMA1], 1);
-    mbar_init(bar[B_MMA2], 1);
-    mbar_init(bar[B_PHI], kComputeThreads);
-    mbar_init(bar[B_P], kComputeThreads);
-    mbar_init(bar[B_EPI], kComputeThreads);
+    mbar_init(bar[B_MMA_P], 1);
+    mbar_init(bar[B_MMA_S], 1);
+    mbar_init(bar[B_MMA_O], 1);
+    mbar_init(bar[B_PHI], kThreadsA);
+    mbar_init(bar[B_PDONE], kThreadsA);
+    mbar_init(bar[B_SB], kThreadsA);
+    mbar_init(bar[B_EPI], kThreadsB);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_proxy_async();
   }
-  if (warp == 8) {
+  if (warp == kCtrlWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
                  "r"(TMEM_COLS)
                  : "memory");
@@ -251,13 +307,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
     halo[idx] = init ? win[(size_t)bh * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
-  if (tid < D) sm.zs[tid] = init ? z[(size_t)bh * D + tid] : 0.f;
+  for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
+    reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  if (tid < TILE) {
+    *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
+    if (init)
+      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)bh * D + tid]);
+  }
+  fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  if (warp == 8) {
+  if (warp == kCtrlWarp) {
     // =============================== TMA + MMA issue (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
@@ -271,68 +335,84 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, n * TILE, bh, bar[B_FULL_V0 + n]);
         tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, n * TILE, bh, bar[B_FULL_V0 + n]);
       }
-      for (int n = 0; n < nchunks && ok; ++n) {
+      for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
         const uint32_t vbuf = sbase + OFF_V0 + par * TILE_BYTES;
+        const uint32_t ocol = tmem + X_COL + par * 128, pcol = tmem + X_COL + (par ^ 1) * 128;
+        const uint32_t dcol = tmem + DEN_COL + par * 16;
         const bool has_state = init || n > 0;
-        ok = mbar_wait(bar[B_PHI], par, abort);
+        ok = mbar_wait(bar[B_PHI], par, abort);                 // phi(Q), phi(K) of tile n are in place
         if (!ok) break;
+        if (n >= 1) {
+          // group B is done with tile n-1: its TMEM buffer takes P of tile n, its V buffer takes tile n+1
+          ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
+          if (!ok) break;
+          if (n + 1 < nchunks) {
+            const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
+            mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
+            tma_load(vnext, &mv, 0, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+            tma_load(vnext + BOX_BYTES, &mv, 64, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+          }
+        }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T
-          mma_bf16(tmem + P_COL, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(sbase + OFF_K, ks), idesc(false, false),
-                   ks > 0);
+          mma_bf16(pcol, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(sbase + OFF_K, ks), idesc(false, false, 128), ks > 0);
+        mma_commit(bar[B_MMA_P]);
+        // the bf16 copy of [S|z] before tile n is complete (and S itself has been read) after n + 1 arrivals
+        ok = mbar_wait(bar[B_SB], par, abort) && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
+        if (!ok) break;
+        tc_fence_after();
         if (has_state) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)   // O = phi(Q) S_prev
-            mma_bf16(tmem + O_COL, desc_kmajor(sbase + OFF_Q, ks), desc_mnmajor(sbase + OFF_S, ks), idesc(false, true),
-                     ks > 0);
+          for (int ks = 0; ks < 8; ++ks) {   // [O | den] = phi(Q) [S | z]_prev
+            const uint64_t qd = desc_kmajor(sbase + OFF_Q, ks);
+            mma_bf16(ocol, qd, desc_mnmajor(sbase + OFF_S, ks), idesc(false, true, 128), ks > 0);
+            mma_bf16(dcol, qd, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
+          }
         }
-        mma_commit(bar[B_MMA1]);
-        ok = mbar_wait(bar[B_P], par, abort) && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {     // [S | z] += phi(K)^T [V | 1]
+          const uint64_t kd = desc_mnmajor(sbase + OFF_K, ks);
+          mma_bf16(tmem + S_COL, kd, desc_mnmajor(vbuf, ks), idesc(true, true, 128), has_state || ks > 0);
+          mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
+        }
+        mma_commit(bar[B_MMA_S]);
+        ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in shared memory
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // O += (P o M) V
-          mma_bf16(tmem + O_COL, desc_kmajor(sbase + OFF_P, ks), desc_mnmajor(vbuf, ks), idesc(false, true),
-                   has_state || ks > 0);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // S += phi(K)^T V
-          mma_bf16(tmem + S_COL, desc_mnmajor(sbase + OFF_K, ks), desc_mnmajor(vbuf, ks), idesc(true, true),
-                   has_state || ks > 0);
-        mma_commit(bar[B_MMA2]);
+        for (int ks = 0; ks < 8; ++ks) {     // [O | den] += (P o M) [V | 1]
+          const uint64_t pd = desc_kmajor(sbase + OFF_P, ks);
+          mma_bf16(ocol, pd, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
+          mma_bf16(dcol, pd, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
+        }
+        mma_commit(bar[B_MMA_O]);
         if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA1], par, abort);      // Q tile is free
+          ok = mbar_wait(bar[B_MMA_S], par, abort);             // Q and K buffers are free
           if (!ok) break;
           mbar_expect_tx(bar[B_FULL_QK], 2 * TILE_BYTES);
           tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-          ok = mbar_wait(bar[B_MMA2], par, abort);      // K tile is free
-          if (!ok) break;
           tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
           tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
         }
-        if (n + 2 < nchunks) {
-          ok = mbar_wait(bar[B_EPI], par, abort);       // V buffer `par` is free
-          if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_V0 + par], TILE_BYTES);
-          tma_load(vbuf, &mv, 0, (n + 2) * TILE, bh, bar[B_FULL_V0 + par]);
-          tma_load(vbuf + BOX_BYTES, &mv, 64, (n + 2) * TILE, bh, bar[B_FULL_V0 + par]);
-        }
       }
     }
-  } else {
-    // =============================== CUDA-core work (256 threads) ===============================
-    const int r = 32 * (warp & 3) + lane;         // tile row = TMEM lane
-    const int hf = warp >> 2;                     // column half
-    const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+  } else if (warp >= 8) {
+    // =============================== group A: phi, P, [S|z] snapshot (256 threads) ===============================
+    const int ta = tid - kThreadsB;               // 0..255
+    const int wa = warp - 8;                      // 0..7
+    const int r = 32 * (wa & 3) + lane;           // tile row = TMEM lane
+    const int hf = wa >> 2;                       // column half
+    const uint32_t lane_addr = (uint32_t)(32 * (wa & 3)) << 16;
     unsigned char* Qb = smem + OFF_Q + hf * BOX_BYTES;
     unsigned char* Pb = smem + OFF_P + hf * BOX_BYTES;
     unsigned char* Sb = smem + OFF_S + hf * BOX_BYTES;
     float* Sg = S + (size_t)bh * D * D + (size_t)r * D + 64 * hf;
     bool ok = true;
 
-    if (init) {   // S -> TMEM (fp32) and -> bf16 copy in shared memory
+    if (init) {   // [S|z] -> TMEM (fp32); S -> bf16 copy in shared memory (z was copied during set-up)
 #pragma unroll
       for (int qq = 0; qq < 2; ++qq) {
         uint32_t v[32];
@@ -344,151 +424,77 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         }
         LA_TMEM_ST32(tmem + lane_addr + S_COL + 64 * hf + 32 * qq, v);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint4 u;
-          u.x = pack2(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1]));
-          u.y = pack2(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3]));
-          u.z = pack2(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5]));
-          u.w = pack2(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7]));
-          *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = u;
-        }
+        for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
+      }
+      if (hf == 0) {
+        tmem_st1(tmem + lane_addr + Z_COL, __float_as_uint(z[(size_t)bh * D + r]));
+#pragma unroll
+        for (int c = 1; c < 16; ++c) tmem_st1(tmem + lane_addr + Z_COL + c, 0u);
       }
       tmem_wait_st();
-      tc_fence_before();
     }
+    fence_proxy_async();
+    tc_fence_before();
+    mbar_arrive(bar[B_SB]);                       // phase 0: the state before tile 0 is in place
 
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
       const int valid = min(TILE, T - n * TILE);
-      unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;    // whole V tile (both boxes)
       const bool last = n + 1 == nchunks;
+      const uint32_t pcol = tmem + X_COL + (par ^ 1) * 128;
 
-      // ---- phi on Q and K in place; den_inter = phi(Q).z_prev; column sums of phi(K) ----
+      // ---- phi on Q and K in place ----
       ok = ok && mbar_wait(bar[B_FULL_QK], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
-        float dot = 0.f;
 #pragma unroll
         for (int cc = 0; cc < 8; ++cc) {
           uint4* p = reinterpret_cast<uint4*>(Qb + swz(r, cc));
-          float f[8];
-          *p = phi8<PHI>(*p, f);
-          const float* zz = &sm.zs[64 * hf + 8 * cc];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) dot = fmaf(f[e], zz[e], dot);
+          *p = phi8<PHI>(*p);
         }
-        sm.den_inter[hf][r] = dot;
-
-        const int ct = tid & 15, rg = tid >> 4;                 // chunk column 0..15, row group 0..15
+        const int ct = ta & 15, rg = ta >> 4;                   // chunk column 0..15, row group 0..15
         unsigned char* Kb = smem + OFF_K + (ct >> 3) * BOX_BYTES;
-        float cs[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) cs[e] = 0.f;
 #pragma unroll
         for (int m = 0; m < 8; ++m) {
           const int j = rg + 16 * m;
           uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-          if (j < valid) {
-            float f[8];
-            *p = phi8<PHI>(*p, f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) cs[e] += f[e];
-          } else {
-            *p = make_uint4(0u, 0u, 0u, 0u);                    // rows past the end contribute nothing
-          }
-        }
-#pragma unroll
-        for (int e = 0; e < 8; ++e) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], 16);
-        if (lane < 16) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) sm.zpart[warp][8 * ct + e] = cs[e];
+          *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);   // rows past the end contribute nothing
         }
       }
       fence_proxy_async();
-      tc_fence_before();
       mbar_arrive(bar[B_PHI]);
-      if (tid == 0) tma_wait_read();                            // the previous output tile has left shared memory
-      compute_sync();
-      if (tid < D && ok) {
-        float a = sm.zs[tid];
-#pragma unroll
-        for (int ww = 0; ww < 8; ++ww) a += sm.zpart[ww][tid];
-        sm.zs[tid] = a;
-      }
 
-      // ---- P: causal mask, row sums, bf16 -> shared memory ----
-      ok = ok && mbar_wait(bar[B_MMA1], par, abort);
+      // ---- P: causal mask, bf16 -> shared memory ----
+      ok = ok && mbar_wait(bar[B_MMA_P], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
-        float rowsum = 0.f;
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           const int col0 = 64 * hf + 32 * qq;
           uint32_t v[32];
-          if (col0 <= 32 * (warp & 3) + 31) {                   // warp-uniform: some row of this warp reaches col0
-            LA_TMEM_LD32(tmem + lane_addr + P_COL + col0, v);
+          if (col0 <= 32 * (wa & 3) + 31) {                     // warp-uniform: some row of this warp reaches col0
+            LA_TMEM_LD32(pcol + lane_addr + col0, v);
             tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) v[e] = col0 + e <= r ? v[e] : 0u;
           } else {
 #pragma unroll
             for (int e = 0; e < 32; ++e) v[e] = 0u;
           }
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t pk[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int j = col0 + 8 * c + 2 * e;
-              const float a = j <= r ? __uint_as_float(v[8 * c + 2 * e]) : 0.f;
-              const float b = j + 1 <= r ? __uint_as_float(v[8 * c + 2 * e + 1]) : 0.f;
-              pk[e] = pack2(a, b);
-              rowsum += lo_f(pk[e]) + hi_f(pk[e]);
-            }
-            *reinterpret_cast<uint4*>(Pb + swz(r, 4 * qq + c)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-          }
+          for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Pb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
         }
-        sm.den_intra[hf][r] = rowsum;
       }
       fence_proxy_async();
       tc_fence_before();
-      mbar_arrive(bar[B_P]);
-      compute_sync();
+      mbar_arrive(bar[B_PDONE]);
 
-      // ---- epilogue: o = O / den + conv(V); S -> bf16 copy (or to global after the last tile) ----
-      ok = ok && mbar_wait(bar[B_MMA2], par, abort);
+      // ---- [S|z]_n: bf16 copy for the next tile, or the final state to global memory ----
+      ok = ok && mbar_wait(bar[B_MMA_S], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
-        const float den = sm.den_intra[0][r] + sm.den_intra[1][r] + sm.den_inter[0][r] + sm.den_inter[1][r] + eps;
-        const float rden = 1.f / den;
-#pragma unroll
-        for (int qq = 0; qq < 2; ++qq) {
-          uint32_t v[32];
-          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32 * qq, v);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const int cc = 4 * qq + c;                          // chunk inside this half's box
-            const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
-            float acc[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
-            for (int t = 0; t < W; ++t) {
-              const int row = r - t;
-              uint4 u;
-              if (row >= 0) u = *reinterpret_cast<const uint4*>(Vt + hf * BOX_BYTES + swz(row, cc));
-              else u = *reinterpret_cast<const uint4*>(halo + (W - 1 + row) * D + ch0);
-              const float4 w0 = *reinterpret_cast<const float4*>(wsm + t * D + ch0);
-              const float4 w1 = *reinterpret_cast<const float4*>(wsm + t * D + ch0 + 4);
-              acc[0] = fmaf(w0.x, lo_f(u.x), acc[0]); acc[1] = fmaf(w0.y, hi_f(u.x), acc[1]);
-              acc[2] = fmaf(w0.z, lo_f(u.y), acc[2]); acc[3] = fmaf(w0.w, hi_f(u.y), acc[3]);
-              acc[4] = fmaf(w1.x, lo_f(u.z), acc[4]); acc[5] = fmaf(w1.y, hi_f(u.z), acc[5]);
-              acc[6] = fmaf(w1.z, lo_f(u.w), acc[6]); acc[7] = fmaf(w1.w, hi_f(u.w), acc[7]);
-            }
-            *reinterpret_cast<uint4*>(Pb + swz(r, cc)) =
-                make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
-          }
-        }
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           uint32_t v[32];
@@ -502,26 +508,60 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                               __uint_as_float(v[e + 3]));
           } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              uint4 u;
-              u.x = pack2(__uint_as_float(v[8 * c]), __uint_as_float(v[8 * c + 1]));
-              u.y = pack2(__uint_as_float(v[8 * c + 2]), __uint_as_float(v[8 * c + 3]));
-              u.z = pack2(__uint_as_float(v[8 * c + 4]), __uint_as_float(v[8 * c + 5]));
-              u.w = pack2(__uint_as_float(v[8 * c + 6]), __uint_as_float(v[8 * c + 7]));
-              *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = u;
-            }
+            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
           }
+        }
+        if (hf == 0) {
+          const float zz = __uint_as_float(tmem_ld1(tmem + lane_addr + Z_COL));
+          tmem_wait_ld();
+          if (last) z[(size_t)bh * D + r] = zz;
+          else *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(r, 0)) = __float2bfloat16_rn(zz);
         }
       }
       fence_proxy_async();
       tc_fence_before();
-      compute_sync();
-      if (tid == 0 && ok) {
-        tma_store(&mo, 0, n * TILE, bh, sbase + OFF_P);
-        tma_store(&mo, 64, n * TILE, bh, sbase + OFF_P + BOX_BYTES);
-        tma_commit();
+      mbar_arrive(bar[B_SB]);
+    }
+  } else {
+    // =============================== group B: epilogue (256 threads) ===============================
+    const int r = 32 * (warp & 3) + lane;         // tile row = TMEM lane
+    const int hf = warp >> 2;                     // column half
+    const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+    bool ok = true;
+    for (int n = 0; n < nchunks; ++n) {
+      const uint32_t par = n & 1;
+      const int valid = min(TILE, T - n * TILE);
+      const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
+      ok = ok && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort) && mbar_wait(bar[B_MMA_O], par, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        tc_fence_after();
+        const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL + par * 16));
+        tmem_wait_ld();
+        const float rden = 1.f / (den + eps);
+        __nv_bfloat16* og = o + ((size_t)bh * T + (size_t)n * TILE + r) * D;
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          uint32_t v[32];
+          LA_TMEM_LD32(tmem + lane_addr + X_COL + par * 128 + 64 * hf + 32 * qq, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int cc = 4 * qq + c;                          // chunk inside this half's box
+            const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
+            float acc[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
+            conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
+            if (r < valid)
+              *reinterpret_cast<uint4*>(og + ch0) = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]),
+                                                               pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+          }
+        }
       }
-      if (tid < D && ok) {
+      tc_fence_before();
+      sync_group_b();                             // every thread has read the old halo
+      if (ok && tid < D) {
         // halo <- last W-1 rows of (halo ++ valid rows of V); ascending, source index above target
         const unsigned char* Vc = Vt + (tid >> 6) * BOX_BYTES;
         const int cw = tid & 63;
@@ -533,18 +573,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           halo[i * D + tid] = x;
         }
       }
+      sync_group_b();                             // the new halo is visible to the next epilogue
       mbar_arrive(bar[B_EPI]);
     }
-
-    compute_sync();
-    if (ok) {
-      if (tid < D) {
-        z[(size_t)bh * D + tid] = sm.zs[tid];
-        for (int i = 0; i < W - 1; ++i) win[((size_t)bh * (W - 1) + i) * D + tid] = halo[i * D + tid];
-      }
+    if (ok && tid < D) {
+      for (int i = 0; i < W - 1; ++i) win[((size_t)bh * (W - 1) + i) * D + tid] = halo[i * D + tid];
       if (tid == 0 && h == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
-    if (tid == 0) tma_wait_all();
   }
 
   // ---- teardown ----
@@ -554,7 +589,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     if (tid == 0) report(status, LA_ERR_TIMEOUT);
     for (int i = 0; i < 64; ++i) __nanosleep(2000);   // bounded grace period for copies still in flight
   }
-  if (warp == 8) {
+  if (warp == kCtrlWarp) {
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
@@ -594,25 +629,44 @@ static bool make_map(CUtensorMap* m, const void* base, int BH, int T) {
 
 }  // namespace tc
 
+template <int PHI>
+static cudaError_t launch_w(const la_config& c, int BH, int T, const CUtensorMap& mq, const CUtensorMap& mk,
+                            const CUtensorMap& mv, const float* w, int init, const la_state& st, void* o, int* status,
+                            cudaStream_t s) {
+  const size_t smem = tc::smem_bytes(c.conv_taps);
+  void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
+               __nv_bfloat16*, int*, int, int, int, float, int);
+  switch (c.conv_taps) {     // unrolled tap loops for the common small widths
+    case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
+    case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
+    case 3: kern = tc::prefill_tc_kernel<PHI, 3>; break;
+    case 4: kern = tc::prefill_tc_kernel<PHI, 4>; break;
+    case 5: kern = tc::prefill_tc_kernel<PHI, 5>; break;
+    default: kern = tc::prefill_tc_kernel<PHI, 0>; break;
+  }
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<dim3(BH), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, w, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
+                                                  (__nv_bfloat16*)o, status, c.H, T, c.conv_taps, c.eps, init);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
                               int init, const la_state& st, void* o, cudaStream_t s, bool* handled) {
   const la_config& c = ctx->cfg;
   *handled = false;
   if (c.io_dtype != LA_BF16 || c.d != tc::D) return cudaSuccess;
+  if (tc::smem_bytes(c.conv_taps) > 227u * 1024u) return cudaSuccess;   // very long tap windows: CUDA-core kernel
   const int BH = B * c.H;
-  CUtensorMap mq, mk, mv, mo;
-  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
-      !tc::make_map(&mo, o, BH, T))
+  CUtensorMap mq, mk, mv;
+  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T))
     return cudaSuccess;   // no tensor-map support: the CUDA-core kernel takes over
-  const size_t smem = tc::smem_bytes(c.conv_taps);
-  auto kern = c.phi == LA_PHI_ELU1 ? tc::prefill_tc_kernel<LA_PHI_ELU1> : tc::prefill_tc_kernel<LA_PHI_RELU>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  kern<<<dim3(BH), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
-                                                  ctx->d_status, c.H, T, c.conv_taps, c.eps, init);
+  cudaError_t e = c.phi == LA_PHI_ELU1
+                      ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, w, init, st, o, ctx->d_status, s)
+                      : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, w, init, st, o, ctx->d_status, s);
   ctx->launches += 1;
   *handled = true;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace la
