@@ -10,9 +10,9 @@
 //
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
 //   group A  phi applied in place on Q and K (packed bf16x2 arithmetic, fp32 exp)
-//   tcgen05  P = phi(Q) phi(K)^T            -> TMEM buffer (n+1)&1 (idle until tile n+1 needs it)
-//            [O | den] = phi(Q) [S | z]_prev -> TMEM buffer n&1; [S | z]_prev is a bf16 copy in smem
-//            [S | z] += phi(K)^T [V | 1]     -> fp32 in TMEM for the whole chain
+//   tcgen05  P = phi(Q) phi(K)^T
+//            [S | z] += phi(K)^T [V | 1]     (fp32 in TMEM for the whole chain)
+//            [O | den] = phi(Q) [S | z]_prev  ([S | z]_prev is a bf16 copy in shared memory)
 //   group A  P -> causal mask, bf16 -> shared memory;  [S | z] -> bf16 copy for tile n+1
 //   tcgen05  [O | den] += (P o M) [V | 1]
 //   group B  o = O / (den + eps) + conv(V) -> global memory
@@ -36,9 +36,8 @@ constexpr int kCtrlWarp = 16;
 constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns: two 128-column buffers that hold O of tile n (buffer n&1) and P of tile n (buffer (n+1)&1),
-// S, and three 16-column blocks whose first column is den (per O buffer) and z.
-constexpr uint32_t X_COL = 0, S_COL = 256, DEN_COL = 384, Z_COL = 416, TMEM_COLS = 512;
+// TMEM columns: P, O, S (128 each) and two 16-column blocks whose first column is den and z.
+constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, DEN_COL = 384, Z_COL = 400, TMEM_COLS = 512;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait
 
 // shared-memory map (offsets from a 1024-byte aligned base)
@@ -55,14 +54,14 @@ struct Small {
   int pad[2];
 };
 // full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B.
-// MMA_P / MMA_S / MMA_O: tcgen05.commit after P; after [O|den] = phi(Q)[S|z] and [S|z] += phi(K)^T[V|1];
-// after [O|den] += P[V|1].
+// MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T[V|1] (K buffer free);
+// after [O|den] = phi(Q)[S|z] (Q buffer free); after [O|den] += P[V|1].
 enum { B_FULL_QK = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
-       B_SB = 8, B_EPI = 9, kNumBars = 10 };
+       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, kNumBars = 11 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
-__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
+__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -273,7 +272,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const uint32_t sbase = smem_u32(smem);
   Small& sm = *reinterpret_cast<Small*>(smem + OFF_SMALL);
   float* wsm = reinterpret_cast<float*>(smem + off_w());                       // [W][128]
-  __nv_bfloat16* halo = reinterpret_cast<__nv_bfloat16*>(smem + off_halo(W));  // [W-1][128], oldest first
+  // two halo buffers [W-1][128], oldest row first: tile n reads buffer n&1 and writes buffer (n+1)&1
+  __nv_bfloat16* halo0 = reinterpret_cast<__nv_bfloat16*>(smem + off_halo(W));
+  const int halo_elems = (W > 1 ? W - 1 : 1) * D;
   volatile int* abort = &sm.abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -295,6 +296,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     mbar_init(bar[B_PDONE], kThreadsA);
     mbar_init(bar[B_SB], kThreadsA);
     mbar_init(bar[B_EPI], kThreadsB);
+    mbar_init(bar[B_MMA_Q], 1);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -306,7 +308,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   }
   for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
-    halo[idx] = init ? win[(size_t)bh * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
+    halo0[idx] = init ? win[(size_t)bh * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
   for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
     reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
@@ -338,39 +340,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
         const uint32_t vbuf = sbase + OFF_V0 + par * TILE_BYTES;
-        const uint32_t ocol = tmem + X_COL + par * 128, pcol = tmem + X_COL + (par ^ 1) * 128;
-        const uint32_t dcol = tmem + DEN_COL + par * 16;
         const bool has_state = init || n > 0;
         ok = mbar_wait(bar[B_PHI], par, abort);                 // phi(Q), phi(K) of tile n are in place
         if (!ok) break;
-        if (n >= 1) {
-          // group B is done with tile n-1: its TMEM buffer takes P of tile n, its V buffer takes tile n+1
-          ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
-          if (!ok) break;
-          if (n + 1 < nchunks) {
-            const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
-            mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
-            tma_load(vnext, &mv, 0, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-            tma_load(vnext + BOX_BYTES, &mv, 64, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-          }
-        }
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T
-          mma_bf16(pcol, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(sbase + OFF_K, ks), idesc(false, false, 128), ks > 0);
+          mma_bf16(tmem + P_COL, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(sbase + OFF_K, ks),
+                   idesc(false, false, 128), ks > 0);
         mma_commit(bar[B_MMA_P]);
         // the bf16 copy of [S|z] before tile n is complete (and S itself has been read) after n + 1 arrivals
         ok = mbar_wait(bar[B_SB], par, abort) && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after();
-        if (has_state) {
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {   // [O | den] = phi(Q) [S | z]_prev
-            const uint64_t qd = desc_kmajor(sbase + OFF_Q, ks);
-            mma_bf16(ocol, qd, desc_mnmajor(sbase + OFF_S, ks), idesc(false, true, 128), ks > 0);
-            mma_bf16(dcol, qd, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
-          }
-        }
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {     // [S | z] += phi(K)^T [V | 1]
           const uint64_t kd = desc_mnmajor(sbase + OFF_K, ks);
@@ -378,24 +360,49 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_S]);
+        if (n >= 1) {
+          // group B is done with tile n-1: O may be overwritten, and its V buffer takes tile n+1
+          ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
+          if (!ok) break;
+          tc_fence_after();
+          if (n + 1 < nchunks) {
+            const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
+            mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
+            tma_load(vnext, &mv, 0, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+            tma_load(vnext + BOX_BYTES, &mv, 64, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+          }
+        }
+        if (has_state) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {   // [O | den] = phi(Q) [S | z]_prev
+            const uint64_t qd = desc_kmajor(sbase + OFF_Q, ks);
+            mma_bf16(tmem + O_COL, qd, desc_mnmajor(sbase + OFF_S, ks), idesc(false, true, 128), ks > 0);
+            mma_bf16(tmem + DEN_COL, qd, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
+          }
+        }
+        mma_commit(bar[B_MMA_Q]);
+        if (n + 1 < nchunks) {
+          ok = mbar_wait(bar[B_MMA_S], par, abort);             // the K buffer is free
+          if (!ok) break;
+          mbar_expect_tx(bar[B_FULL_QK], 2 * TILE_BYTES);
+          tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
+          tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
+        }
         ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in shared memory
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {     // [O | den] += (P o M) [V | 1]
           const uint64_t pd = desc_kmajor(sbase + OFF_P, ks);
-          mma_bf16(ocol, pd, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
-          mma_bf16(dcol, pd, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
+          mma_bf16(tmem + O_COL, pd, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
+          mma_bf16(tmem + DEN_COL, pd, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_O]);
         if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_S], par, abort);             // Q and K buffers are free
+          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
           if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_QK], 2 * TILE_BYTES);
           tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-          tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-          tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
         }
       }
     }
@@ -441,7 +448,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       const uint32_t par = n & 1;
       const int valid = min(TILE, T - n * TILE);
       const bool last = n + 1 == nchunks;
-      const uint32_t pcol = tmem + X_COL + (par ^ 1) * 128;
+      const uint32_t pcol = tmem + P_COL;
 
       // ---- phi on Q and K in place ----
       ok = ok && mbar_wait(bar[B_FULL_QK], par, abort);
@@ -491,7 +498,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       mbar_arrive(bar[B_PDONE]);
 
       // ---- [S|z]_n: bf16 copy for the next tile, or the final state to global memory ----
-      ok = ok && mbar_wait(bar[B_MMA_S], par, abort);
+      // S_n is final after MMA_S; the old copy may be overwritten once [O|den] = phi(Q)[S|z]_prev has read it
+      ok = ok && mbar_wait(bar[B_MMA_S], par, abort) && mbar_wait(bar[B_MMA_Q], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
@@ -532,18 +540,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       const uint32_t par = n & 1;
       const int valid = min(TILE, T - n * TILE);
       const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
-      ok = ok && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort) && mbar_wait(bar[B_MMA_O], par, abort);
+      const __nv_bfloat16* halo = halo0 + par * halo_elems;         // rows before this tile
+      __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
+      ok = ok && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok && tid < D) {
+        // next halo <- last W-1 rows of (halo ++ valid rows of V)
+        const unsigned char* Vc = Vt + (tid >> 6) * BOX_BYTES;
+        const int cw = tid & 63;
+        for (int i = 0; i < W - 1; ++i) {
+          const int src = valid + i;
+          __nv_bfloat16 x;
+          if (src < W - 1) x = halo[src * D + tid];
+          else x = *reinterpret_cast<const __nv_bfloat16*>(Vc + swz(src - (W - 1), cw >> 3) + (cw & 7) * 2);
+          halo_next[i * D + tid] = x;
+        }
+      }
+      ok = ok && mbar_wait(bar[B_MMA_O], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
-        const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL + par * 16));
+        const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
         tmem_wait_ld();
         const float rden = 1.f / (den + eps);
         __nv_bfloat16* og = o + ((size_t)bh * T + (size_t)n * TILE + r) * D;
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           uint32_t v[32];
-          LA_TMEM_LD32(tmem + lane_addr + X_COL + par * 128 + 64 * hf + 32 * qq, v);
+          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32 * qq, v);
           tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
@@ -553,30 +577,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
             conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
-            if (r < valid)
-              *reinterpret_cast<uint4*>(og + ch0) = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]),
-                                                               pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+            const uint4 out =
+                make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+            if (r < valid) *reinterpret_cast<uint4*>(og + ch0) = out;
           }
         }
       }
       tc_fence_before();
-      sync_group_b();                             // every thread has read the old halo
-      if (ok && tid < D) {
-        // halo <- last W-1 rows of (halo ++ valid rows of V); ascending, source index above target
-        const unsigned char* Vc = Vt + (tid >> 6) * BOX_BYTES;
-        const int cw = tid & 63;
-        for (int i = 0; i < W - 1; ++i) {
-          const int src = valid + i;
-          __nv_bfloat16 x;
-          if (src < W - 1) x = halo[src * D + tid];
-          else x = *reinterpret_cast<const __nv_bfloat16*>(Vc + swz(src - (W - 1), cw >> 3) + (cw & 7) * 2);
-          halo[i * D + tid] = x;
-        }
-      }
-      sync_group_b();                             // the new halo is visible to the next epilogue
-      mbar_arrive(bar[B_EPI]);
+      mbar_arrive(bar[B_EPI]);                    // O, V and the old halo have been read
+      sync_group_b();                             // the next halo is complete before any thread reads it
     }
     if (ok && tid < D) {
+      const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
       for (int i = 0; i < W - 1; ++i) win[((size_t)bh * (W - 1) + i) * D + tid] = halo[i * D + tid];
       if (tid == 0 && h == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
