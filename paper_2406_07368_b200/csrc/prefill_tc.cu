@@ -56,8 +56,8 @@ struct Small {
 // full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B.
 // MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T[V|1] (K buffer free);
 // after [O|den] = phi(Q)[S|z] (Q buffer free); after [O|den] += P[V|1].
-enum { B_FULL_QK = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
-       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, kNumBars = 11 };
+enum { B_FULL_K = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
+       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, kNumBars = 12 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
@@ -286,7 +286,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 
   // ---- set-up ----
   if (tid == 0) {
-    mbar_init(bar[B_FULL_QK], 1);
+    mbar_init(bar[B_FULL_K], 1);
+    mbar_init(bar[B_FULL_Q], 1);
     mbar_init(bar[B_FULL_V0], 1);
     mbar_init(bar[B_FULL_V1], 1);
     mbar_init(bar[B_MMA_P], 1);
@@ -327,11 +328,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     // =============================== TMA + MMA issue (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(bar[B_FULL_QK], 2 * TILE_BYTES);
-      tma_load(sbase + OFF_Q, &mq, 0, 0, bh, bar[B_FULL_QK]);
-      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, 0, bh, bar[B_FULL_QK]);
-      tma_load(sbase + OFF_K, &mk, 0, 0, bh, bar[B_FULL_QK]);
-      tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, 0, bh, bar[B_FULL_QK]);
+      mbar_expect_tx(bar[B_FULL_K], TILE_BYTES);
+      tma_load(sbase + OFF_K, &mk, 0, 0, bh, bar[B_FULL_K]);
+      tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, 0, bh, bar[B_FULL_K]);
+      mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
+      tma_load(sbase + OFF_Q, &mq, 0, 0, bh, bar[B_FULL_Q]);
+      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, 0, bh, bar[B_FULL_Q]);
       for (int n = 0; n < 2 && n < nchunks; ++n) {
         mbar_expect_tx(bar[B_FULL_V0 + n], TILE_BYTES);
         tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, n * TILE, bh, bar[B_FULL_V0 + n]);
@@ -360,6 +362,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_S]);
+        if (n + 1 < nchunks) {
+          ok = mbar_wait(bar[B_MMA_S], par, abort);             // the K buffer is free
+          if (!ok) break;
+          mbar_expect_tx(bar[B_FULL_K], TILE_BYTES);
+          tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_K]);
+          tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_K]);
+        }
         if (n >= 1) {
           // group B is done with tile n-1: O may be overwritten, and its V buffer takes tile n+1
           ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
@@ -382,11 +391,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         }
         mma_commit(bar[B_MMA_Q]);
         if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_S], par, abort);             // the K buffer is free
+          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
           if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_QK], 2 * TILE_BYTES);
-          tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-          tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
+          mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
+          tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_Q]);
+          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_Q]);
         }
         ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in shared memory
         if (!ok) break;
@@ -398,12 +407,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16(tmem + DEN_COL, pd, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_O]);
-        if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
-          if (!ok) break;
-          tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_QK]);
-        }
       }
     }
   } else if (warp >= 8) {
@@ -450,15 +453,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       const bool last = n + 1 == nchunks;
       const uint32_t pcol = tmem + P_COL;
 
-      // ---- phi on Q and K in place ----
-      ok = ok && mbar_wait(bar[B_FULL_QK], par, abort);
+      // ---- phi on K, then on Q, in place (K lands first) ----
+      ok = ok && mbar_wait(bar[B_FULL_K], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
-          uint4* p = reinterpret_cast<uint4*>(Qb + swz(r, cc));
-          *p = phi8<PHI>(*p);
-        }
         const int ct = ta & 15, rg = ta >> 4;                   // chunk column 0..15, row group 0..15
         unsigned char* Kb = smem + OFF_K + (ct >> 3) * BOX_BYTES;
 #pragma unroll
@@ -466,6 +464,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           const int j = rg + 16 * m;
           uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
           *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);   // rows past the end contribute nothing
+        }
+      }
+      ok = ok && mbar_wait(bar[B_FULL_Q], par, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+          uint4* p = reinterpret_cast<uint4*>(Qb + swz(r, cc));
+          *p = phi8<PHI>(*p);
         }
       }
       fence_proxy_async();
