@@ -13,7 +13,8 @@
 //   tcgen05  P = phi(Q) phi(K)^T
 //            [S | z] += phi(K)^T [V | 1]     (fp32 in TMEM for the whole chain)
 //            [O | den] = phi(Q) [S | z]_prev  ([S | z]_prev is a bf16 copy in shared memory)
-//   group A  P -> causal mask, bf16 -> shared memory;  [S | z] -> bf16 copy for tile n+1
+//   group A  P -> causal mask, bf16 -> TMEM (the A operand of the next product);
+//            phi on K of tile n+1 (K is double-buffered);  [S | z] -> bf16 copy for tile n+1
 //   tcgen05  [O | den] += (P o M) [V | 1]
 //   group B  o = O / (den + eps) + conv(V) -> global memory
 //
@@ -36,19 +37,20 @@ constexpr int kCtrlWarp = 16;
 constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns: P, O, S (128 each) and two 16-column blocks whose first column is den and z.
-constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, DEN_COL = 384, Z_COL = 400, TMEM_COLS = 512;
+// TMEM columns: P, O, S (128 each, fp32), two 16-column blocks whose first column is den and z, and the
+// masked P as packed bf16 pairs (64 columns).
+constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, DEN_COL = 384, Z_COL = 400, P16_COL = 416, TMEM_COLS = 512;
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait
 
 // shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
-                   OFF_P = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
+constexpr uint32_t OFF_Q = 0, OFF_K0 = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
+                   OFF_K1 = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
                    OFF_ONES = 6 * TILE_BYTES,      // [128 x 16] bf16, column 0 = 1: the extension of V
                    OFF_SZ = OFF_ONES + 4096,       // [128 x 16] bf16, column 0 = z: the extension of the S copy
                    OFF_SMALL = OFF_SZ + 4096;
 
 struct Small {
-  unsigned long long bars[12];
+  unsigned long long bars[16];
   uint32_t tmem_base;
   int abort;
   int pad[2];
@@ -56,8 +58,8 @@ struct Small {
 // full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B.
 // MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T[V|1] (K buffer free);
 // after [O|den] = phi(Q)[S|z] (Q buffer free); after [O|den] += P[V|1].
-enum { B_FULL_K = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
-       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, kNumBars = 12 };
+enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
+       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, B_FULL_K1 = 12, kNumBars = 13 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
@@ -135,6 +137,15 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint6
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)acc)
       : "memory");
 }
+// The same with the A operand read from TMEM (rows in lanes, two bf16 per 32-bit column).
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)acc)
+      : "memory");
+}
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -170,6 +181,14 @@ __device__ __forceinline__ uint32_t tmem_ld1(uint32_t taddr) {
 __device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t v) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(v) : "memory");
 }
+#define LA_TMEM_ST16(taddr, r)                                                                                   \
+  asm volatile(                                                                                                  \
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "                                                            \
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"                                 \
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),      \
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])             \
+      : "memory")
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -286,7 +305,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 
   // ---- set-up ----
   if (tid == 0) {
-    mbar_init(bar[B_FULL_K], 1);
+    mbar_init(bar[B_FULL_K0], 1);
+    mbar_init(bar[B_FULL_K1], 1);
     mbar_init(bar[B_FULL_Q], 1);
     mbar_init(bar[B_FULL_V0], 1);
     mbar_init(bar[B_FULL_V1], 1);
@@ -328,9 +348,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     // =============================== TMA + MMA issue (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(bar[B_FULL_K], TILE_BYTES);
-      tma_load(sbase + OFF_K, &mk, 0, 0, bh, bar[B_FULL_K]);
-      tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, 0, bh, bar[B_FULL_K]);
+      mbar_expect_tx(bar[B_FULL_K0], TILE_BYTES);
+      tma_load(sbase + OFF_K0, &mk, 0, 0, bh, bar[B_FULL_K0]);
+      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, 0, bh, bar[B_FULL_K0]);
+      if (nchunks > 1) {
+        mbar_expect_tx(bar[B_FULL_K1], TILE_BYTES);
+        tma_load(sbase + OFF_K1, &mk, 0, TILE, bh, bar[B_FULL_K1]);
+        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, TILE, bh, bar[B_FULL_K1]);
+      }
       mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
       tma_load(sbase + OFF_Q, &mq, 0, 0, bh, bar[B_FULL_Q]);
       tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, 0, bh, bar[B_FULL_Q]);
@@ -342,13 +367,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
         const uint32_t vbuf = sbase + OFF_V0 + par * TILE_BYTES;
+        const uint32_t kbuf = sbase + (par ? OFF_K1 : OFF_K0);
+        const uint32_t kbar = bar[par ? B_FULL_K1 : B_FULL_K0];
         const bool has_state = init || n > 0;
         ok = mbar_wait(bar[B_PHI], par, abort);                 // phi(Q), phi(K) of tile n are in place
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T
-          mma_bf16(tmem + P_COL, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(sbase + OFF_K, ks),
+          mma_bf16(tmem + P_COL, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(kbuf, ks),
                    idesc(false, false, 128), ks > 0);
         mma_commit(bar[B_MMA_P]);
         // the bf16 copy of [S|z] before tile n is complete (and S itself has been read) after n + 1 arrivals
@@ -357,17 +384,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {     // [S | z] += phi(K)^T [V | 1]
-          const uint64_t kd = desc_mnmajor(sbase + OFF_K, ks);
+          const uint64_t kd = desc_mnmajor(kbuf, ks);
           mma_bf16(tmem + S_COL, kd, desc_mnmajor(vbuf, ks), idesc(true, true, 128), has_state || ks > 0);
           mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_S]);
-        if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_S], par, abort);             // the K buffer is free
+        if (n + 2 < nchunks) {
+          ok = mbar_wait(bar[B_MMA_S], par, abort);             // this K buffer is free: it takes tile n+2
           if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_K], TILE_BYTES);
-          tma_load(sbase + OFF_K, &mk, 0, (n + 1) * TILE, bh, bar[B_FULL_K]);
-          tma_load(sbase + OFF_K + BOX_BYTES, &mk, 64, (n + 1) * TILE, bh, bar[B_FULL_K]);
+          mbar_expect_tx(kbar, TILE_BYTES);
+          tma_load(kbuf, &mk, 0, (n + 2) * TILE, bh, kbar);
+          tma_load(kbuf + BOX_BYTES, &mk, 64, (n + 2) * TILE, bh, kbar);
         }
         if (n >= 1) {
           // group B is done with tile n-1: O may be overwritten, and its V buffer takes tile n+1
@@ -397,14 +424,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_Q]);
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_Q]);
         }
-        ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in shared memory
+        ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in TMEM
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {     // [O | den] += (P o M) [V | 1]
-          const uint64_t pd = desc_kmajor(sbase + OFF_P, ks);
-          mma_bf16(tmem + O_COL, pd, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
-          mma_bf16(tmem + DEN_COL, pd, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
+          const uint32_t pa = tmem + P16_COL + 8 * ks;       // 16 values of every row = 8 columns
+          mma_bf16_ts(tmem + O_COL, pa, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
+          mma_bf16_ts(tmem + DEN_COL, pa, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_O]);
       }
@@ -417,7 +444,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     const int hf = wa >> 2;                       // column half
     const uint32_t lane_addr = (uint32_t)(32 * (wa & 3)) << 16;
     unsigned char* Qb = smem + OFF_Q + hf * BOX_BYTES;
-    unsigned char* Pb = smem + OFF_P + hf * BOX_BYTES;
     unsigned char* Sb = smem + OFF_S + hf * BOX_BYTES;
     float* Sg = S + (size_t)bh * D * D + (size_t)r * D + 64 * hf;
     bool ok = true;
@@ -447,25 +473,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     tc_fence_before();
     mbar_arrive(bar[B_SB]);                       // phase 0: the state before tile 0 is in place
 
+    // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero
+    auto phi_k = [&](int m) {
+      const int valid = min(TILE, T - m * TILE);
+      const int ct = ta & 15, rg = ta >> 4;                     // chunk column 0..15, row group 0..15
+      unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * BOX_BYTES;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int j = rg + 16 * i;
+        uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
+        *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    };
+    ok = mbar_wait(bar[B_FULL_K0], 0, abort);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) phi_k(0);
+
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
-      const int valid = min(TILE, T - n * TILE);
       const bool last = n + 1 == nchunks;
-      const uint32_t pcol = tmem + P_COL;
 
-      // ---- phi on K, then on Q, in place (K lands first) ----
-      ok = ok && mbar_wait(bar[B_FULL_K], par, abort);
-      ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
-        const int ct = ta & 15, rg = ta >> 4;                   // chunk column 0..15, row group 0..15
-        unsigned char* Kb = smem + OFF_K + (ct >> 3) * BOX_BYTES;
-#pragma unroll
-        for (int m = 0; m < 8; ++m) {
-          const int j = rg + 16 * m;
-          uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-          *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);   // rows past the end contribute nothing
-        }
-      }
+      // ---- phi on Q in place (phi on K of this tile was done one iteration earlier) ----
       ok = ok && mbar_wait(bar[B_FULL_Q], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
@@ -478,7 +506,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       fence_proxy_async();
       mbar_arrive(bar[B_PHI]);
 
-      // ---- P: causal mask, bf16 -> shared memory ----
+      // ---- P: causal mask, packed bf16 -> TMEM ----
       ok = ok && mbar_wait(bar[B_MMA_P], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
@@ -486,23 +514,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           const int col0 = 64 * hf + 32 * qq;
-          uint32_t v[32];
+          uint32_t v[32], pk[16];
           if (col0 <= 32 * (wa & 3) + 31) {                     // warp-uniform: some row of this warp reaches col0
-            LA_TMEM_LD32(pcol + lane_addr + col0, v);
+            LA_TMEM_LD32(tmem + P_COL + lane_addr + col0, v);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = col0 + e <= r ? v[e] : 0u;
+            for (int e = 0; e < 16; ++e)
+              pk[e] = pack2(col0 + 2 * e <= r ? __uint_as_float(v[2 * e]) : 0.f,
+                            col0 + 2 * e + 1 <= r ? __uint_as_float(v[2 * e + 1]) : 0.f);
           } else {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = 0u;
+            for (int e = 0; e < 16; ++e) pk[e] = 0u;
           }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Pb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
+          LA_TMEM_ST16(tmem + P16_COL + lane_addr + (col0 >> 1), pk);
         }
+        tmem_wait_st();
       }
-      fence_proxy_async();
       tc_fence_before();
       mbar_arrive(bar[B_PDONE]);
+
+      // ---- phi on K of the next tile while the tensor cores work on this one ----
+      if (!last) {
+        ok = ok && mbar_wait(bar[((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0], ((n + 1) >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) phi_k(n + 1);
+      }
 
       // ---- [S|z]_n: bf16 copy for the next tile, or the final state to global memory ----
       // S_n is final after MMA_S; the old copy may be overwritten once [O|den] = phi(Q)[S|z]_prev has read it
