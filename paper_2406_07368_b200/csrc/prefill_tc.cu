@@ -230,15 +230,16 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 __device__ __forceinline__ float lo_f(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float hi_f(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-// phi on two packed bf16 values.  elu+1: x + 1 where x > 0 (one correctly rounded bf16 addition), exp(x)
-// elsewhere (fp32 exp2, rounded once to bf16); the two are merged with a lane mask.  ReLU: packed max.
+// phi on two packed bf16 values, entirely in packed arithmetic.  elu+1: x + 1 where x > 0 (one correctly
+// rounded bf16 addition), 2^(x log2 e) elsewhere; the two are merged with a lane mask.  The exponent argument is
+// formed by one fused multiply (x * log2e_hi + x * log2e_lo would not help: the product is rounded to bf16
+// either way), so exp(x) carries a relative error of about |x| 2^-9 on top of the bf16 rounding of the result --
+// below one bf16 ulp for |x| < 1, and in absolute terms largest where exp(x) is close to 1.  ReLU: packed max.
 template <int PHI> __device__ __forceinline__ uint32_t phi2(uint32_t u) {
   if (PHI == LA_PHI_ELU1) {
-    float e0, e1;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(lo_f(u) * 1.4426950408889634f));
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(hi_f(u) * 1.4426950408889634f));
-    const uint32_t e = pack2(e0, e1);
-    uint32_t xp1, mask;
+    uint32_t y, e, xp1, mask;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(y) : "r"(u), "r"(0x3fb93fb9u));        // log2(e) = 1.4453 in bf16
+    asm("ex2.approx.ftz.bf16x2 %0, %1;" : "=r"(e) : "r"(y));
     asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(xp1) : "r"(u), "r"(0x3f803f80u));
     asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(mask) : "r"(u), "r"(0u));
     return (xp1 & mask) | (e & ~mask);
