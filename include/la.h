@@ -193,8 +193,9 @@ la_status la_last_device_status(la_ctx* ctx, void* stream);
 /* Resets the device status word to LA_OK (asynchronous on `stream`). */
 la_status la_clear_device_status(la_ctx* ctx, void* stream);
 
-/* Selects the prefill kernel: 0 = automatic (tensor-core kernel where it applies),
- * 1 = always the fp32 CUDA-core kernel.  For testing one kernel against the other. */
+/* Selects the kernels of la_prefill and la_verify_tree: 0 = automatic (tensor-core kernels where
+ * they apply: bf16 io, d = 128), 1 = always the fp32 CUDA-core kernels.  For testing one kernel
+ * against the other. */
 la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which);
 
 /* Number of kernels the library has launched through this context since creation. */

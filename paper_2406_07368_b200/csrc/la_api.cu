@@ -126,10 +126,13 @@ la_status la_verify_tree(la_ctx* ctx, int32_t B, int32_t N, const void* q, const
   if (!state_ok(ctx, st)) return LA_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   if (!g.ok) return LA_ERR_CUDA;
-  return la::launch_verify(ctx, B, N, q, k, v, parent, conv_w, *st, o, static_cast<cudaStream_t>(stream)) ==
-                 cudaSuccess
-             ? LA_OK
-             : LA_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->prefill_kernel == 0) {
+    bool handled = false;
+    if (la::launch_verify_tc(ctx, B, N, q, k, v, parent, conv_w, *st, o, s, &handled) != cudaSuccess) return LA_ERR_CUDA;
+    if (handled) return LA_OK;
+  }
+  return la::launch_verify(ctx, B, N, q, k, v, parent, conv_w, *st, o, s) == cudaSuccess ? LA_OK : LA_ERR_CUDA;
 }
 
 la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void* v, const int32_t* parent,

@@ -73,4 +73,8 @@ cudaError_t launch_commit(la_ctx* ctx, int B, int N, const void* k, const void* 
 cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v,
                               const float* w, int init_state, const la_state& st, void* o, cudaStream_t s,
                               bool* handled);
+// Tensor-core tree verification (bf16, d = 128).  Sets *handled to false when the shape is not covered.
+cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
+                             const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s,
+                             bool* handled);
 }  // namespace la

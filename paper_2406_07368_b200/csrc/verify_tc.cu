@@ -1,0 +1,353 @@
+// Draft-tree verification on the tensor cores (bf16 io, d = 128, N <= 64).
+//
+// Sec. 4.2 / Sec. 5.3: all N draft nodes of a sequence share the committed state.  The shared part
+// of every node's numerator, phi(Q_tree) S, is one dense product; it is computed transposed,
+//     O^T[c][n] = sum_a S[a][c] phi(q_n)[a],
+// so that the fp32 state is the M x K operand exactly as it lies in memory: TMA brings the 128 x 128
+// fp32 tile of S into shared memory (128-byte swizzle in 32-byte chunks) and tcgen05.mma consumes it as tf32 -- S is read
+// from HBM once, without any conversion pass, while the CUDA cores prepare the tree.  The accumulator
+// (128 channels x 64 nodes, fp32) lives in TMEM; each thread then owns one channel, adds the
+// contributions of the node's ancestors and itself (tree mask), the unfolded convolution along the
+// ancestor chain, and divides by the node's denominator.  Nothing of the state is written.
+#include <cuda.h>
+
+#include "la_common.cuh"
+
+namespace la {
+namespace vtc {
+
+constexpr int D = 128, NMAX = LA_MAX_NODES, kThreads = 256;
+constexpr uint32_t S_BOX = 128 * 128;              // 128 rows x 32 fp32
+constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 32 fp32
+constexpr uint32_t OFF_S = 0, OFF_Q = 4 * S_BOX, OFF_SMALL = OFF_Q + 4 * Q_BOX;   // 64 KiB + 32 KiB
+constexpr uint32_t TMEM_COLS = 64;
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+
+struct Small {
+  float fk[NMAX][D + 4];
+  float v[NMAX][D];
+  float A[NMAX][NMAX + 1];
+  float w[LA_MAX_TAPS][D];
+  float win[LA_MAX_TAPS - 1][D];
+  float z[D];
+  float den[NMAX];
+  unsigned long long mask[NMAX];
+  unsigned long long bars[2];
+  int par[NMAX];
+  int depth[NMAX];
+  uint32_t tmem_base;
+  int bad;
+  int abort;
+};
+constexpr uint32_t kSmemBytes = OFF_SMALL + (uint32_t)sizeof(Small) + 1024;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: false after one second (the CTA's abort flag is raised) or when another thread gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int it = 0; it < 64; ++it)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort = 1;
+      return false;
+    }
+  }
+}
+// 128-byte swizzle: byte offset of 16-byte chunk `cc` of row `row` inside a box with 128-byte rows.
+__device__ __forceinline__ uint32_t swz(int row, int cc) { return (uint32_t)row * 128u + (uint32_t)((cc ^ (row & 7)) << 4); }
+// Shared-memory matrix descriptor; layout 2 = 128-byte swizzle in 16-byte chunks, 1 = 128-byte swizzle in 32-byte
+// chunks (the only layout the hardware takes for a 32-bit operand whose M or N index is the contiguous one).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
+}
+// Instruction descriptor: fp32 accumulate, tf32 x tf32, A with M contiguous (as S lies in memory), B with K
+// contiguous, M = 128, N = 64.
+constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+template <int PHI> __device__ __forceinline__ float phi_f(float x) {
+  if (PHI == LA_PHI_ELU1) return x > 0.f ? x + 1.f : __expf(x);
+  return fmaxf(x, 0.f);
+}
+
+template <int PHI>
+__global__ void __launch_bounds__(kThreads, 1)
+verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __restrict__ q,
+                 const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                 const int32_t* __restrict__ parent, const float* __restrict__ w, const float* __restrict__ z,
+                 const __nv_bfloat16* __restrict__ win, __nv_bfloat16* __restrict__ o, int* status, int H, int N, int W,
+                 float eps) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  Small& sm = *reinterpret_cast<Small*>(smem + OFF_SMALL);
+  volatile int* abort = &sm.abort;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int bh = blockIdx.x, b = bh / H, h = bh % H;
+  const uint32_t bar_s = smem_u32(&sm.bars[0]), bar_mma = smem_u32(&sm.bars[1]);
+
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_mma) : "memory");
+    sm.bad = 0;
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // the committed state of this (sequence, head): four boxes of 32 columns
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_s), "r"(4 * S_BOX) : "memory");
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+      asm volatile(
+          "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+          ::"r"(sbase + OFF_S + x * S_BOX), "l"(&ms), "r"(32 * x), "r"(bh * D), "r"(bar_s)
+          : "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm.tmem_base)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // ---- tree preparation: ancestor-or-self masks and depths (integer work) ----
+  if (tid < N) sm.par[tid] = parent[(size_t)b * N + tid];
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem = sm.tmem_base;
+  if (tid < N) {
+    unsigned long long mask = 0ull;
+    int dep = 0, m = tid;
+    bool ok = true;
+    while (m >= 0) {                     // m strictly decreases: at most N iterations
+      mask |= 1ull << m;
+      ++dep;
+      const int p = sm.par[m];
+      if (p < -1 || p >= m) { ok = false; break; }
+      m = p;
+    }
+    sm.mask[tid] = mask;
+    sm.depth[tid] = dep;
+    if (!ok) sm.bad = 1;
+  }
+
+  // ---- stage phi(q) (fp32, swizzled: the B operand), phi(k), v, z, the window and the taps ----
+  const size_t base = (size_t)bh * N * D;
+  for (int idx = tid; idx < NMAX * (D / 4); idx += kThreads) {
+    const int n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
+    float4 fq = make_float4(0.f, 0.f, 0.f, 0.f), fk = fq, vv = fq;
+    if (n < N) {
+      const uint2 uq = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
+      const uint2 uk = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
+      const uint2 uv = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
+      fq = make_float4(phi_f<PHI>(__uint_as_float(uq.x << 16)), phi_f<PHI>(__uint_as_float(uq.x & 0xffff0000u)),
+                       phi_f<PHI>(__uint_as_float(uq.y << 16)), phi_f<PHI>(__uint_as_float(uq.y & 0xffff0000u)));
+      fk = make_float4(phi_f<PHI>(__uint_as_float(uk.x << 16)), phi_f<PHI>(__uint_as_float(uk.x & 0xffff0000u)),
+                       phi_f<PHI>(__uint_as_float(uk.y << 16)), phi_f<PHI>(__uint_as_float(uk.y & 0xffff0000u)));
+      vv = make_float4(__uint_as_float(uv.x << 16), __uint_as_float(uv.x & 0xffff0000u), __uint_as_float(uv.y << 16),
+                       __uint_as_float(uv.y & 0xffff0000u));
+    }
+    *reinterpret_cast<float4*>(smem + OFF_Q + (a4 >> 5) * Q_BOX + swz(n, (a4 & 31) >> 2)) = fq;
+    *reinterpret_cast<float4*>(&sm.fk[n][a4]) = fk;
+    *reinterpret_cast<float4*>(&sm.v[n][a4]) = vv;
+  }
+  for (int idx = tid; idx < W * D; idx += kThreads) sm.w[idx / D][idx % D] = w[((size_t)h * D + idx % D) * W + idx / D];
+  for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
+    sm.win[idx / D][idx % D] = __bfloat162float(win[(size_t)bh * (W - 1) * D + idx]);
+  if (tid < D) sm.z[tid] = z[(size_t)bh * D + tid];
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  const bool bad = sm.bad != 0;
+
+  // ---- the dense part on the tensor cores: O^T = S^T phi(Q)^T ----
+  if (tid == 0) {
+    if (mbar_wait(bar_s, 0, abort) && !bad) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+      for (int ks = 0; ks < 16; ++ks) {    // 8 values of the contraction index a per step
+        // S: 8 rows of a per step = two groups of 4 rows (512 B apart); the four 32-column boxes are S_BOX apart
+        const uint64_t adesc = smem_desc(sbase + OFF_S + ks * 1024u, S_BOX, 512u, 1u);
+        const uint64_t bdesc = smem_desc(sbase + OFF_Q + (ks >> 2) * Q_BOX + (ks & 3) * 32u, 16u, 1024u, 2u);
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"((uint32_t)(ks > 0))
+            : "memory");
+      }
+    }
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_mma) : "memory");
+  }
+
+  // ---- meanwhile: scores inside the tree where the mask allows, and the denominators ----
+  if (!bad) {
+    for (int idx = tid; idx < N * N; idx += kThreads) {
+      const int n = idx / N, m = idx % N;
+      if ((sm.mask[n] >> m) & 1ull) {
+        float acc = 0.f;
+#pragma unroll 8
+        for (int e = 0; e < D; e += 4) {
+          const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
+          const float4 y = *reinterpret_cast<const float4*>(&sm.fk[m][e]);
+          acc = fmaf(x.x, y.x, acc);
+          acc = fmaf(x.y, y.y, acc);
+          acc = fmaf(x.z, y.z, acc);
+          acc = fmaf(x.w, y.w, acc);
+        }
+        sm.A[n][m] = acc;
+      }
+    }
+  }
+  __syncthreads();
+  if (!bad && tid < N) {
+    float den = 0.f;
+    for (int e = 0; e < D; e += 4) {
+      const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(tid, (e & 31) >> 2));
+      den = fmaf(x.x, sm.z[e], den);
+      den = fmaf(x.y, sm.z[e + 1], den);
+      den = fmaf(x.z, sm.z[e + 2], den);
+      den = fmaf(x.w, sm.z[e + 3], den);
+    }
+    unsigned long long mk = sm.mask[tid];
+    while (mk) {
+      const int m = __ffsll((long long)mk) - 1;
+      mk &= mk - 1;
+      den += sm.A[tid][m];
+    }
+    sm.den[tid] = den;
+  }
+  __syncthreads();
+
+  // ---- epilogue: thread = channel c, 32 nodes per thread ----
+  bool ok = mbar_wait(bar_mma, 0, abort);
+  ok = __all_sync(0xffffffffu, ok);
+  if (ok && !bad) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int c = 32 * (warp & 3) + lane, n0 = 32 * (warp >> 2);
+    uint32_t acc[32];
+    if (n0 < N) {                         // warp-uniform
+      const uint32_t taddr = tmem + ((uint32_t)(32 * (warp & 3)) << 16) + n0;
+      asm volatile(
+          "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+          "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+          "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+          : "=r"(acc[0]), "=r"(acc[1]), "=r"(acc[2]), "=r"(acc[3]), "=r"(acc[4]), "=r"(acc[5]), "=r"(acc[6]),
+            "=r"(acc[7]), "=r"(acc[8]), "=r"(acc[9]), "=r"(acc[10]), "=r"(acc[11]), "=r"(acc[12]), "=r"(acc[13]),
+            "=r"(acc[14]), "=r"(acc[15]), "=r"(acc[16]), "=r"(acc[17]), "=r"(acc[18]), "=r"(acc[19]), "=r"(acc[20]),
+            "=r"(acc[21]), "=r"(acc[22]), "=r"(acc[23]), "=r"(acc[24]), "=r"(acc[25]), "=r"(acc[26]), "=r"(acc[27]),
+            "=r"(acc[28]), "=r"(acc[29]), "=r"(acc[30]), "=r"(acc[31])
+          : "r"(taddr)
+          : "memory");
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int n = n0 + i;
+        if (n < N) {
+          float num = __uint_as_float(acc[i]);
+          unsigned long long mk = sm.mask[n];
+          while (mk) {
+            const int m = __ffsll((long long)mk) - 1;
+            mk &= mk - 1;
+            num = fmaf(sm.A[n][m], sm.v[m][c], num);
+          }
+          float conv = 0.f;
+          int cur = n;
+          const int dep = sm.depth[n];
+          for (int tap = 0; tap < W; ++tap) {
+            float u;
+            if (cur >= 0) {
+              u = sm.v[cur][c];
+              cur = sm.par[cur];
+            } else {
+              u = sm.win[(W - 2) - (tap - dep)][c];     // v_{-(tap-dep+1)} of the committed prefix
+            }
+            conv = fmaf(sm.w[tap][c], u, conv);
+          }
+          o[base + (size_t)n * D + c] = __float2bfloat16_rn(num / (sm.den[n] + eps) + conv);
+        }
+      }
+    }
+  }
+
+  // ---- teardown ----
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (tid == 0) {
+    if (bad) report(status, LA_ERR_BAD_TREE);
+    if (sm.abort) report(status, LA_ERR_TIMEOUT);
+  }
+  if (sm.abort)
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);   // bounded grace period for a copy still in flight
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+        qr != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+}  // namespace vtc
+
+cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
+                             const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s,
+                             bool* handled) {
+  const la_config& c = ctx->cfg;
+  *handled = false;
+  if (c.io_dtype != LA_BF16 || c.d != vtc::D) return cudaSuccess;
+  vtc::EncodeTiledFn fn = vtc::encode_fn();
+  if (!fn) return cudaSuccess;
+  const int BH = B * c.H;
+  CUtensorMap ms;   // S viewed as [BH * 128 rows, 128 columns] fp32; boxes of 32 columns x 128 rows
+  cuuint64_t dims[2] = {(cuuint64_t)vtc::D, (cuuint64_t)BH * vtc::D};
+  cuuint64_t strides[1] = {(cuuint64_t)vtc::D * 4};
+  cuuint32_t box[2] = {32, 128}, es[2] = {1, 1};
+  if (fn(&ms, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, st.S, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+         CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+      CUDA_SUCCESS)
+    return cudaSuccess;
+  auto kern = c.phi == LA_PHI_ELU1 ? vtc::verify_tc_kernel<LA_PHI_ELU1> : vtc::verify_tc_kernel<LA_PHI_RELU>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vtc::kSmemBytes);
+  if (e != cudaSuccess) return e;
+  kern<<<dim3(BH), dim3(vtc::kThreads), vtc::kSmemBytes, s>>>(
+      ms, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, parent, w, st.z,
+      (const __nv_bfloat16*)st.win, (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps);
+  ctx->launches += 1;
+  *handled = true;
+  return cudaGetLastError();
+}
+
+}  // namespace la

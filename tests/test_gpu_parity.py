@@ -152,10 +152,12 @@ def tree_case(io, B, H, d, N, W, seed, phi="elu1", eps=0.0, chain=False):
     ("f32", 64, 4, 3, "elu1", 0.0, True), ("bf16", 64, 64, 3, "elu1", 0.0, False),
     ("bf16", 128, 1, 3, "elu1", 0.0, False), ("f32", 128, 64, 9, "elu1", 0.0, False),
     ("bf16", 128, 20, 32, "elu1", 0.0, True), ("bf16", 128, 16, 1, "elu1", 0.0, False)])
-def test_verify_matches_oracle_and_leaves_state_untouched(io, d, N, W, phi, eps, chain):
+@pytest.mark.parametrize("kernel", [0, 1])
+def test_verify_matches_oracle_and_leaves_state_untouched(kernel, io, d, N, W, phi, eps, chain):
     B, H = 3, 2
     ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=41 + N, phi=phi, eps=eps, chain=chain)
     ctx = binding.Context(H, d, W, phi, eps, io, max_nodes=64, max_depth=64)
+    ctx.la_set_prefill_kernel(kernel)
     st = oracle_state_to_dev(ost, io)
     before = st.clone()
     o = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
