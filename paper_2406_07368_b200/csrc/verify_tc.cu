@@ -26,16 +26,20 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 struct Small {
   float fk[NMAX][D + 4];
   float v[NMAX][D];
-  float A[NMAX][NMAX + 1];
+  float A[NMAX][NMAX + 1];            // A[n][j] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself
   float w[LA_MAX_TAPS][D];
   float win[LA_MAX_TAPS - 1][D];
   float z[D];
   float den[NMAX];
-  unsigned long long mask[NMAX];
   unsigned long long bars[2];
   int par[NMAX];
   int depth[NMAX];
+  int pair_off[NMAX + 1];             // prefix sums of depth: node n owns pairs [pair_off[n], pair_off[n + 1])
+  unsigned char anc[NMAX][NMAX];      // anc[n][j] = ancestor of n at distance j (j < depth[n])
+  unsigned char pair_n[NMAX * (NMAX + 1) / 2];
+  unsigned char pair_j[NMAX * (NMAX + 1) / 2];
   uint32_t tmem_base;
+  int max_depth;
   int bad;
   int abort;
 };
@@ -129,47 +133,73 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
-  // ---- tree preparation: ancestor-or-self masks and depths (integer work) ----
+  // ---- tree preparation: ancestor chains and depths (integer work) ----
   if (tid < N) sm.par[tid] = parent[(size_t)b * N + tid];
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = sm.tmem_base;
   if (tid < N) {
-    unsigned long long mask = 0ull;
     int dep = 0, m = tid;
     bool ok = true;
     while (m >= 0) {                     // m strictly decreases: at most N iterations
-      mask |= 1ull << m;
-      ++dep;
+      sm.anc[tid][dep++] = (unsigned char)m;
       const int p = sm.par[m];
       if (p < -1 || p >= m) { ok = false; break; }
       m = p;
     }
-    sm.mask[tid] = mask;
     sm.depth[tid] = dep;
     if (!ok) sm.bad = 1;
   }
+  __syncthreads();
+  if (tid == 0) {                        // pair offsets and the deepest chain (a few dozen integer steps)
+    int off = 0, md = 0;
+    for (int n = 0; n < N; ++n) {
+      sm.pair_off[n] = off;
+      off += sm.depth[n];
+      md = max(md, sm.depth[n]);
+    }
+    sm.pair_off[N] = off;
+    sm.max_depth = md;
+  }
+  __syncthreads();
+  if (tid < N)
+    for (int j = 0, o0 = sm.pair_off[tid]; j < sm.depth[tid]; ++j) {
+      sm.pair_n[o0 + j] = (unsigned char)tid;
+      sm.pair_j[o0 + j] = (unsigned char)j;
+    }
 
   // ---- stage phi(q) (fp32, swizzled: the B operand), phi(k), v, z, the window and the taps ----
   const size_t base = (size_t)bh * N * D;
-  for (int idx = tid; idx < NMAX * (D / 4); idx += kThreads) {
-    const int n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
-    float4 fq = make_float4(0.f, 0.f, 0.f, 0.f), fk = fq, vv = fq;
-    if (n < N) {
-      const uint2 uq = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
-      const uint2 uk = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
-      const uint2 uv = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
-      fq = make_float4(phi_f<PHI>(__uint_as_float(uq.x << 16)), phi_f<PHI>(__uint_as_float(uq.x & 0xffff0000u)),
-                       phi_f<PHI>(__uint_as_float(uq.y << 16)), phi_f<PHI>(__uint_as_float(uq.y & 0xffff0000u)));
-      fk = make_float4(phi_f<PHI>(__uint_as_float(uk.x << 16)), phi_f<PHI>(__uint_as_float(uk.x & 0xffff0000u)),
-                       phi_f<PHI>(__uint_as_float(uk.y << 16)), phi_f<PHI>(__uint_as_float(uk.y & 0xffff0000u)));
-      vv = make_float4(__uint_as_float(uv.x << 16), __uint_as_float(uv.x & 0xffff0000u), __uint_as_float(uv.y << 16),
-                       __uint_as_float(uv.y & 0xffff0000u));
+  {
+    constexpr int ITERS = NMAX * (D / 4) / kThreads;       // 8 chunks of 4 values per thread
+    uint2 uq[ITERS], uk[ITERS], uv[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {                   // all loads in flight before the first use
+      const int idx = tid + it * kThreads, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
+      uq[it] = uk[it] = uv[it] = make_uint2(0u, 0u);
+      if (n < N) {
+        uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
+        uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
+        uv[it] = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
+      }
     }
-    *reinterpret_cast<float4*>(smem + OFF_Q + (a4 >> 5) * Q_BOX + swz(n, (a4 & 31) >> 2)) = fq;
-    *reinterpret_cast<float4*>(&sm.fk[n][a4]) = fk;
-    *reinterpret_cast<float4*>(&sm.v[n][a4]) = vv;
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+      const int idx = tid + it * kThreads, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
+      float4 fq = make_float4(0.f, 0.f, 0.f, 0.f), fk = fq;
+      if (n < N) {                                         // rows past N stay zero (phi(0) may be 1)
+        fq = make_float4(phi_f<PHI>(__uint_as_float(uq[it].x << 16)), phi_f<PHI>(__uint_as_float(uq[it].x & 0xffff0000u)),
+                         phi_f<PHI>(__uint_as_float(uq[it].y << 16)), phi_f<PHI>(__uint_as_float(uq[it].y & 0xffff0000u)));
+        fk = make_float4(phi_f<PHI>(__uint_as_float(uk[it].x << 16)), phi_f<PHI>(__uint_as_float(uk[it].x & 0xffff0000u)),
+                         phi_f<PHI>(__uint_as_float(uk[it].y << 16)), phi_f<PHI>(__uint_as_float(uk[it].y & 0xffff0000u)));
+      }
+      const float4 vv = make_float4(__uint_as_float(uv[it].x << 16), __uint_as_float(uv[it].x & 0xffff0000u),
+                                    __uint_as_float(uv[it].y << 16), __uint_as_float(uv[it].y & 0xffff0000u));
+      *reinterpret_cast<float4*>(smem + OFF_Q + (a4 >> 5) * Q_BOX + swz(n, (a4 & 31) >> 2)) = fq;
+      *reinterpret_cast<float4*>(&sm.fk[n][a4]) = fk;
+      *reinterpret_cast<float4*>(&sm.v[n][a4]) = vv;
+    }
   }
   for (int idx = tid; idx < W * D; idx += kThreads) sm.w[idx / D][idx % D] = w[((size_t)h * D + idx % D) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
@@ -199,42 +229,42 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_mma) : "memory");
   }
 
-  // ---- meanwhile: scores inside the tree where the mask allows, and the denominators ----
+  // ---- meanwhile: scores of every (node, ancestor) pair, one pair per thread, and the denominators ----
   if (!bad) {
-    for (int idx = tid; idx < N * N; idx += kThreads) {
-      const int n = idx / N, m = idx % N;
-      if ((sm.mask[n] >> m) & 1ull) {
-        float acc = 0.f;
+    const int npairs = sm.pair_off[N];
+    for (int pi = tid; pi < npairs; pi += kThreads) {
+      const int n = sm.pair_n[pi], j = sm.pair_j[pi], m = sm.anc[n][j];
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 8
-        for (int e = 0; e < D; e += 4) {
-          const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
-          const float4 y = *reinterpret_cast<const float4*>(&sm.fk[m][e]);
-          acc = fmaf(x.x, y.x, acc);
-          acc = fmaf(x.y, y.y, acc);
-          acc = fmaf(x.z, y.z, acc);
-          acc = fmaf(x.w, y.w, acc);
-        }
-        sm.A[n][m] = acc;
+      for (int e = 0; e < D; e += 4) {
+        const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
+        const float4 y = *reinterpret_cast<const float4*>(&sm.fk[m][e]);
+        a0 = fmaf(x.x, y.x, a0);
+        a1 = fmaf(x.y, y.y, a1);
+        a2 = fmaf(x.z, y.z, a2);
+        a3 = fmaf(x.w, y.w, a3);
       }
+      sm.A[n][j] = (a0 + a1) + (a2 + a3);
     }
   }
   __syncthreads();
-  if (!bad && tid < N) {
+  if (!bad) {                             // four threads per node share the dot product with z (rows past N are zero)
+    const int n = tid >> 2, part = tid & 3;
     float den = 0.f;
-    for (int e = 0; e < D; e += 4) {
-      const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(tid, (e & 31) >> 2));
+#pragma unroll
+    for (int e = 32 * part; e < 32 * part + 32; e += 4) {
+      const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
       den = fmaf(x.x, sm.z[e], den);
       den = fmaf(x.y, sm.z[e + 1], den);
       den = fmaf(x.z, sm.z[e + 2], den);
       den = fmaf(x.w, sm.z[e + 3], den);
     }
-    unsigned long long mk = sm.mask[tid];
-    while (mk) {
-      const int m = __ffsll((long long)mk) - 1;
-      mk &= mk - 1;
-      den += sm.A[tid][m];
+    den += __shfl_xor_sync(0xffffffffu, den, 1);
+    den += __shfl_xor_sync(0xffffffffu, den, 2);
+    if (part == 0 && n < N) {
+      for (int j = 0; j < sm.depth[n]; ++j) den += sm.A[n][j];
+      sm.den[n] = den;
     }
-    sm.den[tid] = den;
   }
   __syncthreads();
 
@@ -259,32 +289,33 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
           : "r"(taddr)
           : "memory");
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // Walk the ancestor distance j in the outer loop: the value at distance j feeds both the tree term
+      // (weight A[n][j]) and tap j of the unfolded convolution; behind the chain the taps read the committed window.
+      float conv[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) conv[i] = 0.f;
+      const int jmax = max(sm.max_depth, W);
+      for (int j = 0; j < jmax; ++j) {
+        const float wj = j < W ? sm.w[j][c] : 0.f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int n = n0 + i;
+          if (n < N) {
+            const int dep = sm.depth[n];
+            if (j < dep) {
+              const float u = sm.v[sm.anc[n][j]][c];
+              acc[i] = __float_as_uint(fmaf(sm.A[n][j], u, __uint_as_float(acc[i])));
+              conv[i] = fmaf(wj, u, conv[i]);
+            } else if (j < W) {
+              conv[i] = fmaf(wj, sm.win[(W - 2) - (j - dep)][c], conv[i]);   // v_{-(j-dep+1)} of the committed prefix
+            }
+          }
+        }
+      }
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         const int n = n0 + i;
-        if (n < N) {
-          float num = __uint_as_float(acc[i]);
-          unsigned long long mk = sm.mask[n];
-          while (mk) {
-            const int m = __ffsll((long long)mk) - 1;
-            mk &= mk - 1;
-            num = fmaf(sm.A[n][m], sm.v[m][c], num);
-          }
-          float conv = 0.f;
-          int cur = n;
-          const int dep = sm.depth[n];
-          for (int tap = 0; tap < W; ++tap) {
-            float u;
-            if (cur >= 0) {
-              u = sm.v[cur][c];
-              cur = sm.par[cur];
-            } else {
-              u = sm.win[(W - 2) - (tap - dep)][c];     // v_{-(tap-dep+1)} of the committed prefix
-            }
-            conv = fmaf(sm.w[tap][c], u, conv);
-          }
-          o[base + (size_t)n * D + c] = __float2bfloat16_rn(num / (sm.den[n] + eps) + conv);
-        }
+        if (n < N) o[base + (size_t)n * D + c] = __float2bfloat16_rn(__uint_as_float(acc[i]) / (sm.den[n] + eps) + conv[i]);
       }
     }
   }
