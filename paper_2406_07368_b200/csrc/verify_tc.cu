@@ -25,17 +25,18 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 struct Small {
   float fk[NMAX][D + 4];
-  float v[NMAX][D];
-  float A[NMAX][NMAX + 1];            // A[n][j] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself
+  float v[NMAX][D];                   // rows 0..63: the draft values ...
+  float win[LA_MAX_TAPS - 1][D];      // ... rows 64..: the committed window (directly behind v: one row index serves both)
+  float A[NMAX][NMAX + 1];            // A[n][j] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself; 0 past the chain
   float w[LA_MAX_TAPS][D];
-  float win[LA_MAX_TAPS - 1][D];
   float z[D];
   float den[NMAX];
   unsigned long long bars[2];
   int par[NMAX];
   int depth[NMAX];
   int pair_off[NMAX + 1];             // prefix sums of depth: node n owns pairs [pair_off[n], pair_off[n + 1])
-  unsigned char anc[NMAX][NMAX];      // anc[n][j] = ancestor of n at distance j (j < depth[n])
+  unsigned char anc[NMAX][NMAX];      // anc[n][j] = row holding the value at distance j behind n: the ancestor for
+                                      // j < depth[n], else 64 + the window row of v_{-(j - depth[n] + 1)} for j < W, else 0
   unsigned char pair_n[NMAX * (NMAX + 1) / 2];
   unsigned char pair_j[NMAX * (NMAX + 1) / 2];
   uint32_t tmem_base;
@@ -135,6 +136,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 
   // ---- tree preparation: ancestor chains and depths (integer work) ----
   if (tid < N) sm.par[tid] = parent[(size_t)b * N + tid];
+  for (int idx = tid; idx < NMAX * (NMAX + 1); idx += kThreads) (&sm.A[0][0])[idx] = 0.f;
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -163,11 +165,16 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     sm.max_depth = md;
   }
   __syncthreads();
-  if (tid < N)
-    for (int j = 0, o0 = sm.pair_off[tid]; j < sm.depth[tid]; ++j) {
-      sm.pair_n[o0 + j] = (unsigned char)tid;
-      sm.pair_j[o0 + j] = (unsigned char)j;
-    }
+  if (tid < NMAX) {
+    const int dep = tid < N ? sm.depth[tid] : 0, jmax = max(sm.max_depth, W);
+    if (tid < N)
+      for (int j = 0, o0 = sm.pair_off[tid]; j < dep; ++j) {
+        sm.pair_n[o0 + j] = (unsigned char)tid;
+        sm.pair_j[o0 + j] = (unsigned char)j;
+      }
+    for (int j = dep; j < jmax; ++j)     // behind the chain: the committed window while taps remain, else a dummy row
+      sm.anc[tid][j] = (unsigned char)(tid < N && j < W ? NMAX + (W - 2) - (j - dep) : 0);
+  }
 
   // ---- stage phi(q) (fp32, swizzled: the B operand), phi(k), v, z, the window and the taps ----
   const size_t base = (size_t)bh * N * D;
@@ -295,21 +302,14 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 #pragma unroll
       for (int i = 0; i < 32; ++i) conv[i] = 0.f;
       const int jmax = max(sm.max_depth, W);
-      for (int j = 0; j < jmax; ++j) {
+      for (int j = 0; j < jmax; ++j) {     // branch-free: weights are zero where a term does not apply
         const float wj = j < W ? sm.w[j][c] : 0.f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int n = n0 + i;
-          if (n < N) {
-            const int dep = sm.depth[n];
-            if (j < dep) {
-              const float u = sm.v[sm.anc[n][j]][c];
-              acc[i] = __float_as_uint(fmaf(sm.A[n][j], u, __uint_as_float(acc[i])));
-              conv[i] = fmaf(wj, u, conv[i]);
-            } else if (j < W) {
-              conv[i] = fmaf(wj, sm.win[(W - 2) - (j - dep)][c], conv[i]);   // v_{-(j-dep+1)} of the committed prefix
-            }
-          }
+          const float u = sm.v[sm.anc[n][j]][c];          // rows >= 64 fall into the window behind v
+          acc[i] = __float_as_uint(fmaf(sm.A[n][j], u, __uint_as_float(acc[i])));
+          conv[i] = fmaf(wj, u, conv[i]);
         }
       }
 #pragma unroll
