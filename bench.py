@@ -114,6 +114,9 @@ def prefill_workload(W: wl.Workload, rank: int, device):
     sets = [[x.roll(i, dims=0).contiguous() if i else x for x in base] for i in range(nsets)]
     outs = [torch.empty_like(base[0]) for _ in range(nsets)]
     st = ctx.new_state(W.B)
+    ws_bytes = ctx.la_prefill_workspace_bytes(W.B, W.T)      # few chains, long sequence: lend the split workspace
+    if ws_bytes:
+        ctx.la_set_workspace(torch.empty(ws_bytes, dtype=torch.uint8, device=device))
     counter = [0]
 
     def step():
@@ -134,7 +137,7 @@ def prefill_workload(W: wl.Workload, rank: int, device):
     units = W.B * W.H * W.T
     alg_bytes = units * 4 * W.d * 2 + W.B * W.H * (W.d * W.d + W.d) * 4
     info = {"ctx": ctx, "tokens_per_step": tokens, "alg_bytes_per_launch": alg_bytes, "launches_per_step": 1,
-            "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill",
+            "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill" + (" (sequence split: 3 launches)" if ws_bytes else ""),
             "flops_per_launch": units * 4 * W.d * (W.chunk + W.d),
             "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
     return step, e2e_step, info

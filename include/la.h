@@ -198,6 +198,17 @@ la_status la_clear_device_status(la_ctx* ctx, void* stream);
  * against the other. */
 la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which);
 
+/* Optional workspace for la_prefill.  With few (batch, head) chains and a long sequence -- fewer chains
+ * than half the SMs, T >= 2048 -- the grouped processing of Sec. 4.1 is also cut along the sequence:
+ * every segment first computes its own sum of phi(k) v^T, a prefix over the segments gives each its
+ * starting state (the cumulative sum of Sec. 4.1 taken at segment level), and all segments then run
+ * as independent thread blocks.  That needs la_prefill_workspace_bytes(ctx, B, T) bytes of device
+ * memory, which the caller lends to the context here (16-byte aligned; it must stay valid until the
+ * calls that use it have completed; NULL, 0 takes it back).  Without a large enough workspace
+ * la_prefill runs every chain in one thread block; the results agree up to rounding order. */
+la_status la_set_workspace(la_ctx* ctx, void* workspace, uint64_t bytes);
+uint64_t  la_prefill_workspace_bytes(const la_ctx* ctx, int32_t B, int32_t T);
+
 /* Number of kernels the library has launched through this context since creation. */
 int64_t la_launch_count(const la_ctx* ctx);
 

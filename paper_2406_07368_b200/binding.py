@@ -24,7 +24,8 @@ LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
-           "la_launch_count", "la_verify_tree_noalloc"]
+           "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace",
+           "la_prefill_workspace_bytes"]
 
 
 class LaError(RuntimeError):
@@ -66,9 +67,12 @@ def lib() -> C.CDLL:
         L.la_clear_device_status.argtypes = [vp, vp]
         L.la_set_prefill_kernel.argtypes = [vp, i32]
         L.la_launch_count.argtypes = [vp]
+        L.la_set_workspace.argtypes = [vp, vp, C.c_uint64]
+        L.la_prefill_workspace_bytes.argtypes = [vp, i32, i32]
+        L.la_prefill_workspace_bytes.restype = C.c_uint64
         L.la_launch_count.restype = C.c_int64
         for name in EXPORTS:
-            if name not in ("la_status_str", "la_launch_count"):
+            if name not in ("la_status_str", "la_launch_count", "la_prefill_workspace_bytes"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -221,6 +225,18 @@ class Context:
 
     def la_launch_count(self) -> int:
         return int(lib().la_launch_count(self._h))
+
+    def la_prefill_workspace_bytes(self, B: int, T: int) -> int:
+        return int(lib().la_prefill_workspace_bytes(self._h, B, T))
+
+    def la_set_workspace(self, workspace: torch.Tensor | None) -> None:
+        """Lends a device buffer (any dtype, contiguous) to the context; it is kept alive by this object."""
+        self._ws = workspace
+        if workspace is None:
+            _check("la_set_workspace", lib().la_set_workspace(self._h, None, 0))
+        else:
+            _check("la_set_workspace", lib().la_set_workspace(self._h, _ptr(workspace, name="workspace"),
+                                                              workspace.numel() * workspace.element_size()))
 
 
 def la_verify_tree_noalloc(H: int, d: int, conv_taps: int, phi: str, eps: float, io: str, q, k, v, parent, conv_w,

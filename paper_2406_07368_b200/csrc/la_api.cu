@@ -61,6 +61,8 @@ la_status la_create(const la_config* cfg, la_ctx** out) {
   ctx->prefill_kernel = 0;
   ctx->launches = 0;
   ctx->d_status = nullptr;
+  ctx->ws = nullptr;
+  ctx->ws_bytes = 0;
   if (cudaGetDevice(&ctx->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess ||
       cudaMalloc(&ctx->d_status, sizeof(int)) != cudaSuccess ||
@@ -89,6 +91,18 @@ la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which) {
 }
 
 int64_t la_launch_count(const la_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+la_status la_set_workspace(la_ctx* ctx, void* workspace, uint64_t bytes) {
+  if (!ctx || (workspace == nullptr) != (bytes == 0) || !aligned16(workspace)) return LA_ERR_INVALID_ARG;
+  ctx->ws = workspace;
+  ctx->ws_bytes = bytes;
+  return LA_OK;
+}
+
+uint64_t la_prefill_workspace_bytes(const la_ctx* ctx, int32_t B, int32_t T) {
+  if (!ctx || B < 1 || T < 1) return 0;
+  return la::prefill_workspace_bytes(ctx, B, T);
+}
 
 la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
                      const float* conv_w, int32_t init_state, la_state* st, void* o, void* stream) {

@@ -56,6 +56,8 @@ struct la_ctx {
   int prefill_kernel;     // 0 auto, 1 CUDA-core kernel
   int64_t launches;
   int sm_count;
+  void* ws;               // caller-provided device workspace (may be null)
+  size_t ws_bytes;
 };
 
 // Kernel launchers (one per translation unit).  All return the cudaError_t of the launch.
@@ -77,4 +79,6 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
 cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
                              const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s,
                              bool* handled);
+// Workspace la_prefill can use for a launch of B sequences of T tokens (0: none needed).
+size_t prefill_workspace_bytes(const la_ctx* ctx, int B, int T);
 }  // namespace la

@@ -24,6 +24,8 @@
 // records LA_ERR_TIMEOUT, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <algorithm>
+
 #include "la_common.cuh"
 
 namespace la {
@@ -286,7 +288,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                   const __grid_constant__ CUtensorMap mv, const float* __restrict__ w, float* __restrict__ S,
                   float* __restrict__ z, __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos,
-                  __nv_bfloat16* __restrict__ o, int* status, int H, int T, int W, float eps, int init) {
+                  __nv_bfloat16* __restrict__ o, int* status, int H, int Ttot, int W, float eps, int init, int nseg,
+                  int seg_len) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -298,7 +301,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   volatile int* abort = &sm.abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int bh = blockIdx.x, h = bh % H;
+  // A launch covers BH chains cut into nseg segments of seg_len tokens (nseg = 1: whole chains).  Unit u owns
+  // tokens [y0, y0 + T) of chain bh; state, window and z of a unit are addressed by u.
+  const int u = blockIdx.x, bh = u / nseg, h = bh % H;
+  const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
   const int nchunks = (T + TILE - 1) / TILE;
   uint32_t bar[kNumBars];
 #pragma unroll
@@ -330,14 +336,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   }
   for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
-    halo0[idx] = init ? win[(size_t)bh * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
+    halo0[idx] = init ? win[(size_t)u * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
   for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
     reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   if (tid < TILE) {
     *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
     if (init)
-      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)bh * D + tid]);
+      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)u * D + tid]);
   }
   fence_proxy_async();
   tc_fence_before();
@@ -350,20 +356,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     if (lane == 0) {
       bool ok = true;
       mbar_expect_tx(bar[B_FULL_K0], TILE_BYTES);
-      tma_load(sbase + OFF_K0, &mk, 0, 0, bh, bar[B_FULL_K0]);
-      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, 0, bh, bar[B_FULL_K0]);
+      tma_load(sbase + OFF_K0, &mk, 0, y0, bh, bar[B_FULL_K0]);
+      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, y0, bh, bar[B_FULL_K0]);
       if (nchunks > 1) {
         mbar_expect_tx(bar[B_FULL_K1], TILE_BYTES);
-        tma_load(sbase + OFF_K1, &mk, 0, TILE, bh, bar[B_FULL_K1]);
-        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, TILE, bh, bar[B_FULL_K1]);
+        tma_load(sbase + OFF_K1, &mk, 0, y0 + TILE, bh, bar[B_FULL_K1]);
+        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, y0 + TILE, bh, bar[B_FULL_K1]);
       }
       mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
-      tma_load(sbase + OFF_Q, &mq, 0, 0, bh, bar[B_FULL_Q]);
-      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, 0, bh, bar[B_FULL_Q]);
+      tma_load(sbase + OFF_Q, &mq, 0, y0, bh, bar[B_FULL_Q]);
+      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0, bh, bar[B_FULL_Q]);
       for (int n = 0; n < 2 && n < nchunks; ++n) {
         mbar_expect_tx(bar[B_FULL_V0 + n], TILE_BYTES);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, n * TILE, bh, bar[B_FULL_V0 + n]);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, n * TILE, bh, bar[B_FULL_V0 + n]);
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, bar[B_FULL_V0 + n]);
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, bar[B_FULL_V0 + n]);
       }
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
@@ -394,8 +400,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           ok = mbar_wait(bar[B_MMA_S], par, abort);             // this K buffer is free: it takes tile n+2
           if (!ok) break;
           mbar_expect_tx(kbar, TILE_BYTES);
-          tma_load(kbuf, &mk, 0, (n + 2) * TILE, bh, kbar);
-          tma_load(kbuf + BOX_BYTES, &mk, 64, (n + 2) * TILE, bh, kbar);
+          tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
+          tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
         }
         if (n >= 1) {
           // group B is done with tile n-1: O may be overwritten, and its V buffer takes tile n+1
@@ -405,8 +411,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           if (n + 1 < nchunks) {
             const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
             mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
-            tma_load(vnext, &mv, 0, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-            tma_load(vnext + BOX_BYTES, &mv, 64, (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+            tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+            tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
           }
         }
         if (has_state) {
@@ -422,8 +428,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
           if (!ok) break;
           mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
-          tma_load(sbase + OFF_Q, &mq, 0, (n + 1) * TILE, bh, bar[B_FULL_Q]);
-          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, (n + 1) * TILE, bh, bar[B_FULL_Q]);
+          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
+          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
         }
         ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in TMEM
         if (!ok) break;
@@ -446,7 +452,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     const uint32_t lane_addr = (uint32_t)(32 * (wa & 3)) << 16;
     unsigned char* Qb = smem + OFF_Q + hf * BOX_BYTES;
     unsigned char* Sb = smem + OFF_S + hf * BOX_BYTES;
-    float* Sg = S + (size_t)bh * D * D + (size_t)r * D + 64 * hf;
+    float* Sg = S + (size_t)u * D * D + (size_t)r * D + 64 * hf;
     bool ok = true;
 
     if (init) {   // [S|z] -> TMEM (fp32); S -> bf16 copy in shared memory (z was copied during set-up)
@@ -464,7 +470,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
       }
       if (hf == 0) {
-        tmem_st1(tmem + lane_addr + Z_COL, __float_as_uint(z[(size_t)bh * D + r]));
+        tmem_st1(tmem + lane_addr + Z_COL, __float_as_uint(z[(size_t)u * D + r]));
 #pragma unroll
         for (int c = 1; c < 16; ++c) tmem_st1(tmem + lane_addr + Z_COL + c, 0u);
       }
@@ -566,7 +572,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         if (hf == 0) {
           const float zz = __uint_as_float(tmem_ld1(tmem + lane_addr + Z_COL));
           tmem_wait_ld();
-          if (last) z[(size_t)bh * D + r] = zz;
+          if (last) z[(size_t)u * D + r] = zz;
           else *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(r, 0)) = __float2bfloat16_rn(zz);
         }
       }
@@ -607,7 +613,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
         tmem_wait_ld();
         const float rden = 1.f / (den + eps);
-        __nv_bfloat16* og = o + ((size_t)bh * T + (size_t)n * TILE + r) * D;
+        __nv_bfloat16* og = o + ((size_t)bh * Ttot + y0 + (size_t)n * TILE + r) * D;
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           uint32_t v[32];
@@ -633,8 +639,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     }
     if (ok && tid < D) {
       const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
-      for (int i = 0; i < W - 1; ++i) win[((size_t)bh * (W - 1) + i) * D + tid] = halo[i * D + tid];
-      if (tid == 0 && h == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
+      for (int i = 0; i < W - 1; ++i) win[((size_t)u * (W - 1) + i) * D + tid] = halo[i * D + tid];
+      if (tid == 0 && h == 0 && nseg == 1) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
   }
 
@@ -649,6 +655,185 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     __syncwarp();
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---- sequence split: local state of a segment ------------------------------------------------------
+// For chains too few to fill the GPU the sequence is cut into segments that run as separate CTAs.  This
+// kernel computes, for one segment, only its own contribution [dS | dz] = sum phi(k) [v | 1]^T (K and V are
+// read, phi applied to K, one product per tile) and stores it in fp32.  A prefix sum over the segments
+// (prefix_kernel) turns the contributions into the state each segment starts from.
+constexpr int kStateThreads = 288;       // 8 compute warps + 1 issue warp
+constexpr uint32_t ST_OFF_K = 0, ST_OFF_V = 2 * TILE_BYTES, ST_OFF_ONES = 4 * TILE_BYTES, ST_OFF_SMALL = ST_OFF_ONES + 4096;
+constexpr uint32_t kStateSmem = ST_OFF_SMALL + 256 + 1024;
+enum { SB_FULL_K0 = 0, SB_FULL_K1, SB_FULL_V0, SB_FULL_V1, SB_PHI, SB_MMA, kStateBars };
+
+template <int PHI>
+__global__ void __launch_bounds__(kStateThreads, 1)
+segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
+                     float* __restrict__ S_out, float* __restrict__ z_out, int* status, int Ttot, int nseg,
+                     int seg_len) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + ST_OFF_SMALL);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ST_OFF_SMALL + 128);
+  volatile int* abort = reinterpret_cast<int*>(smem + ST_OFF_SMALL + 132);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int u = blockIdx.x, bh = u / nseg;
+  const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
+  const int nchunks = (T + TILE - 1) / TILE;
+  uint32_t bar[kStateBars];
+#pragma unroll
+  for (int i = 0; i < kStateBars; ++i) bar[i] = smem_u32(&bars[i]);
+
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) mbar_init(bar[i], 1);
+    mbar_init(bar[SB_PHI], 256);
+    mbar_init(bar[SB_MMA], 1);
+    *abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(256u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int idx = tid; idx < 4096 / 16; idx += kStateThreads)
+    reinterpret_cast<uint4*>(smem + ST_OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  if (tid < TILE) *reinterpret_cast<__nv_bfloat16*>(smem + ST_OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  constexpr uint32_t SCOL = 0, ZCOL = 128;
+
+  if (warp == 8) {
+    if (lane == 0) {
+      auto load_tile = [&](int n) {
+        const uint32_t b2 = n & 1;
+        mbar_expect_tx(bar[SB_FULL_K0 + b2], TILE_BYTES);
+        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES, &mk, 0, y0 + n * TILE, bh, bar[SB_FULL_K0 + b2]);
+        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES + BOX_BYTES, &mk, 64, y0 + n * TILE, bh, bar[SB_FULL_K0 + b2]);
+        mbar_expect_tx(bar[SB_FULL_V0 + b2], TILE_BYTES);
+        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, bar[SB_FULL_V0 + b2]);
+        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, bar[SB_FULL_V0 + b2]);
+      };
+      for (int n = 0; n < 2 && n < nchunks; ++n) load_tile(n);
+      for (int n = 0; n < nchunks; ++n) {
+        const uint32_t b2 = n & 1;
+        if (!mbar_wait(bar[SB_PHI], n & 1, abort) || !mbar_wait(bar[SB_FULL_V0 + b2], (n >> 1) & 1, abort)) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {     // [dS | dz] += phi(K)^T [V | 1]
+          const uint64_t kd = desc_mnmajor(sbase + ST_OFF_K + b2 * TILE_BYTES, ks);
+          mma_bf16(tmem + SCOL, kd, desc_mnmajor(sbase + ST_OFF_V + b2 * TILE_BYTES, ks), idesc(true, true, 128), n > 0 || ks > 0);
+          mma_bf16(tmem + ZCOL, kd, desc_ext(sbase + ST_OFF_ONES, ks), idesc(true, true, 16), n > 0 || ks > 0);
+        }
+        mma_commit(bar[SB_MMA]);
+        if (!mbar_wait(bar[SB_MMA], n & 1, abort)) break;       // both buffers of this tile are free
+        if (n + 2 < nchunks) load_tile(n + 2);
+      }
+    }
+  } else {
+    bool ok = true;
+    for (int n = 0; n < nchunks; ++n) {
+      const int valid = min(TILE, T - n * TILE);
+      ok = ok && mbar_wait(bar[SB_FULL_K0 + (n & 1)], (n >> 1) & 1, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        const int ct = tid & 15, rg = tid >> 4;
+        unsigned char* Kb = smem + ST_OFF_K + (n & 1) * TILE_BYTES + (ct >> 3) * BOX_BYTES;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int j = rg + 16 * i;
+          uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
+          *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      fence_proxy_async();
+      mbar_arrive(bar[SB_PHI]);
+    }
+    // Wait for the last two products in turn (tile L was loaded only after product L-2 had completed, so the
+    // barrier is at phase L-1 or later here and a parity wait cannot be fooled by an older phase).
+    for (int n = max(0, nchunks - 2); n < nchunks; ++n) ok = ok && mbar_wait(bar[SB_MMA], n & 1, abort);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const int r = 32 * (warp & 3) + lane, hf = warp >> 2;
+      const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
+      float* Sg = S_out + (size_t)u * D * D + (size_t)r * D + 64 * hf;
+#pragma unroll
+      for (int qq = 0; qq < 2; ++qq) {
+        uint32_t v[32];
+        LA_TMEM_LD32(tmem + lane_addr + SCOL + 64 * hf + 32 * qq, v);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; e += 4)
+          *reinterpret_cast<float4*>(Sg + 32 * qq + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                                                     __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+      }
+      if (hf == 0) {
+        const uint32_t zz = tmem_ld1(tmem + lane_addr + ZCOL);
+        tmem_wait_ld();
+        z_out[(size_t)u * D + r] = __uint_as_float(zz);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (*abort) {
+    if (tid == 0) report(status, LA_ERR_TIMEOUT);
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);
+  }
+  if (warp == 8) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  }
+}
+
+// Exclusive prefix over the segments of one chain, in place: on return S_seg[bh][s] / z_seg[bh][s] hold the state
+// segment s starts from, win_seg its incoming window, and S / z / win / pos of the caller the final state.
+// grid = (BH, d*d / 1024), 256 threads, four consecutive elements of S per thread.
+__global__ void __launch_bounds__(256)
+prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat16* __restrict__ win_seg,
+              const __nv_bfloat16* __restrict__ v, float* __restrict__ S, float* __restrict__ z,
+              __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int H, int Ttot, int W, int nseg, int seg_len,
+              int init) {
+  const int bh = blockIdx.x, e4 = (blockIdx.y * 256 + threadIdx.x) * 4;
+  float4 run = init ? *reinterpret_cast<const float4*>(S + (size_t)bh * D * D + e4) : make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int sg = 0; sg < nseg; ++sg) {
+    float4* p = reinterpret_cast<float4*>(S_seg + ((size_t)bh * nseg + sg) * D * D + e4);
+    const float4 d = *p;
+    *p = run;
+    run.x += d.x; run.y += d.y; run.z += d.z; run.w += d.w;
+  }
+  *reinterpret_cast<float4*>(S + (size_t)bh * D * D + e4) = run;
+  if (blockIdx.y == 0 && threadIdx.x < D) {
+    const int c = threadIdx.x;
+    float rz = init ? z[(size_t)bh * D + c] : 0.f;
+    for (int sg = 0; sg < nseg; ++sg) {
+      float* p = z_seg + ((size_t)bh * nseg + sg) * D + c;
+      const float d = *p;
+      *p = rz;
+      rz += d;
+    }
+    z[(size_t)bh * D + c] = rz;
+    // incoming windows: the W-1 values of v before each segment; before the first one the caller's window or zeros
+    for (int sg = 0; sg < nseg; ++sg)
+      for (int i = 0; i < W - 1; ++i) {
+        const int t = sg * seg_len - (W - 1) + i;
+        __nv_bfloat16 x = __float2bfloat16_rn(0.f);
+        if (t >= 0) x = v[((size_t)bh * Ttot + t) * D + c];
+        else if (init) x = win[((size_t)bh * (W - 1) + i) * D + c];      // sg == 0: t = i - (W-1)
+        win_seg[(((size_t)bh * nseg + sg) * (W - 1) + i) * D + c] = x;
+      }
+    for (int i = 0; i < W - 1; ++i)      // final window: the last W-1 values of v (Ttot >= W-1 whenever the split is used)
+      win[((size_t)bh * (W - 1) + i) * D + c] = v[((size_t)bh * Ttot + Ttot - (W - 1) + i) * D + c];
+    if (c == 0 && bh % H == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + Ttot;
   }
 }
 
@@ -686,12 +871,12 @@ static bool make_map(CUtensorMap* m, const void* base, int BH, int T) {
 }  // namespace tc
 
 template <int PHI>
-static cudaError_t launch_w(const la_config& c, int BH, int T, const CUtensorMap& mq, const CUtensorMap& mk,
-                            const CUtensorMap& mv, const float* w, int init, const la_state& st, void* o, int* status,
-                            cudaStream_t s) {
+static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
+                            const CUtensorMap& mv, const float* w, int init, float* S, float* z, __nv_bfloat16* win,
+                            int64_t* pos, void* o, int* status, int nseg, int seg_len, cudaStream_t s) {
   const size_t smem = tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               __nv_bfloat16*, int*, int, int, int, float, int);
+               __nv_bfloat16*, int*, int, int, int, float, int, int, int);
   switch (c.conv_taps) {     // unrolled tap loops for the common small widths
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
@@ -702,9 +887,35 @@ static cudaError_t launch_w(const la_config& c, int BH, int T, const CUtensorMap
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(BH), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, w, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
-                                                  (__nv_bfloat16*)o, status, c.H, T, c.conv_taps, c.eps, init);
+  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, w, S, z, win, pos, (__nv_bfloat16*)o, status, c.H, T,
+                                                     c.conv_taps, c.eps, init, nseg, seg_len);
   return cudaGetLastError();
+}
+
+// Segments per chain for a launch of BH chains of T tokens: 1 unless the chains are too few to fill the GPU and
+// long enough to cut (every segment a multiple of 128 tokens, at least 1024).
+static void plan_split(const la_ctx* ctx, int BH, int T, int* nseg, int* seg_len) {
+  *nseg = 1;
+  *seg_len = T;
+  if (2 * BH > ctx->sm_count || T < 2048) return;
+  int n = std::min(2 * ctx->sm_count / BH, T / 1024);
+  if (n < 2) return;
+  const int len = ((T + n - 1) / n + tc::TILE - 1) / tc::TILE * tc::TILE;
+  n = (T + len - 1) / len;
+  if (n < 2) return;
+  *nseg = n;
+  *seg_len = len;
+}
+static size_t split_bytes(const la_config& c, int BH, int nseg) {
+  return (size_t)BH * nseg * ((size_t)tc::D * tc::D * 4 + tc::D * 4 + (size_t)(c.conv_taps > 1 ? c.conv_taps - 1 : 1) * tc::D * 2);
+}
+
+size_t prefill_workspace_bytes(const la_ctx* ctx, int B, int T) {
+  const la_config& c = ctx->cfg;
+  if (c.io_dtype != LA_BF16 || c.d != tc::D) return 0;
+  int nseg, seg_len;
+  plan_split(ctx, B * c.H, T, &nseg, &seg_len);
+  return nseg > 1 ? split_bytes(c, B * c.H, nseg) : 0;
 }
 
 cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
@@ -717,10 +928,37 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   CUtensorMap mq, mk, mv;
   if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T))
     return cudaSuccess;   // no tensor-map support: the CUDA-core kernel takes over
-  cudaError_t e = c.phi == LA_PHI_ELU1
-                      ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, w, init, st, o, ctx->d_status, s)
-                      : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, w, init, st, o, ctx->d_status, s);
-  ctx->launches += 1;
+  int nseg, seg_len;
+  plan_split(ctx, BH, T, &nseg, &seg_len);
+  if (nseg > 1 && (ctx->ws == nullptr || ctx->ws_bytes < split_bytes(c, BH, nseg) || T < c.conv_taps)) nseg = 1, seg_len = T;
+  const bool elu = c.phi == LA_PHI_ELU1;
+  cudaError_t e;
+  if (nseg == 1) {
+    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, o,
+                                    ctx->d_status, 1, T, s)
+            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, o,
+                                    ctx->d_status, 1, T, s);
+    ctx->launches += 1;
+    *handled = true;
+    return e;
+  }
+  // Sequence split: local states of all segments, prefix over the segments, then every segment as its own CTA.
+  const int units = BH * nseg;
+  float* S_seg = static_cast<float*>(ctx->ws);
+  float* z_seg = S_seg + (size_t)units * tc::D * tc::D;
+  __nv_bfloat16* win_seg = reinterpret_cast<__nv_bfloat16*>(z_seg + (size_t)units * tc::D);
+  auto skern = elu ? tc::segment_state_kernel<LA_PHI_ELU1> : tc::segment_state_kernel<LA_PHI_RELU>;
+  e = cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kStateSmem);
+  if (e != cudaSuccess) return e;
+  skern<<<dim3(units), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, S_seg, z_seg, ctx->d_status, T, nseg, seg_len);
+  tc::prefix_kernel<<<dim3(BH, tc::D * tc::D / 1024), dim3(256), 0, s>>>(S_seg, z_seg, win_seg, (const __nv_bfloat16*)v, st.S,
+                                                                          st.z, (__nv_bfloat16*)st.win, st.pos, c.H, T,
+                                                                          c.conv_taps, nseg, seg_len, init);
+  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, w, 1, S_seg, z_seg, win_seg, st.pos, o, ctx->d_status, nseg,
+                                  seg_len, s)
+          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, w, 1, S_seg, z_seg, win_seg, st.pos, o, ctx->d_status, nseg,
+                                  seg_len, s);
+  ctx->launches += 3;
   *handled = true;
   return e;
 }

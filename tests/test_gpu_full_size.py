@@ -51,6 +51,9 @@ def test_long_prefill_full_size_then_decode():
     q, k, v = W.prefill_inputs()
     w = W.weights()
     ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, W.io, chunk=W.chunk)
+    ws = torch.empty(ctx.la_prefill_workspace_bytes(W.B, W.T), dtype=torch.uint8, device="cuda")
+    assert ws.numel() > 0                       # 32 chains: the sequence-split path, as in the benchmark
+    ctx.la_set_workspace(ws)
     st = ctx.new_state(W.B)
     o = ctx.la_prefill(dev(q), dev(k), dev(v), dev(w, "f32"), st)
     heads = (0, 13, 31)

@@ -85,6 +85,39 @@ def test_prefill_continuation(kernel, io, T1, T2):
     check_state(st, wst, TOL[io])
 
 
+@pytest.mark.parametrize("T,W,phi,eps,init", [(2500, 3, "elu1", 0.0, False), (4099, 5, "relu", 1e-6, False),
+                                              (3000, 4, "elu1", 0.0, True), (2048, 1, "elu1", 0.0, False)])
+def test_prefill_sequence_split_with_workspace(T, W, phi, eps, init):
+    """Few chains and a long sequence: with a workspace the sequence is cut into segments run as separate CTAs."""
+    io, B, H, d = "bf16", 1, 2, 128
+    q, k, v, w = make(io, B, H, d, T, W, seed=T, scale=d ** -0.5)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    need = ctx.la_prefill_workspace_bytes(B, T)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    ctx.la_set_workspace(ws)
+    st = ctx.new_state(B)
+    ost = None
+    if init:
+        q0, k0, v0, _ = make(io, B, H, d, 70, W, seed=1, scale=d ** -0.5)
+        _, ost = orc.prefill_quadratic(q0, k0, v0, w, phi, eps)
+        st = oracle_state_to_dev(ost, io)
+    n0 = ctx.la_launch_count()
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st, init_state=init)
+    assert ctx.la_launch_count() - n0 == 3                     # segment states, prefix, segments
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want, wst = orc.prefill_chunked(q, k, v, w, phi, eps, 256, ost)
+    assert rel_err(host(o), want) < TOL[io]
+    check_state(st, wst, TOL[io])
+    # without the workspace the same call runs one CTA per chain and agrees up to rounding order
+    ctx.la_set_workspace(None)
+    st2 = ctx.new_state(B) if not init else oracle_state_to_dev(ost, io)
+    o2 = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st2, init_state=init)
+    assert rel_err(host(o2), want) < TOL[io]
+    assert rel_err(host(o2), host(o)) < TOL[io]
+    assert torch.equal(st.win, st2.win) and torch.equal(st.pos, st2.pos)
+
+
 def test_prefill_is_causal_bitwise():
     """Perturbing token j leaves every earlier output bit-identical (no leakage through the conv)."""
     io, B, H, d, T, W = "bf16", 1, 2, 128, 300, 8
