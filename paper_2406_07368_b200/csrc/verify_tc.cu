@@ -27,20 +27,21 @@ struct Small {
   float fk[NMAX][D + 4];
   float v[NMAX][D];                   // rows 0..63: the draft values ...
   float win[LA_MAX_TAPS - 1][D];      // ... rows 64..: the committed window (directly behind v: one row index serves both)
-  float A[NMAX][NMAX + 1];            // A[n][j] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself; 0 past the chain
+  float A[NMAX][NMAX];                // A[j][n] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself; 0 past the chain
   float w[LA_MAX_TAPS][D];
   float z[D];
   float den[NMAX];
   unsigned long long bars[2];
   int par[NMAX];
   int depth[NMAX];
-  int pair_off[NMAX + 1];             // prefix sums of depth: node n owns pairs [pair_off[n], pair_off[n + 1])
-  unsigned char anc[NMAX][NMAX];      // anc[n][j] = row holding the value at distance j behind n: the ancestor for
+  int pair_off[NMAX + 1];             // prefix sums of depth: node n owns pairs [pair_off[n], pair_off[n + 1]); [64] = total
+  unsigned char anc[NMAX][NMAX];      // anc[j][n] = row holding the value at distance j behind n: the ancestor for
                                       // j < depth[n], else 64 + the window row of v_{-(j - depth[n] + 1)} for j < W, else 0
   unsigned char pair_n[NMAX * (NMAX + 1) / 2];
   unsigned char pair_j[NMAX * (NMAX + 1) / 2];
   uint32_t tmem_base;
   int max_depth;
+  int scan_carry;
   int bad;
   int abort;
 };
@@ -136,7 +137,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 
   // ---- tree preparation: ancestor chains and depths (integer work) ----
   if (tid < N) sm.par[tid] = parent[(size_t)b * N + tid];
-  for (int idx = tid; idx < NMAX * (NMAX + 1); idx += kThreads) (&sm.A[0][0])[idx] = 0.f;
+  for (int idx = tid; idx < NMAX * NMAX; idx += kThreads) (&sm.A[0][0])[idx] = 0.f;
+  if (tid == 0) sm.max_depth = 0;
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -145,7 +147,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     int dep = 0, m = tid;
     bool ok = true;
     while (m >= 0) {                     // m strictly decreases: at most N iterations
-      sm.anc[tid][dep++] = (unsigned char)m;
+      sm.anc[dep++][tid] = (unsigned char)m;
       const int p = sm.par[m];
       if (p < -1 || p >= m) { ok = false; break; }
       m = p;
@@ -154,26 +156,34 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     if (!ok) sm.bad = 1;
   }
   __syncthreads();
-  if (tid == 0) {                        // pair offsets and the deepest chain (a few dozen integer steps)
-    int off = 0, md = 0;
-    for (int n = 0; n < N; ++n) {
-      sm.pair_off[n] = off;
-      off += sm.depth[n];
-      md = max(md, sm.depth[n]);
+  int my_dep = 0, my_off = 0;
+  if (tid < NMAX) {                      // exclusive prefix of the depths over the two warps that hold the nodes
+    my_dep = tid < N ? sm.depth[tid] : 0;
+    int x = my_dep;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if (lane >= o) x += y;
     }
-    sm.pair_off[N] = off;
-    sm.max_depth = md;
+    my_off = x - my_dep;
+    if (tid == 31) sm.scan_carry = x;
+    atomicMax(&sm.max_depth, my_dep);
   }
   __syncthreads();
   if (tid < NMAX) {
-    const int dep = tid < N ? sm.depth[tid] : 0, jmax = max(sm.max_depth, W);
+    if (tid >= 32) my_off += sm.scan_carry;
+    sm.pair_off[tid] = my_off;
+    if (tid == NMAX - 1) sm.pair_off[NMAX] = my_off + my_dep;
+  }
+  if (tid < NMAX) {
+    const int dep = my_dep, jmax = max(sm.max_depth, W);
     if (tid < N)
-      for (int j = 0, o0 = sm.pair_off[tid]; j < dep; ++j) {
+      for (int j = 0, o0 = my_off; j < dep; ++j) {
         sm.pair_n[o0 + j] = (unsigned char)tid;
         sm.pair_j[o0 + j] = (unsigned char)j;
       }
     for (int j = dep; j < jmax; ++j)     // behind the chain: the committed window while taps remain, else a dummy row
-      sm.anc[tid][j] = (unsigned char)(tid < N && j < W ? NMAX + (W - 2) - (j - dep) : 0);
+      sm.anc[j][tid] = (unsigned char)(tid < N && j < W ? NMAX + (W - 2) - (j - dep) : 0);
   }
 
   // ---- stage phi(q) (fp32, swizzled: the B operand), phi(k), v, z, the window and the taps ----
@@ -238,9 +248,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 
   // ---- meanwhile: scores of every (node, ancestor) pair, one pair per thread, and the denominators ----
   if (!bad) {
-    const int npairs = sm.pair_off[N];
+    const int npairs = sm.pair_off[NMAX];
     for (int pi = tid; pi < npairs; pi += kThreads) {
-      const int n = sm.pair_n[pi], j = sm.pair_j[pi], m = sm.anc[n][j];
+      const int n = sm.pair_n[pi], j = sm.pair_j[pi], m = sm.anc[j][n];
       float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 8
       for (int e = 0; e < D; e += 4) {
@@ -251,7 +261,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
         a2 = fmaf(x.z, y.z, a2);
         a3 = fmaf(x.w, y.w, a3);
       }
-      sm.A[n][j] = (a0 + a1) + (a2 + a3);
+      sm.A[j][n] = (a0 + a1) + (a2 + a3);
     }
   }
   __syncthreads();
@@ -269,7 +279,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     den += __shfl_xor_sync(0xffffffffu, den, 1);
     den += __shfl_xor_sync(0xffffffffu, den, 2);
     if (part == 0 && n < N) {
-      for (int j = 0; j < sm.depth[n]; ++j) den += sm.A[n][j];
+      for (int j = 0; j < sm.depth[n]; ++j) den += sm.A[j][n];
       sm.den[n] = den;
     }
   }
@@ -305,11 +315,19 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
       for (int j = 0; j < jmax; ++j) {     // branch-free: weights are zero where a term does not apply
         const float wj = j < W ? sm.w[j][c] : 0.f;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int n = n0 + i;
-          const float u = sm.v[sm.anc[n][j]][c];          // rows >= 64 fall into the window behind v
-          acc[i] = __float_as_uint(fmaf(sm.A[n][j], u, __uint_as_float(acc[i])));
-          conv[i] = fmaf(wj, u, conv[i]);
+        for (int i = 0; i < 32; i += 4) {                  // four nodes per table load
+          const float4 a4 = *reinterpret_cast<const float4*>(&sm.A[j][n0 + i]);
+          const uint32_t r4 = *reinterpret_cast<const uint32_t*>(&sm.anc[j][n0 + i]);
+          const float u0 = sm.v[r4 & 0xff][c], u1 = sm.v[(r4 >> 8) & 0xff][c];          // rows >= 64: the window behind v
+          const float u2 = sm.v[(r4 >> 16) & 0xff][c], u3 = sm.v[r4 >> 24][c];
+          acc[i] = __float_as_uint(fmaf(a4.x, u0, __uint_as_float(acc[i])));
+          acc[i + 1] = __float_as_uint(fmaf(a4.y, u1, __uint_as_float(acc[i + 1])));
+          acc[i + 2] = __float_as_uint(fmaf(a4.z, u2, __uint_as_float(acc[i + 2])));
+          acc[i + 3] = __float_as_uint(fmaf(a4.w, u3, __uint_as_float(acc[i + 3])));
+          conv[i] = fmaf(wj, u0, conv[i]);
+          conv[i + 1] = fmaf(wj, u1, conv[i + 1]);
+          conv[i + 2] = fmaf(wj, u2, conv[i + 2]);
+          conv[i + 3] = fmaf(wj, u3, conv[i + 3]);
         }
       }
 #pragma unroll
