@@ -30,7 +30,7 @@ struct Small {
   float A[NMAX][NMAX];                // A[j][n] = phi(q_n) . phi(k of the ancestor of n at distance j), j = 0 is n itself; 0 past the chain
   float w[LA_MAX_TAPS][D];
   float z[D];
-  float den[NMAX];
+  float den[NMAX];                    // 1 / (denominator + eps) per node
   unsigned long long bars[2];
   int par[NMAX];
   int depth[NMAX];
@@ -135,6 +135,21 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
 
+  // ---- q, k, v of the tree: all loads in flight before the tree is prepared (used in the staging step below) ----
+  const size_t base = (size_t)bh * N * D;
+  constexpr int ITERS = NMAX * (D / 4) / kThreads;         // 8 chunks of 4 values per thread
+  uint2 uq[ITERS], uk[ITERS], uv[ITERS];
+#pragma unroll
+  for (int it = 0; it < ITERS; ++it) {                   // all loads in flight before the first use
+    const int idx = tid + it * kThreads, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
+    uq[it] = uk[it] = uv[it] = make_uint2(0u, 0u);
+    if (n < N) {
+      uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
+      uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
+      uv[it] = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
+    }
+  }
+
   // ---- tree preparation: ancestor chains and depths (integer work) ----
   if (tid < N) sm.par[tid] = parent[(size_t)b * N + tid];
   for (int idx = tid; idx < NMAX * NMAX; idx += kThreads) (&sm.A[0][0])[idx] = 0.f;
@@ -187,20 +202,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
   }
 
   // ---- stage phi(q) (fp32, swizzled: the B operand), phi(k), v, z, the window and the taps ----
-  const size_t base = (size_t)bh * N * D;
   {
-    constexpr int ITERS = NMAX * (D / 4) / kThreads;       // 8 chunks of 4 values per thread
-    uint2 uq[ITERS], uk[ITERS], uv[ITERS];
-#pragma unroll
-    for (int it = 0; it < ITERS; ++it) {                   // all loads in flight before the first use
-      const int idx = tid + it * kThreads, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
-      uq[it] = uk[it] = uv[it] = make_uint2(0u, 0u);
-      if (n < N) {
-        uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
-        uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
-        uv[it] = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
-      }
-    }
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) {
       const int idx = tid + it * kThreads, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
@@ -280,7 +282,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
     den += __shfl_xor_sync(0xffffffffu, den, 2);
     if (part == 0 && n < N) {
       for (int j = 0; j < sm.depth[n]; ++j) den += sm.A[j][n];
-      sm.den[n] = den;
+      sm.den[n] = 1.f / (den + eps);       // stored as the reciprocal
     }
   }
   __syncthreads();
@@ -333,7 +335,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         const int n = n0 + i;
-        if (n < N) o[base + (size_t)n * D + c] = __float2bfloat16_rn(__uint_as_float(acc[i]) / (sm.den[n] + eps) + conv[i]);
+        if (n < N) o[base + (size_t)n * D + c] = __float2bfloat16_rn(fmaf(__uint_as_float(acc[i]), sm.den[n], conv[i]));
       }
     }
   }
