@@ -1,15 +1,20 @@
-// Draft-tree verification on the tensor cores (bf16 io, d = 128, N <= 64).
+// Draft-tree verification on the tensor cores (bf16 io, d = 128, N <= 64, W <= 4).
 //
-// Sec. 4.2 / Sec. 5.3: all N draft nodes of a sequence share the committed state.  The shared part
-// of every node's numerator, phi(Q_tree) S, is one dense product; it is computed transposed,
-//     O^T[c][n] = sum_a S[a][c] phi(q_n)[a],
-// so that the fp32 state is the M x K operand exactly as it lies in memory: TMA brings the 128 x 128
-// fp32 tile of S into shared memory (128-byte swizzle in 32-byte chunks) and tcgen05.mma consumes it as tf32 -- S is read
-// from HBM once, without any conversion pass, while the CUDA cores prepare the tree.  The accumulator
-// (128 channels x 64 nodes, fp32) lives in TMEM; each thread then owns one channel, adds the
-// contributions of the node's ancestors and itself (tree mask), the unfolded convolution along the
-// ancestor chain, and divides by the node's denominator.  Nothing of the state is written.  CTAs are persistent:
-// while one warp group finishes a unit, another already prepares the next one.
+// Sec. 4.2 / Sec. 5.3: all N draft nodes of a sequence share the committed state and attend, among the draft
+// tokens, to their ancestors and themselves only.  Per (sequence, head) unit everything that is a contraction
+// runs as tcgen05.mma with the accumulators in TMEM:
+//     P[n][m]    = phi(q_n) . phi(k_m)                              (tf32; 64 x 64 scores)
+//     acc[c][n]  = sum_a S[a][c] phi(q_n)[a]                        (tf32; the fp32 state is the M x K operand exactly
+//                                                                    as it lies in memory, brought in by TMA)
+//     acc[c][n] += sum_m v_m[c] Pm[n][m]                            (bf16; Pm = P under the tree mask)
+//     G_j[c][n]  = sum_m v_m[c] Sel_j[n][m]                         (bf16; Sel_j has a single one per row, at the
+//                                                                    ancestor of n at distance j or at a row of the
+//                                                                    committed window: an exact gather of the value
+//                                                                    that tap j of the causal convolution reads)
+// and the CUDA cores are left with phi, the tree walk, the mask, the denominators and
+//     o[n][c] = acc[c][n] / (phi(q_n) . z + sum_m Pm[n][m] + eps) + sum_j w[j][c] G_j[c][n].
+// Nothing of the state is written.  CTAs are persistent: group X prepares unit t + 1 while group Y finishes
+// unit t, and one thread feeds TMA and the tensor cores.
 #include <cuda.h>
 
 #include <algorithm>
@@ -20,48 +25,44 @@ namespace la {
 namespace vtc {
 
 constexpr int D = 128, NMAX = LA_MAX_NODES;
-constexpr int kMaxTaps = 8;                        // longer tap windows are served by the CUDA-core kernel
+constexpr int kMaxTaps = 4;                        // longer tap windows are served by the CUDA-core kernel
 constexpr int kThreadsX = 256, kThreadsY = 256, kCtrlWarp = 16, kThreads = 544;
 constexpr uint32_t S_BOX = 128 * 128;              // 128 rows x 32 fp32
-constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 32 fp32
-constexpr uint32_t TMEM_COLS = 128;                // two accumulators of 64 columns
+constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 32 fp32 (also: 64 rows x 64 bf16)
+constexpr uint32_t V_BOX = (NMAX + 16) * 128;      // 64 draft rows + 16 window rows x 64 bf16
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t ACC_COL = 0, P_COL = 64, G_COL = 128;   // G_j at G_COL + 64 j
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
-// What the epilogue of one unit reads; two copies, so that the next unit is prepared while this one is finished.
-struct alignas(16) Buf {
-  float A[NMAX][NMAX];                             // A[j][n] = phi(q_n) . phi(k of the ancestor of n at distance j); 0 past the chain
-  float w[kMaxTaps][D];                            // taps of this unit's head
-  float rden[NMAX];                                // 1 / (denominator + eps) per node
-  __nv_bfloat16 vrows[NMAX + kMaxTaps - 1][D];     // rows 0..63 the draft values, rows 64.. the committed window
-  unsigned char anc[NMAX][NMAX];                   // anc[j][n] = row of vrows holding the value at distance j behind n
-  int max_depth;
-  int bad;
-  int pad[2];
-};
-// Scratch of the preparing group.
-struct alignas(16) Prep {
-  float fk[NMAX][D + 4];
-  float z[D];
-  int par[NMAX];
-  int depth[NMAX];
-  int pair_off[NMAX + 1];
-  int scan_carry;
-  unsigned char pair_n[NMAX * (NMAX + 1) / 2];
-  unsigned char pair_j[NMAX * (NMAX + 1) / 2];
+// Small tables.  Those that group X writes and group Y reads exist twice (unit parity).
+struct alignas(16) Tab {
+  unsigned long long mask[2][NMAX];                // bit m of mask[n]: m is n or an ancestor of n
+  float qz[2][NMAX];                               // phi(q_n) . z
+  int bad[2][2];                                   // per walking warp: a parent index was out of range
+  float den_part[2][NMAX];                         // masked row sums of P, one per column half
+  float rden[NMAX];                                // 1 / (denominator + eps)
+  int par[2][NMAX];                                // the parent array, one copy per walking warp
 };
 struct alignas(16) Ctl {
-  unsigned long long bars[8];
+  unsigned long long bars[12];
   uint32_t tmem_base;
   int abort;
 };
-// The per-unit barriers come in pairs indexed by t & 1 (phase t >> 1): a barrier is not completed again before
-// every waiter of its previous phase has passed, because the next completion depends on that waiter's own arrival.
-enum { B_FULL_S = 0, B_MMA0 = 1, B_MMA1 = 2, B_XDONE0 = 3, B_XDONE1 = 4, B_EPI0 = 5, B_EPI1 = 6, kNumBars = 7 };
-constexpr uint32_t OFF_S = 0, OFF_Q = 4 * S_BOX, OFF_PREP = OFF_Q + 4 * Q_BOX;
-constexpr uint32_t OFF_BUF = OFF_PREP + (uint32_t)sizeof(Prep);
-constexpr uint32_t OFF_CTL = OFF_BUF + 2 * (uint32_t)sizeof(Buf);
+// XDONE comes as a pair indexed by the unit parity (phase t >> 1); every other barrier completes once per unit
+// (phase t), and the protocol lets none complete again before the waiters of its previous phase have passed.
+enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_P, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
+constexpr uint32_t OFF_S = 0;                               // S: four boxes of 32 columns (fp32)
+constexpr uint32_t OFF_Q = OFF_S + 4 * S_BOX;               // phi(Q): four boxes of 32 columns (fp32 holding tf32)
+constexpr uint32_t OFF_K = OFF_Q + 4 * Q_BOX;               // phi(K): likewise
+constexpr uint32_t OFF_V = OFF_K + 4 * Q_BOX;               // V: two boxes of 64 channels, rows = nodes, then window
+constexpr uint32_t OFF_SEL = OFF_V + 2 * V_BOX;             // Sel_0 .. Sel_3 over the draft rows
+constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // columns 16 j + r: tap j reads window row r
+constexpr uint32_t OFF_PM = OFF_SELW + Q_BOX;               // masked scores, bf16
+constexpr uint32_t OFF_TAB = OFF_PM + Q_BOX;
+constexpr uint32_t OFF_CTL = OFF_TAB + (uint32_t)sizeof(Tab);
 constexpr uint32_t kSmemBytes = OFF_CTL + (uint32_t)sizeof(Ctl) + 1024;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(OFF_V % 1024 == 0 && V_BOX % 1024 == 0 && OFF_TAB % 16 == 0, "swizzled regions are 1024-byte aligned");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
@@ -95,6 +96,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
   }
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void sync_y() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // 128-byte swizzle: byte offset of 16-byte chunk `cc` of row `row` inside a box with 128-byte rows.
 __device__ __forceinline__ uint32_t swz(int row, int cc) { return (uint32_t)row * 128u + (uint32_t)((cc ^ (row & 7)) << 4); }
 // Shared-memory matrix descriptor; layout 2 = 128-byte swizzle in 16-byte chunks, 1 = 128-byte swizzle in 32-byte
@@ -103,37 +115,77 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
 }
-// Instruction descriptor: fp32 accumulate, tf32 x tf32, A with M contiguous (as S lies in memory), B with K
-// contiguous, M = 128, N = 64.
-constexpr uint32_t kIdesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptors (fp32 accumulate, M = 128, N = 64).  fmt: 1 = bf16, 2 = tf32; *_mn: the M (N) index is the
+// contiguous one of that operand.
+__host__ __device__ constexpr uint32_t idesc(uint32_t fmt, bool a_mn, bool b_mn) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((64u >> 3) << 17) |
+         ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void mma(uint32_t kind_tf32, uint32_t d, uint64_t a, uint64_t b, uint32_t id, bool accumulate) {
+  if (kind_tf32)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d), "l"(a), "l"(b), "r"(id),
+        "r"((uint32_t)accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d), "l"(a), "l"(b), "r"(id),
+        "r"((uint32_t)accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive TMEM columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
 
 template <int PHI> __device__ __forceinline__ float phi_f(float x) {
   if (PHI == LA_PHI_ELU1) return x > 0.f ? x + 1.f : __expf(x);
   return fmaxf(x, 0.f);
 }
-
-__device__ __forceinline__ void sync_x() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+// phi, rounded to the nearest tf32 so that the tensor core's truncation of the operand loses nothing more.
+template <int PHI> __device__ __forceinline__ float phi_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(phi_f<PHI>(x)));
+  return __uint_as_float(r);
+}
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Persistent kernel: CTA i handles units i, i + gridDim.x, ...  Three roles run concurrently:
-//   group X (warps 0-7)  prepares unit t: tree tables, phi(q) as the tf32 operand, phi(k), scores, denominators;
-//   warp 16 (one lane)   loads S of unit t by TMA and issues the tf32 product into TMEM accumulator t & 1;
-//   group Y (warps 8-15) finishes unit t: tree terms, unfolded convolution, division, store --
-// while group X already prepares unit t + 1 in the other copy of the per-unit tables.
+// Persistent kernel: CTA i handles units i, i + gridDim.x, ...  Roles:
+//   group X (warps 0-7)  unit t: loads q, k; walks the tree; writes phi(q), phi(k) as tf32 operands, the tree masks,
+//                        phi(q) . z, the selection matrices and the window rows;
+//   warp 16 (one lane)   TMA of S and V; every tcgen05.mma;
+//   group Y (warps 8-15) unit t: masks the scores, forms the denominators, and writes the outputs.
 template <int PHI>
 __global__ void __launch_bounds__(kThreads, 1)
-verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __restrict__ q,
-                 const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__ CUtensorMap mv,
+                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                  const int32_t* __restrict__ parent, const float* __restrict__ w, const float* __restrict__ z,
                  const __nv_bfloat16* __restrict__ win, __nv_bfloat16* __restrict__ o, int* status, int H, int N, int W,
                  float eps, int units) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
-  Prep& pr = *reinterpret_cast<Prep*>(smem + OFF_PREP);
-  Buf* bufs = reinterpret_cast<Buf*>(smem + OFF_BUF);
+  Tab& tab = *reinterpret_cast<Tab*>(smem + OFF_TAB);
   Ctl& ctl = *reinterpret_cast<Ctl*>(smem + OFF_CTL);
   volatile int* abort = &ctl.abort;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -142,31 +194,38 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
 #pragma unroll
   for (int i = 0; i < kNumBars; ++i) bar[i] = smem_u32(&ctl.bars[i]);
 
+  // ---- set-up: barriers, TMEM, the constant parts of the operands ----
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar[B_FULL_S]) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar[B_MMA0]) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar[B_MMA1]) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar[B_XDONE0]), "r"(kThreadsX) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar[B_XDONE1]), "r"(kThreadsX) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar[B_EPI0]), "r"(kThreadsY) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar[B_EPI1]), "r"(kThreadsY) : "memory");
+    mbar_init(bar[B_FULL_S], 1);
+    mbar_init(bar[B_FULL_V], 1);
+    mbar_init(bar[B_XDONE0], kThreadsX);
+    mbar_init(bar[B_XDONE1], kThreadsX);
+    mbar_init(bar[B_P], 1);
+    mbar_init(bar[B_SG], 1);
+    mbar_init(bar[B_PMDONE], kThreadsY);
+    mbar_init(bar[B_O], 1);
+    mbar_init(bar[B_EPI], kThreadsY);
     ctl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  // selection matrices and masked scores start as zeros; so do the 16 window rows below the draft rows of V
+  for (uint32_t i = tid; i < (OFF_TAB - OFF_SEL) / 16; i += kThreads)
+    *reinterpret_cast<uint4*>(smem + OFF_SEL + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+  for (uint32_t i = tid; i < 2 * 16 * 128 / 16; i += kThreads)
+    *reinterpret_cast<uint4*>(smem + OFF_V + (i >> 7) * V_BOX + NMAX * 128 + (i & 127) * 16) = make_uint4(0u, 0u, 0u, 0u);
   if (warp == kCtrlWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
                  "r"(TMEM_COLS)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  tc_fence_after();
   const uint32_t tmem = ctl.tmem_base;
 
   if (warp == kCtrlWarp) {
-    // =============================== TMA of S and the tf32 product (one lane) ===============================
+    // =============================== TMA and the tensor cores (one lane) ===============================
     if (lane == 0) {
       auto load_s = [&](int t) {   // the committed state of unit t: four boxes of 32 columns
         const int u = (int)blockIdx.x + t * (int)gridDim.x;
@@ -178,231 +237,262 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
               ::"r"(sbase + OFF_S + x * S_BOX), "l"(&ms), "r"(32 * x), "r"(u * D), "r"(bar[B_FULL_S])
               : "memory");
       };
-      if (nloc > 0) load_s(0);
-      for (int t = 0; t < nloc; ++t) {
-        const uint32_t par = t & 1, ph = (t >> 1) & 1;
-        if (!mbar_wait(bar[B_XDONE0 + par], ph, abort) || !mbar_wait(bar[B_FULL_S], par, abort)) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (!bufs[par].bad) {
+      auto load_v = [&](int t) {   // the draft values of unit t: two boxes of 64 channels x 64 nodes (rows past N: zeros)
+        const int u = (int)blockIdx.x + t * (int)gridDim.x;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar[B_FULL_V]), "r"(2 * Q_BOX) : "memory");
 #pragma unroll
-          for (int ks = 0; ks < 16; ++ks) {    // 8 values of the contraction index a per step
-            // S: 8 rows of a per step = two groups of 4 rows (512 B apart); the four 32-column boxes are S_BOX apart
-            const uint64_t adesc = smem_desc(sbase + OFF_S + ks * 1024u, S_BOX, 512u, 1u);
-            const uint64_t bdesc = smem_desc(sbase + OFF_Q + (ks >> 2) * Q_BOX + (ks & 3) * 32u, 16u, 1024u, 2u);
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "setp.ne.b32 p, %4, 0;\n\t"
-                "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-                ::"r"(tmem + par * 64u), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"((uint32_t)(ks > 0))
-                : "memory");
+        for (int x = 0; x < 2; ++x)
+          asm volatile(
+              "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+              ::"r"(sbase + OFF_V + x * V_BOX), "l"(&mv), "r"(64 * x), "r"(0), "r"(u), "r"(bar[B_FULL_V])
+              : "memory");
+      };
+      constexpr uint32_t kIdS = idesc(2, true, false), kIdP = idesc(2, false, false), kIdV = idesc(1, true, false);
+      load_s(0);
+      load_v(0);
+      for (int t = 0; t < nloc; ++t) {
+        const uint32_t par = t & 1;
+        if (!mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) || !mbar_wait(bar[B_FULL_S], par, abort)) break;
+        tc_fence_after();
+        const bool good = (tab.bad[par][0] | tab.bad[par][1]) == 0;
+        if (good) {
+#pragma unroll
+          for (int ks = 0; ks < 16; ++ks) {    // P[n][m]: 8 values of the feature index per step
+            const uint32_t off = (ks >> 2) * Q_BOX + (ks & 3) * 32u;
+            mma(1, tmem + P_COL, smem_desc(sbase + OFF_Q + off, 16u, 1024u, 2u), smem_desc(sbase + OFF_K + off, 16u, 1024u, 2u),
+                kIdP, ks > 0);
           }
         }
-        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar[B_MMA0 + par]) : "memory");
-        if (!mbar_wait(bar[B_MMA0 + par], ph, abort)) break;     // S and phi(Q) have been read
+        mma_commit(bar[B_P]);
+        if (t >= 1 && !mbar_wait(bar[B_EPI], (t - 1) & 1, abort)) break;   // the accumulators of unit t - 1 have been read
+        tc_fence_after();
+        if (good) {
+#pragma unroll
+          for (int ks = 0; ks < 16; ++ks)      // acc[c][n] = sum_a S[a][c] phi(q_n)[a]: 8 rows of S per step
+            mma(1, tmem + ACC_COL, smem_desc(sbase + OFF_S + ks * 1024u, S_BOX, 512u, 1u),
+                smem_desc(sbase + OFF_Q + (ks >> 2) * Q_BOX + (ks & 3) * 32u, 16u, 1024u, 2u), kIdS, ks > 0);
+        }
+        if (!mbar_wait(bar[B_FULL_V], par, abort)) break;
+        tc_fence_after();
+        if (good) {
+          for (int j = 0; j < W; ++j) {        // G_j[c][n]: the value tap j reads for node n
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)     // 16 draft rows per step
+              mma(0, tmem + G_COL + 64u * j, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
+                  smem_desc(sbase + OFF_SEL + j * Q_BOX + kk * 32u, 16u, 1024u, 2u), kIdV, kk > 0);
+            if (j > 0)                         // the window rows
+              mma(0, tmem + G_COL + 64u * j, smem_desc(sbase + OFF_V + NMAX * 128u, V_BOX, 1024u, 2u),
+                  smem_desc(sbase + OFF_SELW + j * 32u, 16u, 1024u, 2u), kIdV, true);
+          }
+        }
+        mma_commit(bar[B_SG]);
+        if (!mbar_wait(bar[B_SG], par, abort)) break;      // S, phi(Q), phi(K) and Sel have been read
         if (t + 1 < nloc) load_s(t + 1);
+        if (!mbar_wait(bar[B_PMDONE], par, abort)) break;
+        tc_fence_after();
+        if (good) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)       // acc[c][n] += sum_m v_m[c] Pm[n][m]
+            mma(0, tmem + ACC_COL, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
+                smem_desc(sbase + OFF_PM + kk * 32u, 16u, 1024u, 2u), kIdV, true);
+        }
+        mma_commit(bar[B_O]);
+        if (!mbar_wait(bar[B_O], par, abort)) break;       // V has been read
+        if (t + 1 < nloc) load_v(t + 1);
       }
     }
   } else if (warp < 8) {
     // =============================== group X: prepare unit t ===============================
+    if (tid < NMAX)                                         // Sel_0 is the identity: tap 0 reads the node's own value
+      *reinterpret_cast<unsigned short*>(smem + OFF_SEL + swz(tid, tid >> 3) + (tid & 7) * 2) = 0x3F80;
+    uint32_t prev1 = 0xffffffffu, prev2 = 0xffffffffu, prev3 = 0xffffffffu;   // where this node's ones of the last unit are
     bool ok = true;
     for (int t = 0; t < nloc; ++t) {
-      const int u = (int)blockIdx.x + t * (int)gridDim.x, b = u / H, h = u % H;
-      Buf& bf = bufs[t & 1];
-      // this copy of the tables was last read by the epilogue of unit t - 2
-      if (t >= 2) ok = ok && mbar_wait(bar[B_EPI0 + (t & 1)], ((t >> 1) - 1) & 1, abort);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { mbar_arrive(bar[B_XDONE0 + (t & 1)]); continue; }
-
-      // ---- q, k, v of the tree: all loads in flight before the tree is prepared ----
+      const int u = (int)blockIdx.x + t * (int)gridDim.x, b = u / H, par = t & 1;
+      // ---- everything this unit needs from memory is requested first ----
       const size_t base = (size_t)u * N * D;
-      constexpr int ITERS = NMAX * (D / 4) / kThreadsX;      // 8 chunks of 4 values per thread
-      uint2 uq[ITERS], uk[ITERS], uv[ITERS];
+      uint2 uq[8], uk[8];
 #pragma unroll
-      for (int it = 0; it < ITERS; ++it) {
-        const int idx = tid + it * kThreadsX, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
-        uq[it] = uk[it] = uv[it] = make_uint2(0u, 0u);
+      for (int it = 0; it < 8; ++it) {                      // row n = warp + 8 it, 4 features per lane
+        const int n = warp + 8 * it;
+        uq[it] = uk[it] = make_uint2(0u, 0u);
         if (n < N) {
-          uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + a4);
-          uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + a4);
-          uv[it] = *reinterpret_cast<const uint2*>(v + base + (size_t)n * D + a4);
+          uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + lane * 4);
+          uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + lane * 4);
         }
       }
+      const float4 z4 = *reinterpret_cast<const float4*>(z + (size_t)u * D + lane * 4);
+      uint32_t wv = 0u;
+      if (tid < 64 * (W - 1)) wv = *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * tid);
 
-      // ---- tree preparation: ancestor chains and depths (integer work) ----
-      if (tid < N) pr.par[tid] = parent[(size_t)b * N + tid];
-      for (int idx = tid; idx < NMAX * NMAX; idx += kThreadsX) (&bf.A[0][0])[idx] = 0.f;
-      if (tid == 0) { bf.max_depth = 0; bf.bad = 0; }
-      sync_x();
-      int my_dep = 0, my_off = 0;
-      if (tid < NMAX) {
+      // ---- tree walk: thread n follows the parents of node n (integer work, warps 0 and 1) ----
+      unsigned long long mask = 0ull;
+      int depth = 0, a1 = 0, a2 = 0, a3 = 0;
+      bool bad_any = false;
+      if (warp < 2) {
+        tab.par[warp][lane] = lane < N ? parent[(size_t)b * N + lane] : -1;
+        tab.par[warp][lane + 32] = lane + 32 < N ? parent[(size_t)b * N + lane + 32] : -1;
+        __syncwarp();
+        bool good = true;
         if (tid < N) {
           int m = tid;
-          bool good = true;
-          while (m >= 0) {                     // m strictly decreases: at most N iterations
-            bf.anc[my_dep++][tid] = (unsigned char)m;
-            const int p = pr.par[m];
+          while (m >= 0) {                                  // m strictly decreases: at most N iterations
+            mask |= 1ull << m;
+            if (depth == 1) a1 = m;
+            if (depth == 2) a2 = m;
+            if (depth == 3) a3 = m;
+            ++depth;
+            const int p = tab.par[warp][m];
             if (p < -1 || p >= m) { good = false; break; }
             m = p;
           }
-          if (!good) bf.bad = 1;
         }
-        int x = my_dep;                        // exclusive prefix of the depths over the two warps that hold the nodes
-#pragma unroll
-        for (int o2 = 1; o2 < 32; o2 <<= 1) {
-          const int y = __shfl_up_sync(0xffffffffu, x, o2);
-          if (lane >= o2) x += y;
-        }
-        my_off = x - my_dep;
-        if (tid == 31) pr.scan_carry = x;
-        atomicMax(&bf.max_depth, my_dep);
-        pr.depth[tid] = my_dep;
-      }
-      sync_x();
-      const bool bad = bf.bad != 0;
-      if (tid < NMAX && !bad) {
-        if (tid >= 32) my_off += pr.scan_carry;
-        pr.pair_off[tid] = my_off;
-        if (tid == NMAX - 1) pr.pair_off[NMAX] = my_off + my_dep;
-        const int jmax = max(bf.max_depth, W);
-        for (int j = 0; j < my_dep; ++j) {
-          pr.pair_n[my_off + j] = (unsigned char)tid;
-          pr.pair_j[my_off + j] = (unsigned char)j;
-        }
-        for (int j = my_dep; j < jmax; ++j)    // behind the chain: the committed window while taps remain, else a dummy row
-          bf.anc[j][tid] = (unsigned char)(tid < N && j < W ? NMAX + (W - 2) - (j - my_dep) : 0);
+        bad_any = __any_sync(0xffffffffu, !good);
+        __syncwarp();
       }
 
-      // ---- staging: phi(q) (fp32, swizzled: the B operand), phi(k), v, window, taps, z ----
-      if (t >= 1) ok = mbar_wait(bar[B_MMA0 + ((t - 1) & 1)], ((t - 1) >> 1) & 1, abort);   // the previous product has read phi(Q)
+      // ---- the operands of unit t - 1 have been consumed; this parity's tables were read two units ago ----
+      if (t >= 1) ok = ok && mbar_wait(bar[B_SG], (t - 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && !bad) {
+      if (ok) {
+        if (warp < 2) {
+          tab.mask[par][tid] = mask;
+          if (lane == 0) tab.bad[par][warp] = bad_any ? 1 : 0;
+          // one entry per (node, tap): clear the last unit's, set this unit's
+          auto place = [&](uint32_t& prev, int j, int anc) {
+            if (prev != 0xffffffffu) *reinterpret_cast<unsigned short*>(smem + prev) = 0;
+            prev = 0xffffffffu;
+            if (tid < N && j < W) {
+              if (j < depth) {
+                prev = OFF_SEL + j * Q_BOX + swz(tid, anc >> 3) + (anc & 7) * 2;
+              } else {                                      // behind the chain: the committed window, newest row last
+                const int col = 16 * j + (W - 2) - (j - depth);
+                prev = OFF_SELW + swz(tid, col >> 3) + (col & 7) * 2;
+              }
+              *reinterpret_cast<unsigned short*>(smem + prev) = 0x3F80;
+            }
+          };
+          place(prev1, 1, a1);
+          place(prev2, 2, a2);
+          place(prev3, 3, a3);
+        }
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-          const int idx = tid + it * kThreadsX, n = idx / (D / 4), a4 = (idx % (D / 4)) * 4;
+        for (int it = 0; it < 8; ++it) {
+          const int n = warp + 8 * it;
           float4 fq = make_float4(0.f, 0.f, 0.f, 0.f), fk = fq;
           if (n < N) {                                       // rows past N stay zero (phi(0) may be 1)
-            fq = make_float4(phi_f<PHI>(__uint_as_float(uq[it].x << 16)), phi_f<PHI>(__uint_as_float(uq[it].x & 0xffff0000u)),
-                             phi_f<PHI>(__uint_as_float(uq[it].y << 16)), phi_f<PHI>(__uint_as_float(uq[it].y & 0xffff0000u)));
-            fk = make_float4(phi_f<PHI>(__uint_as_float(uk[it].x << 16)), phi_f<PHI>(__uint_as_float(uk[it].x & 0xffff0000u)),
-                             phi_f<PHI>(__uint_as_float(uk[it].y << 16)), phi_f<PHI>(__uint_as_float(uk[it].y & 0xffff0000u)));
+            fq = make_float4(phi_tf32<PHI>(bf_lo(uq[it].x)), phi_tf32<PHI>(bf_hi(uq[it].x)), phi_tf32<PHI>(bf_lo(uq[it].y)),
+                             phi_tf32<PHI>(bf_hi(uq[it].y)));
+            fk = make_float4(phi_tf32<PHI>(bf_lo(uk[it].x)), phi_tf32<PHI>(bf_hi(uk[it].x)), phi_tf32<PHI>(bf_lo(uk[it].y)),
+                             phi_tf32<PHI>(bf_hi(uk[it].y)));
           }
-          *reinterpret_cast<float4*>(smem + OFF_Q + (a4 >> 5) * Q_BOX + swz(n, (a4 & 31) >> 2)) = fq;
-          *reinterpret_cast<float4*>(&pr.fk[n][a4]) = fk;
-          *reinterpret_cast<uint2*>(&bf.vrows[n][a4]) = uv[it];
-        }
-        for (int idx = tid; idx < W * D; idx += kThreadsX) bf.w[idx / D][idx % D] = w[((size_t)h * D + idx % D) * W + idx / D];
-        for (int idx = tid; idx < (W - 1) * D; idx += kThreadsX) bf.vrows[NMAX + idx / D][idx % D] = win[(size_t)u * (W - 1) * D + idx];
-        if (tid < D) pr.z[tid] = z[(size_t)u * D + tid];
-      }
-      sync_x();
-
-      // ---- scores of every (node, ancestor) pair, one pair per thread, then the denominators ----
-      if (ok && !bad) {
-        const int npairs = pr.pair_off[NMAX];
-        for (int pi = tid; pi < npairs; pi += kThreadsX) {
-          const int n = pr.pair_n[pi], j = pr.pair_j[pi], m = bf.anc[j][n];
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 8
-          for (int e = 0; e < D; e += 4) {
-            const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
-            const float4 y = *reinterpret_cast<const float4*>(&pr.fk[m][e]);
-            a0 = fmaf(x.x, y.x, a0);
-            a1 = fmaf(x.y, y.y, a1);
-            a2 = fmaf(x.z, y.z, a2);
-            a3 = fmaf(x.w, y.w, a3);
-          }
-          bf.A[j][n] = (a0 + a1) + (a2 + a3);
-        }
-      }
-      sync_x();
-      if (ok && !bad) {                         // four threads per node share the dot product with z (rows past N are zero)
-        const int n = tid >> 2, part = tid & 3;
-        float den = 0.f;
+          const uint32_t off = (lane >> 3) * Q_BOX + swz(n, lane & 7);
+          *reinterpret_cast<float4*>(smem + OFF_Q + off) = fq;
+          *reinterpret_cast<float4*>(smem + OFF_K + off) = fk;
+          float d = fmaf(fq.x, z4.x, fmaf(fq.y, z4.y, fmaf(fq.z, z4.z, fq.w * z4.w)));
 #pragma unroll
-        for (int e = 32 * part; e < 32 * part + 32; e += 4) {
-          const float4 x = *reinterpret_cast<const float4*>(smem + OFF_Q + (e >> 5) * Q_BOX + swz(n, (e & 31) >> 2));
-          den = fmaf(x.x, pr.z[e], den);
-          den = fmaf(x.y, pr.z[e + 1], den);
-          den = fmaf(x.z, pr.z[e + 2], den);
-          den = fmaf(x.w, pr.z[e + 3], den);
+          for (int s = 16; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
+          if (lane == 0) tab.qz[par][n] = d;
         }
-        den += __shfl_xor_sync(0xffffffffu, den, 1);
-        den += __shfl_xor_sync(0xffffffffu, den, 2);
-        if (part == 0 && n < N) {
-          for (int j = 0; j < pr.depth[n]; ++j) den += bf.A[j][n];
-          bf.rden[n] = 1.f / (den + eps);
+        if (tid < 64 * (W - 1)) {                            // window row r of both channel halves, below the draft rows
+          const int r = tid >> 6, c2 = (tid & 63) * 2;
+          *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + r, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv;
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(bar[B_XDONE0 + (t & 1)]);    // unit t is ready for the product and for the epilogue
+      proxy_fence();
+      mbar_arrive(bar[B_XDONE0 + par]);
     }
   } else {
-    // =============================== group Y: finish unit t (thread = channel c, 32 nodes per thread) ===============================
-    const int wy = warp - 8;
-    const int c = 32 * (wy & 3) + lane, n0 = 32 * (wy >> 2);
+    // =============================== group Y: finish unit t ===============================
+    const int ty = tid - kThreadsX, wy = warp - 8;
+    const int q4 = wy & 3;                                   // this warp reads TMEM lanes 32 q4 .. 32 q4 + 31
+    const int c = 32 * q4 + lane, n0 = 32 * (wy >> 2);       // epilogue: channel c, nodes n0 .. n0 + 31
     bool ok = true;
     for (int t = 0; t < nloc; ++t) {
-      const int u = (int)blockIdx.x + t * (int)gridDim.x;
-      const Buf& bf = bufs[t & 1];
-      ok = ok && mbar_wait(bar[B_XDONE0 + (t & 1)], (t >> 1) & 1, abort) && mbar_wait(bar[B_MMA0 + (t & 1)], (t >> 1) & 1, abort);
+      const int u = (int)blockIdx.x + t * (int)gridDim.x, h = u % H, par = t & 1;
+      float wt[kMaxTaps];                                    // taps of channel c
+#pragma unroll
+      for (int j = 0; j < kMaxTaps; ++j) wt[j] = j < W ? w[((size_t)h * D + c) * W + j] : 0.f;
+
+      ok = ok && mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) && mbar_wait(bar[B_P], par, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && bf.bad) {
-        if (tid == kThreadsX) report(status, LA_ERR_BAD_TREE);
-      } else if (ok && n0 < N) {               // warp-uniform
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const size_t base = (size_t)u * N * D;
-        uint32_t acc[32];
-        const uint32_t taddr = tmem + ((uint32_t)(32 * (wy & 3)) << 16) + (t & 1) * 64u + n0;
-        asm volatile(
-            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-            "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-            "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-            : "=r"(acc[0]), "=r"(acc[1]), "=r"(acc[2]), "=r"(acc[3]), "=r"(acc[4]), "=r"(acc[5]), "=r"(acc[6]),
-              "=r"(acc[7]), "=r"(acc[8]), "=r"(acc[9]), "=r"(acc[10]), "=r"(acc[11]), "=r"(acc[12]), "=r"(acc[13]),
-              "=r"(acc[14]), "=r"(acc[15]), "=r"(acc[16]), "=r"(acc[17]), "=r"(acc[18]), "=r"(acc[19]), "=r"(acc[20]),
-              "=r"(acc[21]), "=r"(acc[22]), "=r"(acc[23]), "=r"(acc[24]), "=r"(acc[25]), "=r"(acc[26]), "=r"(acc[27]),
-              "=r"(acc[28]), "=r"(acc[29]), "=r"(acc[30]), "=r"(acc[31])
-            : "r"(taddr)
-            : "memory");
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        // Walk the ancestor distance j in the outer loop: the value at distance j feeds both the tree term
-        // (weight A[j][n]) and tap j of the unfolded convolution; behind the chain the taps read the committed
-        // window.  Branch-free: weights are zero where a term does not apply.
-        float conv[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) conv[i] = 0.f;
-        const int jmax = max(bf.max_depth, W);
-        for (int j = 0; j < jmax; ++j) {
-          const float wj = j < W ? bf.w[j][c] : 0.f;
-#pragma unroll
-          for (int i = 0; i < 32; i += 4) {                  // four nodes per table load
-            const float4 a4 = *reinterpret_cast<const float4*>(&bf.A[j][n0 + i]);
-            const uint32_t r4 = *reinterpret_cast<const uint32_t*>(&bf.anc[j][n0 + i]);
-            const float u0 = __bfloat162float(bf.vrows[r4 & 0xff][c]), u1 = __bfloat162float(bf.vrows[(r4 >> 8) & 0xff][c]);
-            const float u2 = __bfloat162float(bf.vrows[(r4 >> 16) & 0xff][c]), u3 = __bfloat162float(bf.vrows[r4 >> 24][c]);
-            acc[i] = __float_as_uint(fmaf(a4.x, u0, __uint_as_float(acc[i])));
-            acc[i + 1] = __float_as_uint(fmaf(a4.y, u1, __uint_as_float(acc[i + 1])));
-            acc[i + 2] = __float_as_uint(fmaf(a4.z, u2, __uint_as_float(acc[i + 2])));
-            acc[i + 3] = __float_as_uint(fmaf(a4.w, u3, __uint_as_float(acc[i + 3])));
-            conv[i] = fmaf(wj, u0, conv[i]);
-            conv[i + 1] = fmaf(wj, u1, conv[i + 1]);
-            conv[i + 2] = fmaf(wj, u2, conv[i + 2]);
-            conv[i + 3] = fmaf(wj, u3, conv[i + 3]);
-          }
-        }
+      tc_fence_after();
+      const bool good = ok && (tab.bad[par][0] | tab.bad[par][1]) == 0;
+      // ---- scores under the tree mask: lane = node n, this warp's half of the columns m ----
+      if (good && q4 < 2) {
+        const int n = 32 * q4 + lane, hc = wy >> 2;
+        uint32_t p[32];
+        tmem_ld32(tmem + ((uint32_t)(32 * q4) << 16) + P_COL + 32u * hc, p);
+        const uint32_t bits = (uint32_t)(tab.mask[par][n] >> (32 * hc));
+        float sum = 0.f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
-          const int n = n0 + i;
-          if (n < N) o[base + (size_t)n * D + c] = __float2bfloat16_rn(fmaf(__uint_as_float(acc[i]), bf.rden[n], conv[i]));
+          const float x = (bits >> i) & 1u ? __uint_as_float(p[i]) : 0.f;
+          sum += x;
+          p[i] = __float_as_uint(x);
+        }
+        tab.den_part[hc][n] = sum;
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc)                       // 8 bf16 per 16-byte chunk of row n
+          *reinterpret_cast<uint4*>(smem + OFF_PM + swz(n, 4 * hc + cc)) =
+              make_uint4(pack2(__uint_as_float(p[8 * cc]), __uint_as_float(p[8 * cc + 1])),
+                         pack2(__uint_as_float(p[8 * cc + 2]), __uint_as_float(p[8 * cc + 3])),
+                         pack2(__uint_as_float(p[8 * cc + 4]), __uint_as_float(p[8 * cc + 5])),
+                         pack2(__uint_as_float(p[8 * cc + 6]), __uint_as_float(p[8 * cc + 7])));
+      }
+      tc_fence_before();
+      proxy_fence();
+      mbar_arrive(bar[B_PMDONE]);
+      sync_y();
+      if (ty < NMAX) tab.rden[ty] = 1.f / (tab.qz[par][ty] + tab.den_part[0][ty] + tab.den_part[1][ty] + eps);
+
+      ok = ok && mbar_wait(bar[B_O], par, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      tc_fence_after();
+      sync_y();
+      if (ok && !good) {
+        if (ty == 0) report(status, LA_ERR_BAD_TREE);
+      } else if (ok && n0 < N) {                             // warp-uniform
+        const uint32_t lane_base = tmem + ((uint32_t)(32 * q4) << 16) + n0;
+        uint32_t r[32];
+        float out[32];
+        tmem_ld32(lane_base + ACC_COL, r);
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+          const float4 rd = *reinterpret_cast<const float4*>(&tab.rden[n0 + i]);
+          out[i] = __uint_as_float(r[i]) * rd.x;
+          out[i + 1] = __uint_as_float(r[i + 1]) * rd.y;
+          out[i + 2] = __uint_as_float(r[i + 2]) * rd.z;
+          out[i + 3] = __uint_as_float(r[i + 3]) * rd.w;
+        }
+#pragma unroll
+        for (int j = 0; j < kMaxTaps; ++j) {
+          if (j < W) {
+            tmem_ld32(lane_base + G_COL + 64u * j, r);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) out[i] = fmaf(wt[j], __uint_as_float(r[i]), out[i]);
+          }
+        }
+        // Two neighbouring lanes trade values so that each stores two adjacent channels of one node: the even
+        // lane takes node n0 + i, the odd lane node n0 + i + 1.
+        const size_t obase = (size_t)u * N * D;
+        const int odd = lane & 1;
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          const float give = odd ? out[i] : out[i + 1];
+          const float got = __shfl_xor_sync(0xffffffffu, give, 1);
+          const int n = n0 + i + odd;
+          const uint32_t pair = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
+          if (n < N) *reinterpret_cast<uint32_t*>(o + obase + (size_t)n * D + (c - odd)) = pair;
         }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      mbar_arrive(bar[B_EPI0 + (t & 1)]);      // this copy of the tables and this accumulator may be reused
+      tc_fence_before();
+      mbar_arrive(bar[B_EPI]);
     }
   }
 
   // ---- teardown ----
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  tc_fence_before();
   __syncthreads();
   if (ctl.abort) {
     if (tid == 0) report(status, LA_ERR_TIMEOUT);
@@ -410,7 +500,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __nv_bfloat16* __
   }
   if (warp == kCtrlWarp) {
     __syncwarp();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
   }
 }
@@ -441,20 +531,33 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
   vtc::EncodeTiledFn fn = vtc::encode_fn();
   if (!fn) return cudaSuccess;
   const int BH = B * c.H;
+  const cuuint32_t es[3] = {1, 1, 1};
   CUtensorMap ms;   // S viewed as [BH * 128 rows, 128 columns] fp32; boxes of 32 columns x 128 rows
-  cuuint64_t dims[2] = {(cuuint64_t)vtc::D, (cuuint64_t)BH * vtc::D};
-  cuuint64_t strides[1] = {(cuuint64_t)vtc::D * 4};
-  cuuint32_t box[2] = {32, 128}, es[2] = {1, 1};
-  if (fn(&ms, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, st.S, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-         CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
-      CUDA_SUCCESS)
-    return cudaSuccess;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)vtc::D, (cuuint64_t)BH * vtc::D};
+    const cuuint64_t strides[1] = {(cuuint64_t)vtc::D * 4};
+    const cuuint32_t box[2] = {32, 128};
+    if (fn(&ms, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, st.S, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaSuccess;
+  }
+  CUtensorMap mv;   // V viewed as [BH][N][128] bf16; boxes of 64 channels x 64 nodes (nodes past N read as zeros)
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)vtc::D, (cuuint64_t)N, (cuuint64_t)BH};
+    const cuuint64_t strides[2] = {(cuuint64_t)vtc::D * 2, (cuuint64_t)N * vtc::D * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)vtc::NMAX, 1};
+    if (fn(&mv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(v), dims, strides, box, es,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return cudaSuccess;
+  }
   auto kern = c.phi == LA_PHI_ELU1 ? vtc::verify_tc_kernel<LA_PHI_ELU1> : vtc::verify_tc_kernel<LA_PHI_RELU>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vtc::kSmemBytes);
   if (e != cudaSuccess) return e;
   kern<<<dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), vtc::kSmemBytes, s>>>(
-      ms, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, parent, w, st.z,
-      (const __nv_bfloat16*)st.win, (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps, BH);
+      ms, mv, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, parent, w, st.z, (const __nv_bfloat16*)st.win,
+      (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps, BH);
   ctx->launches += 1;
   *handled = true;
   return cudaGetLastError();
