@@ -184,7 +184,9 @@ def tree_case(io, B, H, d, N, W, seed, phi="elu1", eps=0.0, chain=False):
     ("bf16", 128, 64, 3, "elu1", 0.0, False), ("bf16", 128, 37, 5, "relu", 1e-6, False),
     ("f32", 64, 4, 3, "elu1", 0.0, True), ("bf16", 64, 64, 3, "elu1", 0.0, False),
     ("bf16", 128, 1, 3, "elu1", 0.0, False), ("f32", 128, 64, 9, "elu1", 0.0, False),
-    ("bf16", 128, 20, 32, "elu1", 0.0, True), ("bf16", 128, 16, 1, "elu1", 0.0, False)])
+    ("bf16", 128, 20, 32, "elu1", 0.0, True), ("bf16", 128, 16, 1, "elu1", 0.0, False),
+    ("bf16", 128, 64, 4, "relu", 1e-6, True), ("bf16", 128, 37, 2, "relu", 1e-6, False),
+    ("bf16", 128, 50, 4, "elu1", 0.0, False), ("bf16", 128, 33, 4, "elu1", 1e-6, True)])
 @pytest.mark.parametrize("kernel", [0, 1])
 def test_verify_matches_oracle_and_leaves_state_untouched(kernel, io, d, N, W, phi, eps, chain):
     B, H = 3, 2
@@ -199,6 +201,28 @@ def test_verify_matches_oracle_and_leaves_state_untouched(kernel, io, d, N, W, p
     assert rel_err(host(o), want) < TOL[io]
     for a, b in ((st.S, before.S), (st.z, before.z), (st.win, before.win), (st.pos, before.pos)):
         assert torch.equal(a, b)
+
+
+def test_verify_more_units_than_sms_with_one_bad_tree():
+    """Several units per persistent CTA; one sequence in the middle carries an invalid tree."""
+    io, B, H, d, N, W = "bf16", 48, 8, 128, 64, 4
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=97, phi="relu", eps=1e-6)
+    ctx = binding.Context(H, d, W, "relu", 1e-6, io, max_nodes=64, max_depth=64)
+    st = oracle_state_to_dev(ost, io)
+    want = orc.verify_tree(q, k, v, parent, w, "relu", 1e-6, ost)
+    o = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    assert rel_err(host(o), want) < TOL[io]
+    for b in (0, 20, 47):                                  # per sequence, so that one wrong unit cannot hide
+        assert rel_err(host(o[b]), want[b]) < TOL[io]
+    bad = parent.copy()
+    bad[20, 9] = 9                                         # a node that is its own parent
+    out = torch.full((B, H, N, d), 123.0, dtype=torch.bfloat16, device="cuda")
+    ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(bad).cuda(), dev(w, "f32"), st, out=out)
+    assert ctx.la_last_device_status() == binding.LA_ERR_BAD_TREE
+    assert torch.all(out[20] == 123.0)
+    good = [b for b in range(B) if b != 20]
+    assert rel_err(host(out[good]), want[good]) < TOL[io]
 
 
 def test_verify_siblings_are_independent_bitwise():
