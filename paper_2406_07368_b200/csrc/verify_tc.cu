@@ -3,7 +3,7 @@
 // Sec. 4.2 / Sec. 5.3: all N draft nodes of a sequence share the committed state and attend, among the draft
 // tokens, to their ancestors and themselves only.  Per (sequence, head) unit everything that is a contraction
 // runs as tcgen05.mma with the accumulators in TMEM:
-//     P[n][m]    = phi(q_n) . phi(k_m)                              (tf32; 64 x 64 scores)
+//     P[n][m]    = phi(q_n) . phi(k_m)                              (bf16; 64 x 64 scores)
 //     acc[c][n]  = sum_a S[a][c] phi(q_n)[a]                        (tf32; the fp32 state is the M x K operand exactly
 //                                                                    as it lies in memory, brought in by TMA)
 //     acc[c][n] += sum_m v_m[c] Pm[n][m]                            (bf16; Pm = P under the tree mask)
@@ -50,11 +50,12 @@ struct alignas(16) Ctl {
 };
 // XDONE comes as a pair indexed by the unit parity (phase t >> 1); every other barrier completes once per unit
 // (phase t), and the protocol lets none complete again before the waiters of its previous phase have passed.
-enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_P, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
+enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_P, B_PS, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
 constexpr uint32_t OFF_S = 0;                               // S: four boxes of 32 columns (fp32)
-constexpr uint32_t OFF_Q = OFF_S + 4 * S_BOX;               // phi(Q): four boxes of 32 columns (fp32 holding tf32)
-constexpr uint32_t OFF_K = OFF_Q + 4 * Q_BOX;               // phi(K): likewise
-constexpr uint32_t OFF_V = OFF_K + 4 * Q_BOX;               // V: two boxes of 64 channels, rows = nodes, then window
+constexpr uint32_t OFF_Q = OFF_S + 4 * S_BOX;               // phi(Q) as fp32: four boxes of 32 features (tf32 operand)
+constexpr uint32_t OFF_QB = OFF_Q + 4 * Q_BOX;              // phi(Q) as bf16: two boxes of 64 features
+constexpr uint32_t OFF_KB = OFF_QB + 2 * Q_BOX;             // phi(K) as bf16: likewise
+constexpr uint32_t OFF_V = OFF_KB + 2 * Q_BOX;              // V: two boxes of 64 channels, rows = nodes, then window
 constexpr uint32_t OFF_SEL = OFF_V + 2 * V_BOX;             // Sel_0 .. Sel_3 over the draft rows
 constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // columns 16 j + r: tap j reads window row r
 constexpr uint32_t OFF_PM = OFF_SELW + Q_BOX;               // masked scores, bf16
@@ -153,15 +154,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-template <int PHI> __device__ __forceinline__ float phi_f(float x) {
-  if (PHI == LA_PHI_ELU1) return x > 0.f ? x + 1.f : __expf(x);
-  return fmaxf(x, 0.f);
-}
-// phi, rounded to the nearest tf32 so that the tensor core's truncation of the operand loses nothing more.
-template <int PHI> __device__ __forceinline__ float phi_tf32(float x) {
+// phi on two packed bf16 values, in packed arithmetic; the results are bf16 (and so exact as tf32 too).  elu + 1:
+// x + 1 where x > 0, 2^(x log2 e) elsewhere, merged with a lane mask.  ReLU: packed max.
+template <int PHI> __device__ __forceinline__ uint32_t phi2(uint32_t u) {
+  if (PHI == LA_PHI_ELU1) {
+    uint32_t y, e, xp1, mask;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(y) : "r"(u), "r"(0x3fb93fb9u));        // log2(e) in bf16
+    asm("ex2.approx.ftz.bf16x2 %0, %1;" : "=r"(e) : "r"(y));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(xp1) : "r"(u), "r"(0x3f803f80u));
+    asm("set.gt.u32.bf16x2 %0, %1, %2;" : "=r"(mask) : "r"(u), "r"(0u));
+    return (xp1 & mask) | (e & ~mask);
+  }
   uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(phi_f<PHI>(x)));
-  return __uint_as_float(r);
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(u), "r"(0u));
+  return r;
 }
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
@@ -201,6 +207,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
     mbar_init(bar[B_XDONE0], kThreadsX);
     mbar_init(bar[B_XDONE1], kThreadsX);
     mbar_init(bar[B_P], 1);
+    mbar_init(bar[B_PS], 1);
     mbar_init(bar[B_SG], 1);
     mbar_init(bar[B_PMDONE], kThreadsY);
     mbar_init(bar[B_O], 1);
@@ -247,7 +254,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
               ::"r"(sbase + OFF_V + x * V_BOX), "l"(&mv), "r"(64 * x), "r"(0), "r"(u), "r"(bar[B_FULL_V])
               : "memory");
       };
-      constexpr uint32_t kIdS = idesc(2, true, false), kIdP = idesc(2, false, false), kIdV = idesc(1, true, false);
+      constexpr uint32_t kIdS = idesc(2, true, false), kIdP = idesc(1, false, false), kIdV = idesc(1, true, false);
       load_s(0);
       load_v(0);
       for (int t = 0; t < nloc; ++t) {
@@ -257,9 +264,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         const bool good = (tab.bad[par][0] | tab.bad[par][1]) == 0;
         if (good) {
 #pragma unroll
-          for (int ks = 0; ks < 16; ++ks) {    // P[n][m]: 8 values of the feature index per step
+          for (int ks = 0; ks < 8; ++ks) {     // P[n][m]: 16 values of the feature index per step
             const uint32_t off = (ks >> 2) * Q_BOX + (ks & 3) * 32u;
-            mma(1, tmem + P_COL, smem_desc(sbase + OFF_Q + off, 16u, 1024u, 2u), smem_desc(sbase + OFF_K + off, 16u, 1024u, 2u),
+            mma(0, tmem + P_COL, smem_desc(sbase + OFF_QB + off, 16u, 1024u, 2u), smem_desc(sbase + OFF_KB + off, 16u, 1024u, 2u),
                 kIdP, ks > 0);
           }
         }
@@ -272,6 +279,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
             mma(1, tmem + ACC_COL, smem_desc(sbase + OFF_S + ks * 1024u, S_BOX, 512u, 1u),
                 smem_desc(sbase + OFF_Q + (ks >> 2) * Q_BOX + (ks & 3) * 32u, 16u, 1024u, 2u), kIdS, ks > 0);
         }
+        mma_commit(bar[B_PS]);
         if (!mbar_wait(bar[B_FULL_V], par, abort)) break;
         tc_fence_after();
         if (good) {
@@ -286,7 +294,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
           }
         }
         mma_commit(bar[B_SG]);
-        if (!mbar_wait(bar[B_SG], par, abort)) break;      // S, phi(Q), phi(K) and Sel have been read
+        if (!mbar_wait(bar[B_PS], par, abort)) break;      // S has been read
         if (t + 1 < nloc) load_s(t + 1);
         if (!mbar_wait(bar[B_PMDONE], par, abort)) break;
         tc_fence_after();
@@ -351,7 +359,51 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         __syncwarp();
       }
 
-      // ---- the operands of unit t - 1 have been consumed; this parity's tables were read two units ago ----
+      // ---- phi(Q), phi(K) of unit t - 1 have been consumed; this parity's tables were read two units ago ----
+      if (t >= 1) ok = ok && mbar_wait(bar[B_PS], (t - 1) & 1, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+        float part[8];                                       // this lane's share of phi(q_n) . z, n = warp + 8 it
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int n = warp + 8 * it;
+          uint2 pq = make_uint2(0u, 0u), pk = pq;            // rows past N stay zero (phi(0) may be 1)
+          if (n < N) {
+            pq = make_uint2(phi2<PHI>(uq[it].x), phi2<PHI>(uq[it].y));
+            pk = make_uint2(phi2<PHI>(uk[it].x), phi2<PHI>(uk[it].y));
+          }
+          const float4 fq = make_float4(bf_lo(pq.x), bf_hi(pq.x), bf_lo(pq.y), bf_hi(pq.y));
+          *reinterpret_cast<float4*>(smem + OFF_Q + (lane >> 3) * Q_BOX + swz(n, lane & 7)) = fq;
+          const uint32_t offb = (lane >> 4) * Q_BOX + swz(n, (lane & 15) >> 1) + (lane & 1) * 8;
+          *reinterpret_cast<uint2*>(smem + OFF_QB + offb) = pq;
+          *reinterpret_cast<uint2*>(smem + OFF_KB + offb) = pk;
+          part[it] = fmaf(fq.x, z4.x, fmaf(fq.y, z4.y, fmaf(fq.z, z4.z, fq.w * z4.w)));
+        }
+        // Sum over the lanes, eight rows at once: each exchange halves the rows a lane carries, so that after three of
+        // them lane l holds row (l >> 2) & 7 and two plain steps finish the sum.
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const bool up = lane & 16;
+          const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 4], 16);
+          part[i] = (up ? part[i + 4] : part[i]) + got;
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const bool up = lane & 8;
+          const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 2], 8);
+          part[i] = (up ? part[i + 2] : part[i]) + got;
+        }
+        {
+          const bool up = lane & 4;
+          const float got = __shfl_xor_sync(0xffffffffu, up ? part[0] : part[1], 4);
+          float d = (up ? part[1] : part[0]) + got;
+          d += __shfl_xor_sync(0xffffffffu, d, 2);
+          d += __shfl_xor_sync(0xffffffffu, d, 1);
+          if ((lane & 3) == 0) tab.qz[par][warp + 8 * ((lane >> 2) & 7)] = d;
+        }
+      }
+
+      // ---- the selection matrices and the window rows of unit t - 1 have been consumed ----
       if (t >= 1) ok = ok && mbar_wait(bar[B_SG], (t - 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
@@ -375,24 +427,6 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
           place(prev1, 1, a1);
           place(prev2, 2, a2);
           place(prev3, 3, a3);
-        }
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int n = warp + 8 * it;
-          float4 fq = make_float4(0.f, 0.f, 0.f, 0.f), fk = fq;
-          if (n < N) {                                       // rows past N stay zero (phi(0) may be 1)
-            fq = make_float4(phi_tf32<PHI>(bf_lo(uq[it].x)), phi_tf32<PHI>(bf_hi(uq[it].x)), phi_tf32<PHI>(bf_lo(uq[it].y)),
-                             phi_tf32<PHI>(bf_hi(uq[it].y)));
-            fk = make_float4(phi_tf32<PHI>(bf_lo(uk[it].x)), phi_tf32<PHI>(bf_hi(uk[it].x)), phi_tf32<PHI>(bf_lo(uk[it].y)),
-                             phi_tf32<PHI>(bf_hi(uk[it].y)));
-          }
-          const uint32_t off = (lane >> 3) * Q_BOX + swz(n, lane & 7);
-          *reinterpret_cast<float4*>(smem + OFF_Q + off) = fq;
-          *reinterpret_cast<float4*>(smem + OFF_K + off) = fk;
-          float d = fmaf(fq.x, z4.x, fmaf(fq.y, z4.y, fmaf(fq.z, z4.z, fq.w * z4.w)));
-#pragma unroll
-          for (int s = 16; s > 0; s >>= 1) d += __shfl_xor_sync(0xffffffffu, d, s);
-          if (lane == 0) tab.qz[par][n] = d;
         }
         if (tid < 64 * (W - 1)) {                            // window row r of both channel halves, below the draft rows
           const int r = tid >> 6, c2 = (tid & 63) * 2;
