@@ -4,8 +4,9 @@
 // tokens, to their ancestors and themselves only.  Per (sequence, head) unit everything that is a contraction
 // runs as tcgen05.mma with the accumulators in TMEM:
 //     P[n][m]    = phi(q_n) . phi(k_m)                              (bf16; 64 x 64 scores)
-//     acc[c][n]  = sum_a S[a][c] phi(q_n)[a]                        (tf32; the fp32 state is the M x K operand exactly
-//                                                                    as it lies in memory, brought in by TMA)
+//     acc[c][n]  = sum_a S[a][c] phi(q_n)[a]                        (bf16; TMA brings the fp32 state into shared
+//                                                                    memory, one warp group rounds it to bf16 in
+//                                                                    the operand layout)
 //     acc[c][n] += sum_m v_m[c] Pm[n][m]                            (bf16; Pm = P under the tree mask)
 //     G_j[c][n]  = sum_m v_m[c] Sel_j[n][m]                         (bf16; Sel_j has a single one per row, at the
 //                                                                    ancestor of n at distance j or at a row of the
@@ -18,6 +19,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <cstddef>
 
 #include "la_common.cuh"
 
@@ -26,22 +28,25 @@ namespace vtc {
 
 constexpr int D = 128, NMAX = LA_MAX_NODES;
 constexpr int kMaxTaps = 4;                        // longer tap windows are served by the CUDA-core kernel
-constexpr int kThreadsX = 256, kThreadsY = 256, kCtrlWarp = 16, kThreads = 544;
-constexpr uint32_t S_BOX = 128 * 128;              // 128 rows x 32 fp32
+constexpr int kThreadsX = 256, kThreadsY = 256, kCtrlWarp = 16, kTreeWarp = 17, kThreads = 576;
+constexpr uint32_t S_BYTES = 128 * 128 * 4;        // the fp32 state of one unit, row-major
+constexpr uint32_t SB_BOX = 128 * 128;             // 128 rows x 64 bf16
 constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 32 fp32 (also: 64 rows x 64 bf16)
 constexpr uint32_t V_BOX = (NMAX + 16) * 128;      // 64 draft rows + 16 window rows x 64 bf16
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t ACC_COL = 0, P_COL = 64, G_COL = 128;   // G_j at G_COL + 64 j
+constexpr uint32_t P_COL = 64, G_COL = 128;                // G_j at G_COL + 64 j
+__host__ __device__ constexpr uint32_t acc_col(int t) { return (t & 1) ? 384u : 0u; }   // acc of unit t
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // Small tables.  Those that group X writes and group Y reads exist twice (unit parity).
 struct alignas(16) Tab {
   unsigned long long mask[2][NMAX];                // bit m of mask[n]: m is n or an ancestor of n
   float qz[2][NMAX];                               // phi(q_n) . z
-  int bad[2][2];                                   // per walking warp: a parent index was out of range
+  int bad[2];                                      // a parent index was out of range
+  int pad0[2];
   float den_part[2][NMAX];                         // masked row sums of P, one per column half
   float rden[NMAX];                                // 1 / (denominator + eps)
-  int par[2][NMAX];                                // the parent array, one copy per walking warp
+  int par[NMAX];                                   // the parent array (private to the tree warp)
 };
 struct alignas(16) Ctl {
   unsigned long long bars[12];
@@ -50,19 +55,20 @@ struct alignas(16) Ctl {
 };
 // XDONE comes as a pair indexed by the unit parity (phase t >> 1); every other barrier completes once per unit
 // (phase t), and the protocol lets none complete again before the waiters of its previous phase have passed.
-enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_P, B_PS, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
-constexpr uint32_t OFF_S = 0;                               // S: four boxes of 32 columns (fp32)
-constexpr uint32_t OFF_Q = OFF_S + 4 * S_BOX;               // phi(Q) as fp32: four boxes of 32 features (tf32 operand)
-constexpr uint32_t OFF_QB = OFF_Q + 4 * Q_BOX;              // phi(Q) as bf16: two boxes of 64 features
+enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_SCONV, B_P, B_PS, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
+constexpr uint32_t OFF_S = 0;                               // S as it lies in memory (fp32, rows = features)
+constexpr uint32_t OFF_SB = OFF_S + S_BYTES;                // S as bf16: two boxes of 64 channels, rows = features
+constexpr uint32_t OFF_QB = OFF_SB + 2 * SB_BOX;            // phi(Q) as bf16: two boxes of 64 features
 constexpr uint32_t OFF_KB = OFF_QB + 2 * Q_BOX;             // phi(K) as bf16: likewise
 constexpr uint32_t OFF_V = OFF_KB + 2 * Q_BOX;              // V: two boxes of 64 channels, rows = nodes, then window
 constexpr uint32_t OFF_SEL = OFF_V + 2 * V_BOX;             // Sel_0 .. Sel_3 over the draft rows
-constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // columns 16 j + r: tap j reads window row r
+constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // row 64 j + n, column r: tap j of node n reads window row r
 constexpr uint32_t OFF_PM = OFF_SELW + Q_BOX;               // masked scores, bf16
 constexpr uint32_t OFF_TAB = OFF_PM + Q_BOX;
 constexpr uint32_t OFF_CTL = OFF_TAB + (uint32_t)sizeof(Tab);
 constexpr uint32_t kSmemBytes = OFF_CTL + (uint32_t)sizeof(Ctl) + 1024;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+static_assert(offsetof(Tab, rden) % 16 == 0, "rden is read four at a time");
 static_assert(OFF_V % 1024 == 0 && V_BOX % 1024 == 0 && OFF_TAB % 16 == 0, "swizzled regions are 1024-byte aligned");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -110,31 +116,28 @@ __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.
 
 // 128-byte swizzle: byte offset of 16-byte chunk `cc` of row `row` inside a box with 128-byte rows.
 __device__ __forceinline__ uint32_t swz(int row, int cc) { return (uint32_t)row * 128u + (uint32_t)((cc ^ (row & 7)) << 4); }
-// Shared-memory matrix descriptor; layout 2 = 128-byte swizzle in 16-byte chunks, 1 = 128-byte swizzle in 32-byte
-// chunks (the only layout the hardware takes for a 32-bit operand whose M or N index is the contiguous one).
+// Shared-memory matrix descriptor; layout 2 = 128-byte swizzle in 16-byte chunks, 0 = none (8 x 16-byte cores).
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
   return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
          ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout << 61);
 }
-// Instruction descriptors (fp32 accumulate, M = 128, N = 64).  fmt: 1 = bf16, 2 = tf32; *_mn: the M (N) index is the
-// contiguous one of that operand.
-__host__ __device__ constexpr uint32_t idesc(uint32_t fmt, bool a_mn, bool b_mn) {
-  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((64u >> 3) << 17) |
+// Instruction descriptor: bf16 x bf16 with fp32 accumulate, M = 128, N = n; *_mn: the M (N) index is the contiguous
+// one of that operand.
+__host__ __device__ constexpr uint32_t idesc(bool a_mn, bool b_mn, uint32_t n = 64u) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) | ((n >> 3) << 17) |
          ((128u >> 4) << 24);
 }
-__device__ __forceinline__ void mma(uint32_t kind_tf32, uint32_t d, uint64_t a, uint64_t b, uint32_t id, bool accumulate) {
-  if (kind_tf32)
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}" ::"r"(d), "l"(a), "l"(b), "r"(id),
-        "r"((uint32_t)accumulate)
-        : "memory");
-  else
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d), "l"(a), "l"(b), "r"(id),
-        "r"((uint32_t)accumulate)
-        : "memory");
+__device__ __forceinline__ void mma(uint32_t d, uint64_t a, uint64_t b, uint32_t id, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d), "l"(a), "l"(b), "r"(id),
+      "r"((uint32_t)accumulate)
+      : "memory");
+}
+// The window selectors: 256 rows (64 j + n) x 16 columns, no swizzle: cores of 8 rows x 8 columns (128 bytes), the two
+// cores of a row group side by side, row groups 256 bytes apart.
+__device__ __forceinline__ uint32_t selw_offset(int row, int col) {
+  return (uint32_t)(row >> 3) * 256u + (uint32_t)(col >> 3) * 128u + (uint32_t)(row & 7) * 16u + (uint32_t)(col & 7) * 2u;
 }
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -156,6 +159,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 
 // phi on two packed bf16 values, in packed arithmetic; the results are bf16 (and so exact as tf32 too).  elu + 1:
 // x + 1 where x > 0, 2^(x log2 e) elsewhere, merged with a lane mask.  ReLU: packed max.
+// 8 consecutive TMEM columns of this thread's lane; the caller waits once for all the loads it has issued.
+__device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 template <int PHI> __device__ __forceinline__ uint32_t phi2(uint32_t u) {
   if (PHI == LA_PHI_ELU1) {
     uint32_t y, e, xp1, mask;
@@ -177,10 +188,10 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 // Persistent kernel: CTA i handles units i, i + gridDim.x, ...  Roles:
-//   group X (warps 0-7)  unit t: loads q, k; walks the tree; writes phi(q), phi(k) as tf32 operands, the tree masks,
-//                        phi(q) . z, the selection matrices and the window rows;
+//   group X (warps 0-7)  unit t: phi(q), phi(k) as bf16 operands, phi(q) . z; rounds S to bf16;
+//   warp 17              unit t: walks the tree; writes the tree masks, the selection matrices and the window rows;
 //   warp 16 (one lane)   TMA of S and V; every tcgen05.mma;
-//   group Y (warps 8-15) unit t: masks the scores, forms the denominators, and writes the outputs.
+//   group Y (warps 8-15) masks the scores, forms the denominators, and writes the outputs.
 template <int PHI>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__ CUtensorMap mv,
@@ -204,8 +215,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
   if (tid == 0) {
     mbar_init(bar[B_FULL_S], 1);
     mbar_init(bar[B_FULL_V], 1);
-    mbar_init(bar[B_XDONE0], kThreadsX);
-    mbar_init(bar[B_XDONE1], kThreadsX);
+    mbar_init(bar[B_XDONE0], kThreadsX + 32);
+    mbar_init(bar[B_XDONE1], kThreadsX + 32);
+    mbar_init(bar[B_SCONV], kThreadsX);
     mbar_init(bar[B_P], 1);
     mbar_init(bar[B_PS], 1);
     mbar_init(bar[B_SG], 1);
@@ -234,15 +246,13 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
   if (warp == kCtrlWarp) {
     // =============================== TMA and the tensor cores (one lane) ===============================
     if (lane == 0) {
-      auto load_s = [&](int t) {   // the committed state of unit t: four boxes of 32 columns
+      auto load_s = [&](int t) {   // the committed state of unit t, 128 x 128 fp32 in one copy
         const int u = (int)blockIdx.x + t * (int)gridDim.x;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar[B_FULL_S]), "r"(4 * S_BOX) : "memory");
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-          asm volatile(
-              "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-              ::"r"(sbase + OFF_S + x * S_BOX), "l"(&ms), "r"(32 * x), "r"(u * D), "r"(bar[B_FULL_S])
-              : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar[B_FULL_S]), "r"(S_BYTES) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(sbase + OFF_S), "l"(&ms), "r"(0), "r"(u * D), "r"(bar[B_FULL_S])
+            : "memory");
       };
       auto load_v = [&](int t) {   // the draft values of unit t: two boxes of 64 channels x 64 nodes (rows past N: zeros)
         const int u = (int)blockIdx.x + t * (int)gridDim.x;
@@ -254,54 +264,56 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
               ::"r"(sbase + OFF_V + x * V_BOX), "l"(&mv), "r"(64 * x), "r"(0), "r"(u), "r"(bar[B_FULL_V])
               : "memory");
       };
-      constexpr uint32_t kIdS = idesc(2, true, false), kIdP = idesc(1, false, false), kIdV = idesc(1, true, false);
+      constexpr uint32_t kIdP = idesc(false, false), kIdV = idesc(true, false);
       load_s(0);
       load_v(0);
       for (int t = 0; t < nloc; ++t) {
         const uint32_t par = t & 1;
-        if (!mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) || !mbar_wait(bar[B_FULL_S], par, abort)) break;
+        if (!mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort)) break;
         tc_fence_after();
-        const bool good = (tab.bad[par][0] | tab.bad[par][1]) == 0;
+        const bool good = tab.bad[par] == 0;
         if (good) {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {     // P[n][m]: 16 values of the feature index per step
             const uint32_t off = (ks >> 2) * Q_BOX + (ks & 3) * 32u;
-            mma(0, tmem + P_COL, smem_desc(sbase + OFF_QB + off, 16u, 1024u, 2u), smem_desc(sbase + OFF_KB + off, 16u, 1024u, 2u),
+            mma(tmem + P_COL, smem_desc(sbase + OFF_QB + off, 16u, 1024u, 2u), smem_desc(sbase + OFF_KB + off, 16u, 1024u, 2u),
                 kIdP, ks > 0);
           }
         }
         mma_commit(bar[B_P]);
-        if (t >= 1 && !mbar_wait(bar[B_EPI], (t - 1) & 1, abort)) break;   // the accumulators of unit t - 1 have been read
+        if (!mbar_wait(bar[B_SCONV], par, abort)) break;   // the bf16 copy of S is in place, the fp32 one consumed
+        if (t + 1 < nloc) load_s(t + 1);
         tc_fence_after();
         if (good) {
 #pragma unroll
-          for (int ks = 0; ks < 16; ++ks)      // acc[c][n] = sum_a S[a][c] phi(q_n)[a]: 8 rows of S per step
-            mma(1, tmem + ACC_COL, smem_desc(sbase + OFF_S + ks * 1024u, S_BOX, 512u, 1u),
-                smem_desc(sbase + OFF_Q + (ks >> 2) * Q_BOX + (ks & 3) * 32u, 16u, 1024u, 2u), kIdS, ks > 0);
+          for (int kk = 0; kk < 8; ++kk)       // acc[c][n] = sum_a S[a][c] phi(q_n)[a]: 16 rows of S per step
+            mma(tmem + acc_col(t), smem_desc(sbase + OFF_SB + kk * 2048u, SB_BOX, 1024u, 2u),
+                smem_desc(sbase + OFF_QB + (kk >> 2) * Q_BOX + (kk & 3) * 32u, 16u, 1024u, 2u), kIdV, kk > 0);
         }
         mma_commit(bar[B_PS]);
+        // G of unit t - 1 has been read (this unit's accumulator was last read two units ago)
+        if (t >= 1 && !mbar_wait(bar[B_EPI], (t - 1) & 1, abort)) break;
         if (!mbar_wait(bar[B_FULL_V], par, abort)) break;
         tc_fence_after();
         if (good) {
-          for (int j = 0; j < W; ++j) {        // G_j[c][n]: the value tap j reads for node n
+          // G_j[c][n], the value tap j reads for node n, for all taps at once: the selection matrices lie one after
+          // the other, so they form one operand of 64 W rows and the products land in 64 W consecutive columns
+          const uint32_t idG = idesc(true, false, 64u * (uint32_t)W);
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)     // 16 draft rows per step
-              mma(0, tmem + G_COL + 64u * j, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
-                  smem_desc(sbase + OFF_SEL + j * Q_BOX + kk * 32u, 16u, 1024u, 2u), kIdV, kk > 0);
-            if (j > 0)                         // the window rows
-              mma(0, tmem + G_COL + 64u * j, smem_desc(sbase + OFF_V + NMAX * 128u, V_BOX, 1024u, 2u),
-                  smem_desc(sbase + OFF_SELW + j * 32u, 16u, 1024u, 2u), kIdV, true);
-          }
+          for (int kk = 0; kk < 4; ++kk)       // 16 draft rows per step
+            mma(tmem + G_COL, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
+                smem_desc(sbase + OFF_SEL + kk * 32u, 16u, 1024u, 2u), idG, kk > 0);
+          if (W > 1)                           // the window rows
+            mma(tmem + G_COL, smem_desc(sbase + OFF_V + NMAX * 128u, V_BOX, 1024u, 2u),
+                smem_desc(sbase + OFF_SELW, 128u, 256u, 0u), idG, true);
         }
         mma_commit(bar[B_SG]);
-        if (!mbar_wait(bar[B_PS], par, abort)) break;      // S has been read
-        if (t + 1 < nloc) load_s(t + 1);
         if (!mbar_wait(bar[B_PMDONE], par, abort)) break;
         tc_fence_after();
         if (good) {
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)       // acc[c][n] += sum_m v_m[c] Pm[n][m]
-            mma(0, tmem + ACC_COL, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
+            mma(tmem + acc_col(t), smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
                 smem_desc(sbase + OFF_PM + kk * 32u, 16u, 1024u, 2u), kIdV, true);
         }
         mma_commit(bar[B_O]);
@@ -309,134 +321,172 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         if (t + 1 < nloc) load_v(t + 1);
       }
     }
-  } else if (warp < 8) {
-    // =============================== group X: prepare unit t ===============================
-    if (tid < NMAX)                                         // Sel_0 is the identity: tap 0 reads the node's own value
-      *reinterpret_cast<unsigned short*>(smem + OFF_SEL + swz(tid, tid >> 3) + (tid & 7) * 2) = 0x3F80;
-    uint32_t prev1 = 0xffffffffu, prev2 = 0xffffffffu, prev3 = 0xffffffffu;   // where this node's ones of the last unit are
+  } else if (warp == kTreeWarp) {
+    // =============================== the tree of unit t (one warp, nodes lane and lane + 32) ===============================
+    for (int n = lane; n < NMAX; n += 32)                   // Sel_0 is the identity: tap 0 reads the node's own value
+      *reinterpret_cast<unsigned short*>(smem + OFF_SEL + swz(n, n >> 3) + (n & 7) * 2) = 0x3F80;
+    uint32_t prev[2][3];                                    // where the ones of this lane's nodes were put for the last unit
+#pragma unroll
+    for (int i = 0; i < 6; ++i) prev[i / 3][i % 3] = 0xffffffffu;
     bool ok = true;
     for (int t = 0; t < nloc; ++t) {
       const int u = (int)blockIdx.x + t * (int)gridDim.x, b = u / H, par = t & 1;
-      // ---- everything this unit needs from memory is requested first ----
-      const size_t base = (size_t)u * N * D;
-      uint2 uq[8], uk[8];
+      tab.par[lane] = lane < N ? parent[(size_t)b * N + lane] : -1;
+      tab.par[lane + 32] = lane + 32 < N ? parent[(size_t)b * N + lane + 32] : -1;
+      uint32_t wv[6];                                       // the committed window: (W - 1) rows of 128 channels
 #pragma unroll
-      for (int it = 0; it < 8; ++it) {                      // row n = warp + 8 it, 4 features per lane
-        const int n = warp + 8 * it;
-        uq[it] = uk[it] = make_uint2(0u, 0u);
-        if (n < N) {
-          uq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + lane * 4);
-          uk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + lane * 4);
-        }
+      for (int i = 0; i < 6; ++i) {
+        const int idx = lane + 32 * i;
+        wv[i] = idx < 64 * (W - 1) ? *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx) : 0u;
       }
-      const float4 z4 = *reinterpret_cast<const float4*>(z + (size_t)u * D + lane * 4);
-      uint32_t wv = 0u;
-      if (tid < 64 * (W - 1)) wv = *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * tid);
-
-      // ---- tree walk: thread n follows the parents of node n (integer work, warps 0 and 1) ----
-      unsigned long long mask = 0ull;
-      int depth = 0, a1 = 0, a2 = 0, a3 = 0;
-      bool bad_any = false;
-      if (warp < 2) {
-        tab.par[warp][lane] = lane < N ? parent[(size_t)b * N + lane] : -1;
-        tab.par[warp][lane + 32] = lane + 32 < N ? parent[(size_t)b * N + lane + 32] : -1;
-        __syncwarp();
-        bool good = true;
-        if (tid < N) {
-          int m = tid;
+      __syncwarp();
+      // ---- each lane follows the parents of its two nodes (integer work) ----
+      unsigned long long mask[2] = {0ull, 0ull};
+      int depth[2] = {0, 0}, anc[2][3] = {{0, 0, 0}, {0, 0, 0}};
+      bool good = true;
+#pragma unroll
+      for (int s2 = 0; s2 < 2; ++s2) {
+        const int n = lane + 32 * s2;
+        if (n < N) {
+          int m = n;
           while (m >= 0) {                                  // m strictly decreases: at most N iterations
-            mask |= 1ull << m;
-            if (depth == 1) a1 = m;
-            if (depth == 2) a2 = m;
-            if (depth == 3) a3 = m;
-            ++depth;
-            const int p = tab.par[warp][m];
+            mask[s2] |= 1ull << m;
+            if (depth[s2] == 1) anc[s2][0] = m;
+            if (depth[s2] == 2) anc[s2][1] = m;
+            if (depth[s2] == 3) anc[s2][2] = m;
+            ++depth[s2];
+            const int p = tab.par[m];
             if (p < -1 || p >= m) { good = false; break; }
             m = p;
           }
         }
-        bad_any = __any_sync(0xffffffffu, !good);
-        __syncwarp();
       }
+      const bool bad_any = __any_sync(0xffffffffu, !good);
+      __syncwarp();
 
-      // ---- phi(Q), phi(K) of unit t - 1 have been consumed; this parity's tables were read two units ago ----
-      if (t >= 1) ok = ok && mbar_wait(bar[B_PS], (t - 1) & 1, abort);
-      ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
-        float part[8];                                       // this lane's share of phi(q_n) . z, n = warp + 8 it
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int n = warp + 8 * it;
-          uint2 pq = make_uint2(0u, 0u), pk = pq;            // rows past N stay zero (phi(0) may be 1)
-          if (n < N) {
-            pq = make_uint2(phi2<PHI>(uq[it].x), phi2<PHI>(uq[it].y));
-            pk = make_uint2(phi2<PHI>(uk[it].x), phi2<PHI>(uk[it].y));
-          }
-          const float4 fq = make_float4(bf_lo(pq.x), bf_hi(pq.x), bf_lo(pq.y), bf_hi(pq.y));
-          *reinterpret_cast<float4*>(smem + OFF_Q + (lane >> 3) * Q_BOX + swz(n, lane & 7)) = fq;
-          const uint32_t offb = (lane >> 4) * Q_BOX + swz(n, (lane & 15) >> 1) + (lane & 1) * 8;
-          *reinterpret_cast<uint2*>(smem + OFF_QB + offb) = pq;
-          *reinterpret_cast<uint2*>(smem + OFF_KB + offb) = pk;
-          part[it] = fmaf(fq.x, z4.x, fmaf(fq.y, z4.y, fmaf(fq.z, z4.z, fq.w * z4.w)));
-        }
-        // Sum over the lanes, eight rows at once: each exchange halves the rows a lane carries, so that after three of
-        // them lane l holds row (l >> 2) & 7 and two plain steps finish the sum.
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const bool up = lane & 16;
-          const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 4], 16);
-          part[i] = (up ? part[i + 4] : part[i]) + got;
-        }
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const bool up = lane & 8;
-          const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 2], 8);
-          part[i] = (up ? part[i + 2] : part[i]) + got;
-        }
-        {
-          const bool up = lane & 4;
-          const float got = __shfl_xor_sync(0xffffffffu, up ? part[0] : part[1], 4);
-          float d = (up ? part[1] : part[0]) + got;
-          d += __shfl_xor_sync(0xffffffffu, d, 2);
-          d += __shfl_xor_sync(0xffffffffu, d, 1);
-          if ((lane & 3) == 0) tab.qz[par][warp + 8 * ((lane >> 2) & 7)] = d;
-        }
-      }
-
-      // ---- the selection matrices and the window rows of unit t - 1 have been consumed ----
+      // ---- the selection matrices and the window rows of unit t - 1 have been consumed (and with them everything
+      //      issued before: this parity's tables were last read two units ago) ----
       if (t >= 1) ok = ok && mbar_wait(bar[B_SG], (t - 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
-        if (warp < 2) {
-          tab.mask[par][tid] = mask;
-          if (lane == 0) tab.bad[par][warp] = bad_any ? 1 : 0;
-          // one entry per (node, tap): clear the last unit's, set this unit's
-          auto place = [&](uint32_t& prev, int j, int anc) {
-            if (prev != 0xffffffffu) *reinterpret_cast<unsigned short*>(smem + prev) = 0;
-            prev = 0xffffffffu;
-            if (tid < N && j < W) {
-              if (j < depth) {
-                prev = OFF_SEL + j * Q_BOX + swz(tid, anc >> 3) + (anc & 7) * 2;
+        if (lane == 0) tab.bad[par] = bad_any ? 1 : 0;
+#pragma unroll
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int n = lane + 32 * s2;
+          tab.mask[par][n] = mask[s2];
+#pragma unroll
+          for (int j = 1; j < kMaxTaps; ++j) {              // one entry per (node, tap): clear the last unit's, set this unit's
+            uint32_t& pv = prev[s2][j - 1];
+            if (pv != 0xffffffffu) *reinterpret_cast<unsigned short*>(smem + pv) = 0;
+            pv = 0xffffffffu;
+            if (n < N && j < W) {
+              if (j < depth[s2]) {
+                const int a = anc[s2][j - 1];
+                pv = OFF_SEL + j * Q_BOX + swz(n, a >> 3) + (a & 7) * 2;
               } else {                                      // behind the chain: the committed window, newest row last
-                const int col = 16 * j + (W - 2) - (j - depth);
-                prev = OFF_SELW + swz(tid, col >> 3) + (col & 7) * 2;
+                pv = OFF_SELW + selw_offset(64 * j + n, (W - 2) - (j - depth[s2]));
               }
-              *reinterpret_cast<unsigned short*>(smem + prev) = 0x3F80;
+              *reinterpret_cast<unsigned short*>(smem + pv) = 0x3F80;
             }
-          };
-          place(prev1, 1, a1);
-          place(prev2, 2, a2);
-          place(prev3, 3, a3);
+          }
         }
-        if (tid < 64 * (W - 1)) {                            // window row r of both channel halves, below the draft rows
-          const int r = tid >> 6, c2 = (tid & 63) * 2;
-          *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + r, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv;
+#pragma unroll
+        for (int i = 0; i < 6; ++i) {                        // window row r of both channel halves, below the draft rows
+          const int idx = lane + 32 * i, r = idx >> 6, c2 = (idx & 63) * 2;
+          if (idx < 64 * (W - 1))
+            *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + r, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv[i];
         }
       }
       proxy_fence();
       mbar_arrive(bar[B_XDONE0 + par]);
     }
-  } else {
+  } else if (warp < 8) {
+    // =============================== group X: phi(q), phi(k) and the bf16 copy of S of unit t ===============================
+    bool ok = true;
+    uint2 pq[8], pk[8];
+    float4 z4;
+    auto load_qk = [&](int t2) {                            // row n = warp + 8 it, 4 features per lane
+      const int u = (int)blockIdx.x + t2 * (int)gridDim.x;
+      const size_t base = (size_t)u * N * D;
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int n = warp + 8 * it;
+        pq[it] = pk[it] = make_uint2(0u, 0u);
+        if (n < N) {
+          pq[it] = *reinterpret_cast<const uint2*>(q + base + (size_t)n * D + lane * 4);
+          pk[it] = *reinterpret_cast<const uint2*>(k + base + (size_t)n * D + lane * 4);
+        }
+      }
+      z4 = *reinterpret_cast<const float4*>(z + (size_t)u * D + lane * 4);
+    };
+    load_qk(0);
+    for (int t = 0; t < nloc; ++t) {
+      const int par = t & 1;
+      // ---- everything that needs no shared memory happens while the tensor cores still read unit t - 1 ----
+      float part[8];                                         // this lane's share of phi(q_n) . z, n = warp + 8 it
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        if (warp + 8 * it < N) {                             // rows past N stay zero (phi(0) may be 1)
+          pq[it] = make_uint2(phi2<PHI>(pq[it].x), phi2<PHI>(pq[it].y));
+          pk[it] = make_uint2(phi2<PHI>(pk[it].x), phi2<PHI>(pk[it].y));
+        }
+        part[it] = fmaf(bf_lo(pq[it].x), z4.x, fmaf(bf_hi(pq[it].x), z4.y, fmaf(bf_lo(pq[it].y), z4.z, bf_hi(pq[it].y) * z4.w)));
+      }
+      // Sum over the lanes, eight rows at once: each exchange halves the rows a lane carries, so that after three of
+      // them lane l holds row (l >> 2) & 7 and two plain steps finish the sum.
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const bool up = lane & 16;
+        const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 4], 16);
+        part[i] = (up ? part[i + 4] : part[i]) + got;
+      }
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const bool up = lane & 8;
+        const float got = __shfl_xor_sync(0xffffffffu, up ? part[i] : part[i + 2], 8);
+        part[i] = (up ? part[i + 2] : part[i]) + got;
+      }
+      float qz;
+      {
+        const bool up = lane & 4;
+        const float got = __shfl_xor_sync(0xffffffffu, up ? part[0] : part[1], 4);
+        qz = (up ? part[1] : part[0]) + got;
+        qz += __shfl_xor_sync(0xffffffffu, qz, 2);
+        qz += __shfl_xor_sync(0xffffffffu, qz, 1);
+      }
+
+      // ---- phi(Q), phi(K) and the bf16 copy of S of unit t - 1 have been consumed ----
+      if (t >= 1) ok = ok && mbar_wait(bar[B_PS], (t - 1) & 1, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const uint32_t offb = (lane >> 4) * Q_BOX + swz(warp + 8 * it, (lane & 15) >> 1) + (lane & 1) * 8;
+          *reinterpret_cast<uint2*>(smem + OFF_QB + offb) = pq[it];
+          *reinterpret_cast<uint2*>(smem + OFF_KB + offb) = pk[it];
+        }
+        if ((lane & 3) == 0) tab.qz[par][warp + 8 * ((lane >> 2) & 7)] = qz;
+      }
+      proxy_fence();
+      mbar_arrive(bar[B_XDONE0 + par]);
+      if (t + 1 < nloc) load_qk(t + 1);                      // in flight during the conversion below
+
+      // ---- S of unit t has landed: round it to bf16 in the operand layout (rows = features, channels contiguous) ----
+      ok = ok && mbar_wait(bar[B_FULL_S], par, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok) {
+#pragma unroll 8
+        for (int it = 0; it < 16; ++it) {
+          const int a = warp + 8 * it;                         // row a, channels 4 lane .. 4 lane + 3
+          const float4 s4 = *reinterpret_cast<const float4*>(smem + OFF_S + a * 512 + lane * 16);
+          *reinterpret_cast<uint2*>(smem + OFF_SB + (lane >> 4) * SB_BOX + swz(a, (lane & 15) >> 1) + (lane & 1) * 8) =
+              make_uint2(pack2(s4.x, s4.y), pack2(s4.z, s4.w));
+        }
+      }
+      proxy_fence();
+      mbar_arrive(bar[B_SCONV]);
+    }
+  } else if (warp < 16) {
     // =============================== group Y: finish unit t ===============================
     const int ty = tid - kThreadsX, wy = warp - 8;
     const int q4 = wy & 3;                                   // this warp reads TMEM lanes 32 q4 .. 32 q4 + 31
@@ -446,12 +496,12 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       const int u = (int)blockIdx.x + t * (int)gridDim.x, h = u % H, par = t & 1;
       float wt[kMaxTaps];                                    // taps of channel c
 #pragma unroll
-      for (int j = 0; j < kMaxTaps; ++j) wt[j] = j < W ? w[((size_t)h * D + c) * W + j] : 0.f;
+      for (int j = 0; j < kMaxTaps; ++j) wt[j] = w[((size_t)h * D + c) * W + min(j, W - 1)];   // used where j < W
 
       ok = ok && mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) && mbar_wait(bar[B_P], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
-      const bool good = ok && (tab.bad[par][0] | tab.bad[par][1]) == 0;
+      const bool good = ok && tab.bad[par] == 0;
       // ---- scores under the tree mask: lane = node n, this warp's half of the columns m ----
       if (good && q4 < 2) {
         const int n = 32 * q4 + lane, hc = wy >> 2;
@@ -465,7 +515,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
           sum += x;
           p[i] = __float_as_uint(x);
         }
-        tab.den_part[hc][n] = sum;
+        tab.den_part[hc][n] = hc == 0 ? sum + tab.qz[par][n] : sum;   // phi(q_n) . z joins the first half
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc)                       // 8 bf16 per 16-byte chunk of row n
           *reinterpret_cast<uint4*>(smem + OFF_PM + swz(n, 4 * hc + cc)) =
@@ -478,7 +528,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       proxy_fence();
       mbar_arrive(bar[B_PMDONE]);
       sync_y();
-      if (ty < NMAX) tab.rden[ty] = 1.f / (tab.qz[par][ty] + tab.den_part[0][ty] + tab.den_part[1][ty] + eps);
+      if (ty < NMAX) tab.rden[ty] = 1.f / (tab.den_part[0][ty] + tab.den_part[1][ty] + eps);
 
       ok = ok && mbar_wait(bar[B_O], par, abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -488,36 +538,42 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         if (ty == 0) report(status, LA_ERR_BAD_TREE);
       } else if (ok && n0 < N) {                             // warp-uniform
         const uint32_t lane_base = tmem + ((uint32_t)(32 * q4) << 16) + n0;
-        uint32_t r[32];
-        float out[32];
-        tmem_ld32(lane_base + ACC_COL, r);
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-          const float4 rd = *reinterpret_cast<const float4*>(&tab.rden[n0 + i]);
-          out[i] = __uint_as_float(r[i]) * rd.x;
-          out[i + 1] = __uint_as_float(r[i + 1]) * rd.y;
-          out[i + 2] = __uint_as_float(r[i + 2]) * rd.z;
-          out[i + 3] = __uint_as_float(r[i + 3]) * rd.w;
-        }
-#pragma unroll
-        for (int j = 0; j < kMaxTaps; ++j) {
-          if (j < W) {
-            tmem_ld32(lane_base + G_COL + 64u * j, r);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) out[i] = fmaf(wt[j], __uint_as_float(r[i]), out[i]);
-          }
-        }
-        // Two neighbouring lanes trade values so that each stores two adjacent channels of one node: the even
-        // lane takes node n0 + i, the odd lane node n0 + i + 1.
         const size_t obase = (size_t)u * N * D;
         const int odd = lane & 1;
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float give = odd ? out[i] : out[i + 1];
-          const float got = __shfl_xor_sync(0xffffffffu, give, 1);
-          const int n = n0 + i + odd;
-          const uint32_t pair = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
-          if (n < N) *reinterpret_cast<uint32_t*>(o + obase + (size_t)n * D + (c - odd)) = pair;
+        for (int part = 0; part < 4; ++part) {               // 8 nodes at a time, all their TMEM loads in flight at once
+          const int nb = n0 + 8 * part;
+          uint32_t ra[8], rg[kMaxTaps][8];
+          tmem_ld8_issue(lane_base + acc_col(t) + 8u * part, ra);
+#pragma unroll
+          for (int j = 0; j < kMaxTaps; ++j)
+            if (j < W) tmem_ld8_issue(lane_base + G_COL + 64u * j + 8u * part, rg[j]);
+          tmem_ld_wait();
+          float out[8];
+#pragma unroll
+          for (int i = 0; i < 8; i += 4) {
+            const float4 rd = *reinterpret_cast<const float4*>(&tab.rden[nb + i]);
+            out[i] = __uint_as_float(ra[i]) * rd.x;
+            out[i + 1] = __uint_as_float(ra[i + 1]) * rd.y;
+            out[i + 2] = __uint_as_float(ra[i + 2]) * rd.z;
+            out[i + 3] = __uint_as_float(ra[i + 3]) * rd.w;
+          }
+#pragma unroll
+          for (int j = 0; j < kMaxTaps; ++j)
+            if (j < W) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) out[i] = fmaf(wt[j], __uint_as_float(rg[j][i]), out[i]);
+            }
+          // Two neighbouring lanes trade values so that each stores two adjacent channels of one node: the even
+          // lane takes node nb + i, the odd lane node nb + i + 1.
+#pragma unroll
+          for (int i = 0; i < 8; i += 2) {
+            const float give = odd ? out[i] : out[i + 1];
+            const float got = __shfl_xor_sync(0xffffffffu, give, 1);
+            const int n = nb + i + odd;
+            const uint32_t pair = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
+            if (n < N) *reinterpret_cast<uint32_t*>(o + obase + (size_t)n * D + (c - odd)) = pair;
+          }
         }
       }
       tc_fence_before();
@@ -566,13 +622,13 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
   if (!fn) return cudaSuccess;
   const int BH = B * c.H;
   const cuuint32_t es[3] = {1, 1, 1};
-  CUtensorMap ms;   // S viewed as [BH * 128 rows, 128 columns] fp32; boxes of 32 columns x 128 rows
+  CUtensorMap ms;   // S viewed as [BH * 128 rows, 128 columns] fp32; one unit per box, no swizzle
   {
     const cuuint64_t dims[2] = {(cuuint64_t)vtc::D, (cuuint64_t)BH * vtc::D};
     const cuuint64_t strides[1] = {(cuuint64_t)vtc::D * 4};
-    const cuuint32_t box[2] = {32, 128};
+    const cuuint32_t box[2] = {128, 128};
     if (fn(&ms, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, st.S, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-           CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaSuccess;
   }
