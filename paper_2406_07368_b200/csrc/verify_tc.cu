@@ -534,12 +534,10 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
       sync_y();
-      if (ok && !good) {
-        if (ty == 0) report(status, LA_ERR_BAD_TREE);
-      } else if (ok && n0 < N) {                             // warp-uniform
+      if (good && n0 < N) {                                  // warp-uniform (good implies ok)
         const uint32_t lane_base = tmem + ((uint32_t)(32 * q4) << 16) + n0;
-        const size_t obase = (size_t)u * N * D;
         const int odd = lane & 1;
+        uint32_t pairs[16];                                  // two adjacent channels of node n0 + 2 i + odd
 #pragma unroll
         for (int part = 0; part < 4; ++part) {               // 8 nodes at a time, all their TMEM loads in flight at once
           const int nb = n0 + 8 * part;
@@ -570,14 +568,21 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
           for (int i = 0; i < 8; i += 2) {
             const float give = odd ? out[i] : out[i + 1];
             const float got = __shfl_xor_sync(0xffffffffu, give, 1);
-            const int n = nb + i + odd;
-            const uint32_t pair = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
-            if (n < N) *reinterpret_cast<uint32_t*>(o + obase + (size_t)n * D + (c - odd)) = pair;
+            pairs[4 * part + i / 2] = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
           }
         }
+        // the accumulators are free again before the outputs leave: the barrier's release would wait for the stores
+        tc_fence_before();
+        mbar_arrive(bar[B_EPI]);
+        __nv_bfloat16* orow = o + ((size_t)u * N + n0 + odd) * D + (c - odd);
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          if (n0 + 2 * i + odd < N) *reinterpret_cast<uint32_t*>(orow + (size_t)(2 * i) * D) = pairs[i];
+      } else {
+        if (ok && !good && ty == 0) report(status, LA_ERR_BAD_TREE);
+        tc_fence_before();
+        mbar_arrive(bar[B_EPI]);
       }
-      tc_fence_before();
-      mbar_arrive(bar[B_EPI]);
     }
   }
 
