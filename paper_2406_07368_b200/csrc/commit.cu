@@ -1,14 +1,20 @@
 // Commit of the accepted draft path (Sec. 4.2: later tokens interact with the verified
-// tokens of earlier groups).  One CTA per (sequence, head): rebuild the root-to-node path from
+// tokens of earlier groups).  Per (sequence, head): rebuild the root-to-node path from
 // the parent array (integer work, bit-exact), then stream the d x d state once, adding the
 // rank-1 updates of all path tokens in order, and advance z, the convolution window and pos.
+// The loads of the state are issued first, so that they are in flight while the path is rebuilt and the path
+// tokens are gathered.
 #include "la_common.cuh"
 
 namespace la {
 
-template <int D> struct CommitSmem {
-  float fk[LA_MAX_NODES][D];
-  float v[LA_MAX_NODES][D];
+// The d x d state of one (sequence, head) unit is shared out among kCommitSplit CTAs (a band of rows each), so that
+// a launch of few units still spreads evenly over the SMs; the first of them also advances z and the window.
+constexpr int kCommitSplit = 4;
+
+// Shared memory: phi(k) and v of the path tokens (max_depth rows each), then the integer tables.
+struct CommitTables {
+  int par[LA_MAX_NODES];
   int path[LA_MAX_NODES];
   int len;
   int bad;
@@ -20,11 +26,22 @@ commit_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* _
               const int32_t* __restrict__ accept, float* __restrict__ S, float* __restrict__ z, T* __restrict__ win,
               int64_t* __restrict__ pos, int32_t* __restrict__ path_out, int32_t* __restrict__ commit_len, int* status,
               int H, int N, int W, int max_depth) {
-  constexpr int TPR = D / 4, RPP = 256 / TPR, PASSES = D / RPP;
+  constexpr int TPR = D / 4, RPP = 256 / TPR, ROWS = D / kCommitSplit, PASSES = ROWS / RPP;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  CommitSmem<D>& sm = *reinterpret_cast<CommitSmem<D>*>(smem_raw);
-  const int bh = blockIdx.x, b = bh / H, h = bh % H, t = threadIdx.x;
+  float (*fk)[D] = reinterpret_cast<float (*)[D]>(smem_raw);
+  float (*vv)[D] = fk + max_depth;
+  CommitTables& sm = *reinterpret_cast<CommitTables*>(vv + max_depth);
+  const int bh = blockIdx.x / kCommitSplit, part = blockIdx.x % kCommitSplit, b = bh / H, h = bh % H, t = threadIdx.x;
 
+  // The state is requested before anything else: the loads are in flight while the path is rebuilt.
+  const int c4 = (t % TPR) * 4, rg = part * ROWS + t / TPR;   // this CTA's rows of S: part * ROWS .. + ROWS - 1
+  float* Sb = S + (size_t)bh * D * D;
+  float4 s[PASSES];
+#pragma unroll
+  for (int m = 0; m < PASSES; ++m) s[m] = __ldcs(reinterpret_cast<const float4*>(Sb + (size_t)(rg + RPP * m) * D + c4));
+
+  if (t < N) sm.par[t] = parent[(size_t)b * N + t];
+  __syncthreads();
   if (t == 0) {
     int a = accept[b], L = 0, bad = 0;
     if (a < -1 || a >= N) bad = 1;
@@ -32,7 +49,7 @@ commit_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* _
     while (m >= 0) {                       // m strictly decreases: terminates
       if (L >= max_depth) { bad = 1; break; }
       sm.path[L++] = m;
-      const int p = parent[(size_t)b * N + m];
+      const int p = sm.par[m];
       if (p < -1 || p >= m) { bad = 1; break; }
       m = p;
     }
@@ -50,32 +67,26 @@ commit_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* _
     return;
   }
   const int L = sm.len;
-  if (h == 0) {
+  if (h == 0 && part == 0) {
     for (int i = t; i < max_depth; i += 256) path_out[(size_t)b * max_depth + i] = i < L ? sm.path[i] : -1;
     if (t == 0) commit_len[b] = L;
   }
   if (L == 0) return;
 
-  const int c4 = (t % TPR) * 4, rg = t / TPR;
-  float* Sb = S + (size_t)bh * D * D;
-  float4 s[PASSES];
-#pragma unroll
-  for (int m = 0; m < PASSES; ++m) s[m] = __ldcs(reinterpret_cast<const float4*>(Sb + (size_t)(rg + RPP * m) * D + c4));
-
   const size_t base = (size_t)bh * N * D;
   for (int idx = t; idx < L * D; idx += 256) {
     const int l = idx / D, e = idx % D;
     const size_t g = base + (size_t)sm.path[l] * D + e;
-    sm.fk[l][e] = phi<PHI>(to_f32(k[g]));
-    sm.v[l][e] = to_f32(v[g]);
+    fk[l][e] = phi<PHI>(to_f32(k[g]));
+    vv[l][e] = to_f32(v[g]);
   }
   __syncthreads();
 
   for (int l = 0; l < L; ++l) {
-    const float4 v4 = *reinterpret_cast<const float4*>(&sm.v[l][c4]);
+    const float4 v4 = *reinterpret_cast<const float4*>(&vv[l][c4]);
 #pragma unroll
     for (int m = 0; m < PASSES; ++m) {
-      const float a = sm.fk[l][rg + RPP * m];
+      const float a = fk[l][rg + RPP * m];
       s[m].x = fmaf(a, v4.x, s[m].x);
       s[m].y = fmaf(a, v4.y, s[m].y);
       s[m].z = fmaf(a, v4.z, s[m].z);
@@ -85,18 +96,18 @@ commit_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* _
 #pragma unroll
   for (int m = 0; m < PASSES; ++m) __stcs(reinterpret_cast<float4*>(Sb + (size_t)(rg + RPP * m) * D + c4), s[m]);
 
-  if (t < D) {
+  if (part == 0 && t < D) {
     float zz = z[(size_t)bh * D + t];
-    for (int l = 0; l < L; ++l) zz += sm.fk[l][t];
+    for (int l = 0; l < L; ++l) zz += fk[l][t];
     z[(size_t)bh * D + t] = zz;
     // window <- last W-1 entries of (window ++ v_path); ascending, source index above target
     T* wb = win + (size_t)bh * (W - 1) * D;
     for (int i = 0; i < W - 1; ++i) {
       const int src = L + i;
-      wb[(size_t)i * D + t] = src < W - 1 ? wb[(size_t)src * D + t] : from_f32<T>(sm.v[src - (W - 1)][t]);
+      wb[(size_t)i * D + t] = src < W - 1 ? wb[(size_t)src * D + t] : from_f32<T>(vv[src - (W - 1)][t]);
     }
   }
-  if (h == 0 && t == 0) pos[b] += L;
+  if (h == 0 && part == 0 && t == 0) pos[b] += L;
 }
 
 template <typename T, int D, int PHI>
@@ -105,10 +116,10 @@ static cudaError_t launch_t(la_ctx* ctx, int B, int N, const void* k, const void
                             cudaStream_t s) {
   const la_config& c = ctx->cfg;
   auto kern = commit_kernel<T, D, PHI>;
-  const size_t smem = sizeof(CommitSmem<D>);
+  const size_t smem = (size_t)2 * c.max_depth * D * sizeof(float) + sizeof(CommitTables);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(B * c.H), dim3(256), smem, s>>>((const T*)k, (const T*)v, parent, accept, st.S, st.z, (T*)st.win, st.pos,
+  kern<<<dim3(B * c.H * kCommitSplit), dim3(256), smem, s>>>((const T*)k, (const T*)v, parent, accept, st.S, st.z, (T*)st.win, st.pos,
                                                path_out, commit_len, ctx->d_status, c.H, N, c.conv_taps, c.max_depth);
   ctx->launches += 1;
   return cudaGetLastError();
