@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -139,6 +140,7 @@ def prefill_workload(W: wl.Workload, rank: int, device):
     info = {"ctx": ctx, "tokens_per_step": tokens, "alg_bytes_per_launch": alg_bytes, "launches_per_step": 1,
             "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill" + (" (sequence split: 3 launches)" if ws_bytes else ""),
             "flops_per_launch": units * 4 * W.d * (W.chunk + W.d),
+            "period": nsets,
             "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
     return step, e2e_step, info
 
@@ -177,6 +179,7 @@ def decode_workload(W: wl.Workload, rank: int, device):
     info = {"ctx": ctx, "tokens_per_step": W.B, "alg_bytes_per_launch": alg, "launches_per_step": 1,
             "h2d": 3 * units * W.d * el, "d2h": units * W.d * el, "kernel": "decode",
             "flops_per_launch": units * 4 * W.d * W.d,
+            "period": nrot,
             "l2": f"state of {units * W.d * W.d * 4 / 2**20:.0f} MiB streamed every step (larger than L2)"}
     return step, e2e_step, info
 
@@ -232,6 +235,7 @@ def verify_workload(W: wl.Workload, rank: int, device):
     info = {"ctx": ctx, "tokens_per_step": W.B * N, "alg_bytes_per_launch": alg_verify, "launches_per_step": 2,
             "h2d": 3 * units * N * W.d * el, "d2h": units * N * W.d * el, "kernel": "verify", "probe": probe,
             "flops_per_launch": units * (2 * N * W.d * W.d + 4 * N * N * W.d),
+            "period": nrot * nsets // math.gcd(nrot, nsets),
             "l2": f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"}
     return step, e2e_step, info
 
@@ -325,6 +329,7 @@ def main():
     ap.add_argument("--workload", default="llama7b_prefill", choices=sorted(FACTORIES))
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step from Python instead of replaying a CUDA graph")
     args = ap.parse_args()
     W = wl.WORKLOADS[args.workload]()
     rank, world = ladist.rank_world()
@@ -355,19 +360,47 @@ def main():
     if ctx.la_last_device_status() != 0:
         raise RuntimeError("device status not OK after warm-up")
 
+    # The same calls, recorded once into a CUDA graph of one rotation period and replayed: the steps are short
+    # enough for the Python interpreter to be the bottleneck otherwise.  K steps = K // period replays, the rest eager.
+    period = info["period"]
+
+    def capture(fn):
+        n0 = ctx.la_launch_count()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(period):
+                fn(i)
+        return g, ctx.la_launch_count() - n0
+
+    graph = None
+    if not args.no_graph and args.steps >= period:
+        graph, launches_per_replay = capture(lambda i: step())
+        graph.replay()                                     # one untimed replay
+        torch.cuda.synchronize()
+
+    def run_steps(n):
+        extra = 0
+        if graph is not None:
+            for _ in range(n // period):
+                graph.replay()
+            extra = (n // period) * launches_per_replay
+            n = n % period
+        for _ in range(n):
+            step()
+        return extra
+
     ladist.barrier(world)
     torch.cuda.synchronize()
     launches0 = ctx.la_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clocks:
         ev0.record(stream)
-        for _ in range(args.steps):
-            step()
+        replayed = run_steps(args.steps)
         ev1.record(stream)
         torch.cuda.synchronize()
     ladist.barrier(world)
     ms = ev0.elapsed_time(ev1)
-    launches = ctx.la_launch_count() - launches0
+    launches = ctx.la_launch_count() - launches0 + replayed
     ms_max = ladist.max_over_ranks(ms, world, device)
     value = world * info["tokens_per_step"] * args.steps / (ms_max * 1e-3)
 
@@ -376,14 +409,19 @@ def main():
     if info["launches_per_step"] == 1:
         kernel_ms = ms / args.steps
     else:
-        n_probe = min(args.steps, 100)
         for i in range(3):
             info["probe"](i)
         torch.cuda.synchronize()
+        pgraph = None if graph is None else capture(info["probe"])[0]
+        n_probe = min(args.steps, 100) if pgraph is None else period * max(1, 100 // period)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         p0.record(stream)
-        for i in range(n_probe):
-            info["probe"](i)
+        if pgraph is None:
+            for i in range(n_probe):
+                info["probe"](i)
+        else:
+            for _ in range(n_probe // period):
+                pgraph.replay()
         p1.record(stream)
         torch.cuda.synchronize()
         kernel_ms = p0.elapsed_time(p1) / n_probe
@@ -431,6 +469,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16" if W.io == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": W.name, "B": W.B, "H": W.H, "d": W.d, "T": W.T, "chunk": W.chunk, "phi": W.phi,
                        "conv_taps": W.W, "tree_nodes": W.tree_nodes, "l2": info["l2"],
+                       "launch": f"CUDA graph of {period} steps, replayed" if graph is not None else "one Python call per kernel",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks.summary(),
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
