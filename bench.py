@@ -34,7 +34,7 @@ from paper_2406_07368_b200 import dist as ladist   # noqa: E402
 L2_BYTES = 126 * 2 ** 20
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu captures summarised under
 # profiles/; None where no capture of the current kernel exists.
-NCU_TRAFFIC = {"llama7b_prefill": 249.5e6, "batched_decode": 216.0e6, "tree_verify": 59.9e6, "long_prefill": None}
+NCU_TRAFFIC = {"llama7b_prefill": 249.5e6, "batched_decode": 216.0e6, "tree_verify": 61.7e6, "long_prefill": None}
 
 
 # ----------------------------------------------------------------------------------------
