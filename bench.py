@@ -32,6 +32,7 @@ from paper_2406_07368_b200 import workloads as wl  # noqa: E402
 from paper_2406_07368_b200 import dist as ladist   # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
+NOMINAL_HBM_GBS = 7700.0        # HGX B200 data-sheet figure, printed beside the measured copy bandwidth
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu captures summarised under
 # profiles/; None where no capture of the current kernel exists.
 NCU_TRAFFIC = {"llama7b_prefill": 249.5e6, "batched_decode": 216.0e6, "tree_verify": 61.7e6, "long_prefill": None}
@@ -229,11 +230,21 @@ def verify_workload(W: wl.Workload, rank: int, device):
         ctx.la_verify_tree(drafts[i % nrot][0], drafts[i % nrot][1], drafts[i % nrot][2], parents[i % nrot], w,
                            states[i % nsets], out=out)
 
+    def probe_commit(i):   # the second kernel of the step alone (it advances the state, which timing does not mind)
+        r = i % nrot
+        ctx.la_commit(drafts[r][1], drafts[r][2], parents[r], accepts[r], states[i % nsets], path_out=path, commit_len=clen)
+
+    # accepted tokens per round: the depth of the accepted node, averaged over the rotation
+    acc_len = float(np.mean([[wl.tree_depths(p[b])[a[b]] if a[b] >= 0 else 0 for b in range(W.B)] for p, a in trees]))
     units = W.B * W.H
     el = 2
     alg_verify = units * (4 * W.d * W.d + 4 * W.d + 4 * N * W.d * el + (W.W - 1) * W.d * el)
     info = {"ctx": ctx, "tokens_per_step": W.B * N, "alg_bytes_per_launch": alg_verify, "launches_per_step": 2,
             "h2d": 3 * units * N * W.d * el, "d2h": units * N * W.d * el, "kernel": "verify", "probe": probe,
+            "second": {"kernel": "commit", "probe": probe_commit,
+                       "alg_bytes_per_launch": units * (8 * W.d * W.d + 8 * W.d + acc_len * 2 * W.d * el
+                                                        + 2 * (W.W - 1) * W.d * el)},
+            "accepted_tokens_per_step": W.B * acc_len,
             "flops_per_launch": units * (2 * N * W.d * W.d + 4 * N * N * W.d),
             "period": nrot * nsets // math.gcd(nrot, nsets),
             "l2": f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"}
@@ -406,25 +417,32 @@ def main():
 
     # per-launch duration of the dominant kernel, measured live: events around every launch of a
     # short second pass on the same stream (for two-kernel steps only the first kernel is bracketed)
-    if info["launches_per_step"] == 1:
-        kernel_ms = ms / args.steps
-    else:
+    def time_probe(fn):
         for i in range(3):
-            info["probe"](i)
+            fn(i)
         torch.cuda.synchronize()
-        pgraph = None if graph is None else capture(info["probe"])[0]
+        pgraph = None if graph is None else capture(fn)[0]
         n_probe = min(args.steps, 100) if pgraph is None else period * max(1, 100 // period)
         p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         p0.record(stream)
         if pgraph is None:
             for i in range(n_probe):
-                info["probe"](i)
+                fn(i)
         else:
             for _ in range(n_probe // period):
                 pgraph.replay()
         p1.record(stream)
         torch.cuda.synchronize()
-        kernel_ms = p0.elapsed_time(p1) / n_probe
+        return p0.elapsed_time(p1) / n_probe
+
+    second = None
+    if info["launches_per_step"] == 1:
+        kernel_ms = ms / args.steps
+    else:
+        kernel_ms = time_probe(info["probe"])
+        if "second" in info:
+            second = dict(info["second"])
+            second["launch_ms"] = time_probe(second.pop("probe"))
 
     # end to end: pinned host inputs copied in, result copied out, every step
     for _ in range(2):
@@ -456,8 +474,13 @@ def main():
                 "tensor_tflops": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12,
                 "tensor_frac_of_sustained": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
                 / peaks["bf16_tflops_sustained"]}
+    roofline["frac_of_nominal_7700"] = achieved / NOMINAL_HBM_GBS
     if info["launches_per_step"] > 1:
         roofline["step_ms"] = ms / args.steps      # all kernels of the step; launch_ms is the dominant one alone
+    if second is not None:
+        a2 = second["alg_bytes_per_launch"] / (second["launch_ms"] * 1e-3) / 1e9
+        second.update({"achieved": a2, "unit": "GB/s", "frac": a2 / peaks["hbm_gbs"]})
+        roofline["second_kernel"] = second
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         reps = {"llama7b_prefill": 4, "long_prefill": 4, "batched_decode": 3, "tree_verify": 1}[W.name]
@@ -475,6 +498,8 @@ def main():
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
                     "d2h_bytes_per_step": info["d2h"], "steps": args.e2e_steps},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    if "accepted_tokens_per_step" in info:
+        line["accepted_tokens_per_s"] = world * info["accepted_tokens_per_step"] * args.steps / (ms_max * 1e-3)
     print(json.dumps(line), flush=True)
     ladist.finish(world)
     return 0
