@@ -57,11 +57,12 @@ struct Small {
   int abort;
   int pad[2];
 };
-// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B.
+// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B (O has been read).
+// VFREE: the outputs staged in a V buffer have left it (one arrival by the thread that issued the TMA store).
 // MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T[V|1] (K buffer free);
 // after [O|den] = phi(Q)[S|z] (Q buffer free); after [O|den] += P[V|1].
 enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
-       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, B_FULL_K1 = 12, kNumBars = 13 };
+       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, B_FULL_K1 = 12, B_VFREE = 13, kNumBars = 14 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
@@ -286,9 +287,9 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* v) {
 template <int PHI, int WT>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-                  const __grid_constant__ CUtensorMap mv, const float* __restrict__ w, float* __restrict__ S,
-                  float* __restrict__ z, __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos,
-                  __nv_bfloat16* __restrict__ o, int* status, int H, int Ttot, int W, float eps, int init, int nseg,
+                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
+                  const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
+                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int* status, int H, int Ttot, int W, float eps, int init, int nseg,
                   int seg_len) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -325,6 +326,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     mbar_init(bar[B_SB], kThreadsA);
     mbar_init(bar[B_EPI], kThreadsB);
     mbar_init(bar[B_MMA_Q], 1);
+    mbar_init(bar[B_VFREE], 1);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -404,16 +406,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
         }
         if (n >= 1) {
-          // group B is done with tile n-1: O may be overwritten, and its V buffer takes tile n+1
+          // group B has read O of tile n-1: it may be overwritten
           ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
           if (!ok) break;
           tc_fence_after();
-          if (n + 1 < nchunks) {
-            const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
-            mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
-            tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-            tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-          }
         }
         if (has_state) {
 #pragma unroll
@@ -424,6 +420,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
         }
         mma_commit(bar[B_MMA_Q]);
+        if (n >= 1 && n + 1 < nchunks) {
+          // the outputs of tile n-1, staged in its V buffer, have left: the buffer takes tile n+1
+          ok = mbar_wait(bar[B_VFREE], (n - 1) & 1, abort);
+          if (!ok) break;
+          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
+          mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
+          tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+          tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+        }
         if (n + 1 < nchunks) {
           ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
           if (!ok) break;
@@ -608,12 +613,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       }
       ok = ok && mbar_wait(bar[B_MMA_O], par, abort);
       ok = __all_sync(0xffffffffu, ok);
+      uint4 outp[8];                              // this thread's 64 channels of row r, packed
       if (ok) {
         tc_fence_after();
         const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
         tmem_wait_ld();
         const float rden = 1.f / (den + eps);
-        __nv_bfloat16* og = o + ((size_t)bh * Ttot + y0 + (size_t)n * TILE + r) * D;
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           uint32_t v[32];
@@ -627,16 +632,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
             conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
-            const uint4 out =
-                make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
-            if (r < valid) *reinterpret_cast<uint4*>(og + ch0) = out;
+            outp[cc] = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
           }
         }
       }
       tc_fence_before();
-      mbar_arrive(bar[B_EPI]);                    // O, V and the old halo have been read
-      sync_group_b();                             // the next halo is complete before any thread reads it
+      mbar_arrive(bar[B_EPI]);                    // O has been read
+      // The outputs leave through the V buffer of this tile: once every thread has taken its taps from it, each row
+      // is overwritten with its outputs (same swizzled layout) and one TMA store per box writes whole rows.
+      sync_group_b();                             // V and the old halo have been read; the next halo is complete
+      if (ok) {
+        unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) *reinterpret_cast<uint4*>(Ob + swz(r, cc)) = outp[cc];
+      }
+      fence_proxy_async();
+      sync_group_b();
+      if (tid == 0) {
+        if (ok) {
+          const uint32_t src = sbase + OFF_V0 + par * TILE_BYTES;
+          tma_store(&mo, 0, y0 + n * TILE, bh, src);            // rows past the end of the sequence are clipped
+          tma_store(&mo, 64, y0 + n * TILE, bh, src + BOX_BYTES);
+          tma_commit();
+          tma_wait_read();                                      // the buffer has been read
+        }
+        mbar_arrive(bar[B_VFREE]);
+      }
     }
+    if (tid == 0) tma_wait_all();                 // the last stores are complete before the CTA exits
     if (ok && tid < D) {
       const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
       for (int i = 0; i < W - 1; ++i) win[((size_t)u * (W - 1) + i) * D + tid] = halo[i * D + tid];
@@ -872,11 +895,11 @@ static bool make_map(CUtensorMap* m, const void* base, int BH, int T) {
 
 template <int PHI>
 static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
-                            const CUtensorMap& mv, const float* w, int init, float* S, float* z, __nv_bfloat16* win,
-                            int64_t* pos, void* o, int* status, int nseg, int seg_len, cudaStream_t s) {
+                            const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
+                            __nv_bfloat16* win, int64_t* pos, int* status, int nseg, int seg_len, cudaStream_t s) {
   const size_t smem = tc::smem_bytes(c.conv_taps);
-  void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               __nv_bfloat16*, int*, int, int, int, float, int, int, int);
+  void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
+               int*, int, int, int, float, int, int, int);
   switch (c.conv_taps) {     // unrolled tap loops for the common small widths
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
@@ -887,8 +910,8 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, w, S, z, win, pos, (__nv_bfloat16*)o, status, c.H, T,
-                                                     c.conv_taps, c.eps, init, nseg, seg_len);
+  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, status, c.H, T, c.conv_taps, c.eps,
+                                                     init, nseg, seg_len);
   return cudaGetLastError();
 }
 
@@ -925,8 +948,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   if (c.io_dtype != LA_BF16 || c.d != tc::D) return cudaSuccess;
   if (tc::smem_bytes(c.conv_taps) > 227u * 1024u) return cudaSuccess;   // very long tap windows: CUDA-core kernel
   const int BH = B * c.H;
-  CUtensorMap mq, mk, mv;
-  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T))
+  CUtensorMap mq, mk, mv, mo;
+  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
+      !tc::make_map(&mo, o, BH, T))
     return cudaSuccess;   // no tensor-map support: the CUDA-core kernel takes over
   int nseg, seg_len;
   plan_split(ctx, BH, T, &nseg, &seg_len);
@@ -934,9 +958,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   const bool elu = c.phi == LA_PHI_ELU1;
   cudaError_t e;
   if (nseg == 1) {
-    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, o,
+    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                     ctx->d_status, 1, T, s)
-            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, o,
+            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                     ctx->d_status, 1, T, s);
     ctx->launches += 1;
     *handled = true;
@@ -954,9 +978,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   tc::prefix_kernel<<<dim3(BH, tc::D * tc::D / 1024), dim3(256), 0, s>>>(S_seg, z_seg, win_seg, (const __nv_bfloat16*)v, st.S,
                                                                           st.z, (__nv_bfloat16*)st.win, st.pos, c.H, T,
                                                                           c.conv_taps, nseg, seg_len, init);
-  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, w, 1, S_seg, z_seg, win_seg, st.pos, o, ctx->d_status, nseg,
+  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
                                   seg_len, s)
-          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, w, 1, S_seg, z_seg, win_seg, st.pos, o, ctx->d_status, nseg,
+          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
                                   seg_len, s);
   ctx->launches += 3;
   *handled = true;
