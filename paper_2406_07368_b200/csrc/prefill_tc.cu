@@ -391,23 +391,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         ok = mbar_wait(bar[B_SB], par, abort) && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {     // [S | z] += phi(K)^T [V | 1]
-          const uint64_t kd = desc_mnmajor(kbuf, ks);
-          mma_bf16(tmem + S_COL, kd, desc_mnmajor(vbuf, ks), idesc(true, true, 128), has_state || ks > 0);
-          mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
-        }
-        mma_commit(bar[B_MMA_S]);
-        if (n + 2 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_S], par, abort);             // this K buffer is free: it takes tile n+2
-          if (!ok) break;
-          mbar_expect_tx(kbar, TILE_BYTES);
-          tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
-          tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
-        }
+        // Two chains decide the pace: the epilogue of tile n-1 -> [O|den] = phi(Q)[S|z] -> [O|den] += P[V|1] -> the
+        // epilogue of tile n; and the last read of the Q buffer -> its reload -> phi -> the products of tile n+1.
+        // Both start with the product on phi(Q), which has to wait for the epilogue of tile n-1; the state update
+        // [S|z] += phi(K)^T[V|1] is needed much later, so its steps only fill the time until that epilogue is done.
+        int s_steps = 0;
+        auto issue_s = [&](int upto) {
+          for (; s_steps < upto; ++s_steps) {
+            const uint64_t kd = desc_mnmajor(kbuf, s_steps);
+            mma_bf16(tmem + S_COL, kd, desc_mnmajor(vbuf, s_steps), idesc(true, true, 128), has_state || s_steps > 0);
+            mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, s_steps), idesc(true, true, 16), has_state || s_steps > 0);
+          }
+        };
         if (n >= 1) {
-          // group B has read O of tile n-1: it may be overwritten
-          ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
+          while (!mbar_try_wait(bar[B_EPI], (n - 1) & 1)) {
+            if (s_steps < 8) {
+              issue_s(s_steps + 1);
+            } else {
+              ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
+              break;
+            }
+          }
           if (!ok) break;
           tc_fence_after();
         }
@@ -420,22 +424,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
         }
         mma_commit(bar[B_MMA_Q]);
-        if (n >= 1 && n + 1 < nchunks) {
-          // the outputs of tile n-1, staged in its V buffer, have left: the buffer takes tile n+1
-          ok = mbar_wait(bar[B_VFREE], (n - 1) & 1, abort);
-          if (!ok) break;
-          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
-          mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
-          tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-          tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-        }
-        if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
-          if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
-          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
-          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
-        }
         ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in TMEM
         if (!ok) break;
         tc_fence_after();
@@ -446,6 +434,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16_ts(tmem + DEN_COL, pa, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
         }
         mma_commit(bar[B_MMA_O]);
+        if (n + 1 < nchunks) {
+          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
+          if (!ok) break;
+          mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
+          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
+          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
+        }
+        issue_s(8);                          // the rest of [S | z] += phi(K)^T [V | 1]
+        mma_commit(bar[B_MMA_S]);
+        if (n >= 1 && n + 1 < nchunks) {
+          // the outputs of tile n-1, staged in its V buffer, have left: the buffer takes tile n+1
+          ok = mbar_wait(bar[B_VFREE], (n - 1) & 1, abort);
+          if (!ok) break;
+          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
+          mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
+          tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+          tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
+        }
+        if (n + 2 < nchunks) {
+          ok = mbar_wait(bar[B_MMA_S], par, abort);             // this K buffer is free: it takes tile n+2
+          if (!ok) break;
+          mbar_expect_tx(kbar, TILE_BYTES);
+          tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
+          tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
+        }
       }
     }
   } else if (warp >= 8) {
@@ -636,6 +649,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
         }
       }
+      // the state update, issued after the products of this tile's outputs, reads V too: it must be complete before
+      // the outputs overwrite the buffer (it is, long since; the wait comes before the arrival below so that the
+      // next completion of that barrier cannot overtake it)
+      ok = ok && mbar_wait(bar[B_MMA_S], par, abort);
+      ok = __all_sync(0xffffffffu, ok);
       tc_fence_before();
       mbar_arrive(bar[B_EPI]);                    // O has been read
       // The outputs leave through the V buffer of this tile: once every thread has taken its taps from it, each row
