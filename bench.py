@@ -55,11 +55,25 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        self.t0 = self.t1 = None
+
+    def wait_ready(self, timeout: float = 5.0):
+        """nvidia-smi's start-up can stall CUDA calls for a moment: let it pass before anything is timed."""
+        end = time.time() + timeout
+        while self.proc is not None and not self.rows and time.time() < end:
+            time.sleep(0.05)
+
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        time.sleep(0.15)
+        self.t1 = time.time()
 
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -69,18 +83,18 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
     def __exit__(self, *a):
         if self.proc is not None:
-            time.sleep(0.15)
             self.proc.terminate()
             self.thread.join(timeout=2)
 
     def summary(self):
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        inside = [r for t, r in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t)]
+        for r in inside or [r for _, r in self.rows]:     # samples taken during the timed region, if any fell into it
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
@@ -365,6 +379,8 @@ def main():
     ctx = info["ctx"]
     stream = torch.cuda.current_stream()
 
+    clocks = ClockSampler(local)
+    clocks.__enter__()
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
@@ -404,11 +420,15 @@ def main():
     torch.cuda.synchronize()
     launches0 = ctx.la_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clocks:
-        ev0.record(stream)
-        replayed = run_steps(args.steps)
-        ev1.record(stream)
-        torch.cuda.synchronize()
+    clocks.wait_ready()
+    torch.cuda.synchronize()
+    clocks.mark_start()
+    ev0.record(stream)
+    replayed = run_steps(args.steps)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    clocks.mark_end()
+    clocks.__exit__()
     ladist.barrier(world)
     ms = ev0.elapsed_time(ev1)
     launches = ctx.la_launch_count() - launches0 + replayed

@@ -845,36 +845,52 @@ prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat1
               __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int H, int Ttot, int W, int nseg, int seg_len,
               int init) {
   const int bh = blockIdx.x, e4 = (blockIdx.y * 256 + threadIdx.x) * 4;
+  // Loads in batches of eight segments, all in flight at once; only the additions are sequential.
   float4 run = init ? *reinterpret_cast<const float4*>(S + (size_t)bh * D * D + e4) : make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int sg = 0; sg < nseg; ++sg) {
-    float4* p = reinterpret_cast<float4*>(S_seg + ((size_t)bh * nseg + sg) * D * D + e4);
-    const float4 d = *p;
-    *p = run;
-    run.x += d.x; run.y += d.y; run.z += d.z; run.w += d.w;
+  for (int sg0 = 0; sg0 < nseg; sg0 += 8) {
+    float4 d[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (sg0 + j < nseg) d[j] = *reinterpret_cast<const float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (sg0 + j < nseg) {
+        *reinterpret_cast<float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4) = run;
+        run.x += d[j].x; run.y += d[j].y; run.z += d[j].z; run.w += d[j].w;
+      }
   }
   *reinterpret_cast<float4*>(S + (size_t)bh * D * D + e4) = run;
   if (blockIdx.y == 0 && threadIdx.x < D) {
     const int c = threadIdx.x;
     float rz = init ? z[(size_t)bh * D + c] : 0.f;
-    for (int sg = 0; sg < nseg; ++sg) {
-      float* p = z_seg + ((size_t)bh * nseg + sg) * D + c;
-      const float d = *p;
-      *p = rz;
-      rz += d;
+    for (int sg0 = 0; sg0 < nseg; sg0 += 8) {
+      float d[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (sg0 + j < nseg) d[j] = z_seg[((size_t)bh * nseg + sg0 + j) * D + c];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        if (sg0 + j < nseg) {
+          z_seg[((size_t)bh * nseg + sg0 + j) * D + c] = rz;
+          rz += d[j];
+        }
     }
     z[(size_t)bh * D + c] = rz;
-    // incoming windows: the W-1 values of v before each segment; before the first one the caller's window or zeros
-    for (int sg = 0; sg < nseg; ++sg)
-      for (int i = 0; i < W - 1; ++i) {
-        const int t = sg * seg_len - (W - 1) + i;
-        __nv_bfloat16 x = __float2bfloat16_rn(0.f);
-        if (t >= 0) x = v[((size_t)bh * Ttot + t) * D + c];
-        else if (init) x = win[((size_t)bh * (W - 1) + i) * D + c];      // sg == 0: t = i - (W-1)
-        win_seg[(((size_t)bh * nseg + sg) * (W - 1) + i) * D + c] = x;
-      }
-    for (int i = 0; i < W - 1; ++i)      // final window: the last W-1 values of v (Ttot >= W-1 whenever the split is used)
-      win[((size_t)bh * (W - 1) + i) * D + c] = v[((size_t)bh * Ttot + Ttot - (W - 1) + i) * D + c];
     if (c == 0 && bh % H == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + Ttot;
+  }
+  // Incoming windows: the W-1 values of v before each segment; before the first one the caller's window or zeros.
+  // One element per thread over all blocks of this chain.  The thread that reads the caller's window entry (i, c)
+  // is also the one that overwrites it with the final window: the last W-1 values of v (Ttot >= W-1 whenever the
+  // split is used).
+  const int per_chain = nseg * (W - 1) * D;
+  for (int idx = blockIdx.y * 256 + threadIdx.x; idx < per_chain; idx += gridDim.y * 256) {
+    const int c = idx % D, i = (idx / D) % (W - 1), sg = idx / (D * (W - 1));
+    const int t = sg * seg_len - (W - 1) + i;
+    __nv_bfloat16 x = __float2bfloat16_rn(0.f);
+    if (t >= 0) x = v[((size_t)bh * Ttot + t) * D + c];
+    else if (init) x = win[((size_t)bh * (W - 1) + i) * D + c];          // sg == 0: t = i - (W-1)
+    win_seg[(((size_t)bh * nseg + sg) * (W - 1) + i) * D + c] = x;
+    if (sg == 0) win[((size_t)bh * (W - 1) + i) * D + c] = v[((size_t)bh * Ttot + Ttot - (W - 1) + i) * D + c];
   }
 }
 
