@@ -298,6 +298,54 @@ def test_bad_trees_set_the_status_word_and_write_nothing():
         st = before.clone()
 
 
+def test_calls_recorded_in_a_cuda_graph_replay_bit_exactly():
+    """Decode steps, a verification and a commit recorded once on a capturing stream, then replayed: the benchmark
+    launches its steps this way.  Same kernels, same inputs: the results equal the eager ones bit for bit."""
+    io, B, H, d, N, W = "bf16", 3, 4, 128, 16, 3
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=83)
+    accept = np.array([wl.random_accept(wl.rng(9, 6, 0, b), parent[b]) for b in range(B)], dtype=np.int32)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=16, max_depth=6)
+    dq, dk, dv = dev(q, io), dev(k, io), dev(v, io)
+    par, acc, dw = torch.from_numpy(parent).cuda(), torch.from_numpy(accept).cuda(), dev(w, "f32")
+
+    def run(st, outs):
+        for i in range(3):
+            ctx.la_decode_step(dq[:, :, i].contiguous(), dk[:, :, i].contiguous(), dv[:, :, i].contiguous(), dw, st,
+                               out=outs["dec"][i])
+        ctx.la_verify_tree(dq, dk, dv, par, dw, st, out=outs["ver"])
+        ctx.la_commit(dk, dv, par, acc, st, path_out=outs["path"], commit_len=outs["len"])
+
+    def buffers():
+        return {"dec": [torch.empty(B, H, d, dtype=torch.bfloat16, device="cuda") for _ in range(3)],
+                "ver": torch.empty(B, H, N, d, dtype=torch.bfloat16, device="cuda"),
+                "path": torch.empty(B, 6, dtype=torch.int32, device="cuda"),
+                "len": torch.empty(B, dtype=torch.int32, device="cuda")}
+
+    st_e, out_e = oracle_state_to_dev(ost, io), buffers()
+    run(st_e, out_e)
+    torch.cuda.synchronize()
+    st_g, out_g = oracle_state_to_dev(ost, io), buffers()
+    slices = [(dq[:, :, i].contiguous(), dk[:, :, i].contiguous(), dv[:, :, i].contiguous()) for i in range(3)]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(3):
+            ctx.la_decode_step(slices[i][0], slices[i][1], slices[i][2], dw, st_g, out=out_g["dec"][i])
+        ctx.la_verify_tree(dq, dk, dv, par, dw, st_g, out=out_g["ver"])
+        ctx.la_commit(dk, dv, par, acc, st_g, path_out=out_g["path"], commit_len=out_g["len"])
+    fresh = oracle_state_to_dev(ost, io)                    # capture does not run anything: start from the same state
+    for a, b in ((st_g.S, fresh.S), (st_g.z, fresh.z), (st_g.win, fresh.win), (st_g.pos, fresh.pos)):
+        a.copy_(b)
+    g.replay()
+    torch.cuda.synchronize()
+    assert ctx.la_last_device_status() == binding.LA_OK
+    for i in range(3):
+        assert torch.equal(out_e["dec"][i], out_g["dec"][i])
+    assert torch.equal(out_e["ver"], out_g["ver"]) and torch.equal(out_e["path"], out_g["path"])
+    assert torch.equal(out_e["len"], out_g["len"])
+    for a, b in ((st_e.S, st_g.S), (st_e.z, st_g.z), (st_e.win, st_g.win), (st_e.pos, st_g.pos)):
+        assert torch.equal(a, b)
+
+
 def test_host_side_rejections():
     ctx = binding.Context(2, 128, 3, "elu1", 0.0, "bf16", max_nodes=8)
     st = ctx.new_state(1)
