@@ -248,6 +248,15 @@ def verify_workload(W: wl.Workload, rank: int, device):
         r = i % nrot
         ctx.la_commit(drafts[r][1], drafts[r][2], parents[r], accepts[r], states[i % nsets], path_out=path, commit_len=clen)
 
+    # the acceptance step that sits between verify and commit in real use (the whole model runs in between, so it is
+    # not part of the timed step): timed alone, as a latency figure
+    toks = [[torch.from_numpy(x).to(device) for x in wl.token_batch(W.seed, r, W.B, N)] for r in range(nrot)]
+    acc_out = [torch.empty(W.B, dtype=torch.int32, device=device) for _ in range(3)]
+
+    def probe_accept(i):
+        r = i % nrot
+        ctx.la_accept_greedy(parents[r], toks[r][0], toks[r][1], toks[r][2], *acc_out)
+
     # accepted tokens per round: the depth of the accepted node, averaged over the rotation
     acc_len = float(np.mean([[wl.tree_depths(p[b])[a[b]] if a[b] >= 0 else 0 for b in range(W.B)] for p, a in trees]))
     units = W.B * W.H
@@ -258,7 +267,7 @@ def verify_workload(W: wl.Workload, rank: int, device):
             "second": {"kernel": "commit", "probe": probe_commit,
                        "alg_bytes_per_launch": units * (8 * W.d * W.d + 8 * W.d + acc_len * 2 * W.d * el
                                                         + 2 * (W.W - 1) * W.d * el)},
-            "accepted_tokens_per_step": W.B * acc_len,
+            "accepted_tokens_per_step": W.B * acc_len, "accept_probe": probe_accept,
             "flops_per_launch": units * (2 * N * W.d * W.d + 4 * N * N * W.d),
             "period": nrot * nsets // math.gcd(nrot, nsets),
             "l2": f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"}
@@ -518,6 +527,9 @@ def main():
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
                     "d2h_bytes_per_step": info["d2h"], "steps": args.e2e_steps},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    if "accept_probe" in info:
+        line["accept_kernel"] = {"kernel": "accept_greedy", "launch_ms": time_probe(info["accept_probe"]),
+                                 "note": "integer kernel, one warp per sequence: latency, not bandwidth"}
     if "accepted_tokens_per_step" in info:
         line["accepted_tokens_per_s"] = world * info["accepted_tokens_per_step"] * args.steps / (ms_max * 1e-3)
     print(json.dumps(line), flush=True)

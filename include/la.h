@@ -153,6 +153,28 @@ la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void
                     const int32_t* accept_node, la_state* st /*host struct*/, int32_t* path_out,
                     int32_t* commit_len, void* stream);
 
+/* Greedy acceptance: which draft nodes does the verifier accept?  (Sec. 4.2: the original model acts as the
+ * verifier and accepts or rejects the drafted tokens.  The rule implemented is the greedy one: a draft node is
+ * accepted when its token is the verifier's most likely token at the node it hangs from -- at the committed prefix
+ * for a child of the prefix -- and that node is accepted itself.)  Pure integer work; the result feeds la_commit.
+ *
+ *   parent       [B, N] int32 device, as for la_verify_tree
+ *   draft_token  [B, N] int32 device: token id drafted at node n
+ *   pred_root    [B]    int32 device: the verifier's arg-max token after the committed prefix
+ *   pred         [B, N] int32 device: the verifier's arg-max token after node n (its guess for a child of n)
+ *   accept_node  [B]    int32 device, out: the deepest accepted node, the smallest index among equally deep ones;
+ *                       -1 when no child of the prefix matches
+ *   accept_len   [B]    int32 device, out: the number of accepted draft tokens (the depth of accept_node; 0)
+ *   next_token   [B]    int32 device, out, may be null: the verifier's token that follows the accepted chain
+ *                       (pred[accept_node], or pred_root when nothing was accepted)
+ *
+ * A sequence whose parent array is invalid gets accept_node = -1, accept_len = 0, next_token = pred_root and the
+ * device status LA_ERR_BAD_TREE.  Returns LA_ERR_INVALID_ARG for null pointers or N outside 1..max_nodes.
+ */
+la_status la_accept_greedy(la_ctx* ctx, int32_t B, int32_t N, const int32_t* parent, const int32_t* draft_token,
+                           const int32_t* pred_root, const int32_t* pred, int32_t* accept_node, int32_t* accept_len,
+                           int32_t* next_token, void* stream);
+
 /* Tree verification for callers that cannot allocate device memory.  (The paper has no
  * counterpart to this entry point; it exists for the way the library is embedded.)
  *

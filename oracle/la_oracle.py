@@ -287,3 +287,40 @@ def commit(k, v, parent, accept_node, kind: str, state: State, max_depth: int):
             new.win[b] = _next_window(new.win[b][None], v[b, :, n][None, :, None, :])[0]
         new.pos[b] += len(chain)
     return new, path, clen
+
+
+def accept_greedy(parent, draft_token, pred_root, pred):
+    """Greedy acceptance of a draft tree by the verifier's arg-max tokens (Sec. 4.2: the original model accepts or
+    rejects the drafted tokens).
+
+    Node n is accepted when draft_token[n] equals the verifier's token at the node it hangs from (pred_root for a
+    child of the committed prefix, pred[parent[n]] otherwise) and that node is accepted itself.  Written as the
+    definition, in node order (parent[n] < n, so a node's parent is decided before the node).
+
+    parent, draft_token, pred: [B, N] integers; pred_root: [B].  Returns (accept_node [B], accept_len [B],
+    next_token [B]): the deepest accepted node (the smallest index among equally deep ones, -1 for none), its depth,
+    and the verifier's token that follows the accepted chain.
+    """
+    parent = np.asarray(parent)
+    B, N = parent.shape
+    node = np.full((B,), -1, dtype=np.int32)
+    length = np.zeros((B,), dtype=np.int32)
+    nxt = np.zeros((B,), dtype=np.int32)
+    for b in range(B):
+        check_tree(parent[b])
+        accepted = [False] * N
+        depth = [0] * N
+        best, best_depth = -1, 0
+        for n in range(N):
+            p = int(parent[b, n])
+            if p < 0:
+                accepted[n] = int(draft_token[b][n]) == int(pred_root[b])
+                depth[n] = 1
+            else:
+                accepted[n] = accepted[p] and int(draft_token[b][n]) == int(pred[b][p])
+                depth[n] = depth[p] + 1
+            if accepted[n] and depth[n] > best_depth:      # strict: the first (smallest) index of a depth wins
+                best, best_depth = n, depth[n]
+        node[b], length[b] = best, best_depth
+        nxt[b] = int(pred[b][best]) if best >= 0 else int(pred_root[b])
+    return node, length, nxt

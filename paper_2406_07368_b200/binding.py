@@ -24,7 +24,7 @@ LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
-           "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace",
+           "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy",
            "la_prefill_workspace_bytes"]
 
 
@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         L.la_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
+        L.la_accept_greedy.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
         L.la_verify_tree_noalloc.argtypes = [C.POINTER(la_config), i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state),
                                              vp, vp, vp]
         L.la_last_device_status.argtypes = [vp, vp]
@@ -213,6 +214,21 @@ class Context:
             C.byref(cs), _ptr(path_out, torch.int32, (B, self.max_depth), "path_out"),
             _ptr(commit_len, torch.int32, (B,), "commit_len"), _stream(stream)))
         return path_out, commit_len
+
+    def la_accept_greedy(self, parent, draft_token, pred_root, pred, accept_node=None, accept_len=None,
+                         next_token=None, stream=None):
+        B, N = parent.shape
+        dev = parent.device
+        accept_node = torch.empty(B, dtype=torch.int32, device=dev) if accept_node is None else accept_node
+        accept_len = torch.empty(B, dtype=torch.int32, device=dev) if accept_len is None else accept_len
+        next_token = torch.empty(B, dtype=torch.int32, device=dev) if next_token is None else next_token
+        _check("la_accept_greedy", lib().la_accept_greedy(
+            self._h, B, N, _ptr(parent, torch.int32, (B, N), "parent"),
+            _ptr(draft_token, torch.int32, (B, N), "draft_token"), _ptr(pred_root, torch.int32, (B,), "pred_root"),
+            _ptr(pred, torch.int32, (B, N), "pred"), _ptr(accept_node, torch.int32, (B,), "accept_node"),
+            _ptr(accept_len, torch.int32, (B,), "accept_len"), _ptr(next_token, torch.int32, (B,), "next_token"),
+            _stream(stream)))
+        return accept_node, accept_len, next_token
 
     def la_last_device_status(self, stream=None) -> int:
         return int(lib().la_last_device_status(self._h, _stream(stream)))

@@ -163,6 +163,20 @@ la_status la_commit(la_ctx* ctx, int32_t B, int32_t N, const void* k, const void
              : LA_ERR_CUDA;
 }
 
+la_status la_accept_greedy(la_ctx* ctx, int32_t B, int32_t N, const int32_t* parent, const int32_t* draft_token,
+                           const int32_t* pred_root, const int32_t* pred, int32_t* accept_node, int32_t* accept_len,
+                           int32_t* next_token, void* stream) {
+  if (!ctx || B < 1 || N < 1 || !parent || !draft_token || !pred_root || !pred || !accept_node || !accept_len)
+    return LA_ERR_INVALID_ARG;
+  if (N > ctx->cfg.max_nodes) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return la::launch_accept(ctx, B, N, parent, draft_token, pred_root, pred, accept_node, accept_len, next_token,
+                           static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
 la_status la_last_device_status(la_ctx* ctx, void* stream) {
   if (!ctx) return LA_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);

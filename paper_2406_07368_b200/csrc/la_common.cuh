@@ -79,6 +79,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
 cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const void* k, const void* v,
                              const int32_t* parent, const float* w, const la_state& st, void* o, cudaStream_t s,
                              bool* handled);
+cudaError_t launch_accept(la_ctx* ctx, int B, int N, const int32_t* parent, const int32_t* draft, const int32_t* pred_root,
+                          const int32_t* pred, int32_t* accept_node, int32_t* accept_len, int32_t* next_token,
+                          cudaStream_t s);
 // Workspace la_prefill can use for a launch of B sequences of T tokens (0: none needed).
 size_t prefill_workspace_bytes(const la_ctx* ctx, int B, int T);
 }  // namespace la

@@ -30,6 +30,7 @@ _STREAM_TREE = 4
 _STREAM_DRAFT = 5
 _STREAM_ACCEPT = 6
 _STREAM_STATE = 7
+_STREAM_TOKENS = 8
 
 
 def rng(seed: int, stream: int, a: int = 0, b: int = 0) -> np.random.Generator:
@@ -137,6 +138,17 @@ def random_accept(gen: np.random.Generator, parent: np.ndarray) -> int:
     path.reverse()
     L = int(gen.integers(1, len(path) + 1))
     return path[L - 1]
+
+
+def token_batch(seed: int, rnd: int, B: int, N: int, vocab: int = 4):
+    """Token ids for the acceptance step: what the drafter proposed at every node and what the verifier predicts
+    after the prefix and after every node.  A small vocabulary makes matches (and so accepted chains of several
+    tokens) frequent.  Returns (draft_token [B,N], pred_root [B], pred [B,N]) int32."""
+    g = rng(seed, _STREAM_TOKENS, rnd)
+    draft = g.integers(0, vocab, size=(B, N), dtype=np.int32)
+    pred_root = g.integers(0, vocab, size=(B,), dtype=np.int32)
+    pred = g.integers(0, vocab, size=(B, N), dtype=np.int32)
+    return draft, pred_root, pred
 
 
 def tree_batch(seed: int, rnd: int, B: int, N: int, max_depth: int = 5, max_fanout: int = 4):

@@ -272,6 +272,59 @@ def test_commit_matches_oracle_and_paths_are_exact(io, d, N, W):
         assert torch.equal(sb.win, st.win[b:b + 1]) and torch.equal(sb.pos, st.pos[b:b + 1])
 
 
+@pytest.mark.parametrize("B,N,vocab,depth", [(7, 64, 3, 5), (1, 1, 2, 1), (13, 37, 2, 8), (4, 64, 1, 64)])
+def test_accept_greedy_is_bit_exact(B, N, vocab, depth):
+    ctx = binding.Context(2, 128, 3, "elu1", 0.0, "bf16", max_nodes=64, max_depth=64)
+    for rnd in range(3):
+        if depth == 64:
+            parent = np.stack([wl.chain_tree(N)] * B)
+        else:
+            parent, _ = wl.tree_batch(21 + N, rnd, B, N, max_depth=depth, max_fanout=4)
+        draft, pred_root, pred = wl.token_batch(21 + N, rnd, B, N, vocab=vocab)
+        want = orc.accept_greedy(parent, draft, pred_root, pred)
+        got = ctx.la_accept_greedy(*(torch.from_numpy(x).cuda() for x in (parent, draft, pred_root, pred)))
+        assert ctx.la_last_device_status() == binding.LA_OK
+        for g, w_ in zip(got, want):
+            np.testing.assert_array_equal(g.cpu().numpy(), w_)
+
+
+def test_accept_then_commit_matches_the_oracle():
+    io, B, H, d, N, W = "bf16", 5, 2, 128, 32, 3
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=91)
+    draft, pred_root, pred = wl.token_batch(91, 0, B, N, vocab=2)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=64, max_depth=8)
+    st = oracle_state_to_dev(ost, io)
+    par = torch.from_numpy(parent).cuda()
+    node, length, _ = ctx.la_accept_greedy(par, *(torch.from_numpy(x).cuda() for x in (draft, pred_root, pred)))
+    path, clen = ctx.la_commit(dev(k, io), dev(v, io), par, node, st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    wnode, wlen, _ = orc.accept_greedy(parent, draft, pred_root, pred)
+    wst, wpath, wclen = orc.commit(k, v, parent, wnode, "elu1", ost, max_depth=8)
+    np.testing.assert_array_equal(host(clen), wlen)
+    np.testing.assert_array_equal(host(path), wpath)
+    assert torch.equal(clen, length)
+    check_state(st, wst, TOL[io])
+
+
+def test_accept_greedy_flags_bad_trees():
+    B, N = 3, 8
+    parent, _ = wl.tree_batch(5, 0, B, N)
+    draft, pred_root, pred = wl.token_batch(5, 0, B, N, vocab=1)           # everything matches
+    bad = parent.copy()
+    bad[1, 2] = 6                                                          # parent after child
+    ctx = binding.Context(2, 128, 3, "elu1", 0.0, "bf16", max_nodes=8)
+    node, length, nxt = ctx.la_accept_greedy(*(torch.from_numpy(x).cuda() for x in (bad, draft, pred_root, pred)))
+    assert ctx.la_last_device_status() == binding.LA_ERR_BAD_TREE
+    assert int(node[1]) == -1 and int(length[1]) == 0 and int(nxt[1]) == int(pred_root[1])
+    want = orc.accept_greedy(parent[[0, 2]], draft[[0, 2]], pred_root[[0, 2]], pred[[0, 2]])
+    np.testing.assert_array_equal(node[[0, 2]].cpu().numpy(), want[0])
+    ctx.la_clear_device_status()
+    with pytest.raises(binding.LaError):
+        ctx.la_accept_greedy(*(torch.zeros(1, 9, dtype=torch.int32, device="cuda") for _ in range(2)),
+                             torch.zeros(1, dtype=torch.int32, device="cuda"),
+                             torch.zeros(1, 9, dtype=torch.int32, device="cuda"))      # N > max_nodes
+
+
 def test_bad_trees_set_the_status_word_and_write_nothing():
     io, B, H, d, N, W = "bf16", 2, 2, 128, 8, 3
     ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=71)

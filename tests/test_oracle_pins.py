@@ -379,6 +379,78 @@ def test_verify_leaves_state_untouched_and_commit_equals_decode():
     assert new.pos[1] == st.pos[1]
 
 
+# ---------------------------------------------------------------------- greedy acceptance
+def test_hand_example_accept():
+    g = json.load(open(os.path.join(GOLD, "hand_example_accept.json")))
+    parent = np.array([g["parent"]], dtype=np.int32)
+    draft = np.array([g["draft_token"]], dtype=np.int32)
+    pred = np.array([g["pred"]], dtype=np.int32)
+    node, length, nxt = orc.accept_greedy(parent, draft, np.array([g["pred_root"]]), pred)
+    assert (int(node[0]), int(length[0]), int(nxt[0])) == (g["accept_node"], g["accept_len"], g["next_token"])
+    node, length, nxt = orc.accept_greedy(parent, draft, np.array([g["pred_root_none"]]), pred)
+    assert (int(node[0]), int(length[0]), int(nxt[0])) == (g["accept_node_none"], g["accept_len_none"],
+                                                           g["next_token_none"])
+
+
+def _accepted_by_path_enumeration(parent, draft, pred_root, pred):
+    """The definition read the other way round: for every node spell out its root-to-node path and check every
+    token on it against the verifier's prediction at the position before it."""
+    N = len(parent)
+    best, best_len = -1, 0
+    for n in range(N):
+        path = orc.ancestors_or_self(parent, n)
+        expected = [pred_root] + [pred[m] for m in path[:-1]]
+        if all(int(draft[m]) == int(e) for m, e in zip(path, expected)) and len(path) > best_len:
+            best, best_len = n, len(path)
+    return best, best_len, (int(pred[best]) if best >= 0 else int(pred_root))
+
+
+@pytest.mark.parametrize("vocab", [2, 3, 6])
+def test_accept_brute_force_over_all_paths(vocab):
+    for rnd in range(6):
+        parent, _ = wl.tree_batch(11, rnd, 5, 24, max_depth=6, max_fanout=3)
+        draft, pred_root, pred = wl.token_batch(11, rnd, 5, 24, vocab=vocab)
+        node, length, nxt = orc.accept_greedy(parent, draft, pred_root, pred)
+        for b in range(5):
+            assert (int(node[b]), int(length[b]), int(nxt[b])) == _accepted_by_path_enumeration(
+                parent[b], draft[b], int(pred_root[b]), pred[b])
+
+
+def test_accept_on_a_chain_stops_at_the_first_mismatch():
+    N = 12
+    parent = wl.chain_tree(N)[None]
+    pred_root = np.array([5])
+    pred = np.arange(100, 100 + N, dtype=np.int32)[None]               # after node n the verifier says 100 + n
+    draft = np.concatenate([[5], pred[0, :-1]]).astype(np.int32)[None]  # the drafter guessed everything right
+    node, length, nxt = orc.accept_greedy(parent, draft, pred_root, pred)
+    assert (int(node[0]), int(length[0]), int(nxt[0])) == (N - 1, N, 100 + N - 1)
+    for miss in (0, 4, N - 1):                                          # one wrong draft at position `miss`
+        d = draft.copy()
+        d[0, miss] = -7
+        node, length, nxt = orc.accept_greedy(parent, d, pred_root, pred)
+        assert (int(node[0]), int(length[0])) == (miss - 1, miss)
+        assert int(nxt[0]) == (5 if miss == 0 else 100 + miss - 1)
+
+
+def test_accepted_chain_is_accepted_and_cannot_be_extended():
+    parent, _ = wl.tree_batch(12, 0, 8, 40, max_depth=6, max_fanout=3)
+    draft, pred_root, pred = wl.token_batch(12, 0, 8, 40, vocab=3)
+    node, length, nxt = orc.accept_greedy(parent, draft, pred_root, pred)
+    depths = [wl.tree_depths(parent[b]) for b in range(8)]
+    for b in range(8):
+        a = int(node[b])
+        if a >= 0:
+            path = orc.ancestors_or_self(parent[b], a)
+            assert len(path) == int(length[b]) == depths[b][a]
+            assert int(draft[b][path[0]]) == int(pred_root[b])
+            for m, c in zip(path[:-1], path[1:]):
+                assert int(draft[b][c]) == int(pred[b][m])
+            # no child of the accepted node carries the token the verifier wants next
+            assert not any(parent[b][c] == a and draft[b][c] == nxt[b] for c in range(40))
+        else:
+            assert not any(parent[b][c] == -1 and draft[b][c] == pred_root[b] for c in range(40))
+
+
 def test_bad_trees_are_rejected():
     st, q, k, v, parent, w = _tree_case(23, B=1, N=5)
     bad = parent.copy()
