@@ -33,6 +33,8 @@ commit_kernel(const T* __restrict__ k, const T* __restrict__ v, const int32_t* _
   CommitTables& sm = *reinterpret_cast<CommitTables*>(vv + max_depth);
   const int bh = blockIdx.x / kCommitSplit, part = blockIdx.x % kCommitSplit, b = bh / H, h = bh % H, t = threadIdx.x;
 
+  pdl_wait();                      // the kernel before this one in the stream may still be running until here
+  pdl_trigger();
   // The state is requested before anything else: the loads are in flight while the path is rebuilt.
   const int c4 = (t % TPR) * 4, rg = part * ROWS + t / TPR;   // this CTA's rows of S: part * ROWS .. + ROWS - 1
   float* Sb = S + (size_t)bh * D * D;
@@ -119,10 +121,9 @@ static cudaError_t launch_t(la_ctx* ctx, int B, int N, const void* k, const void
   const size_t smem = (size_t)2 * c.max_depth * D * sizeof(float) + sizeof(CommitTables);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(B * c.H * kCommitSplit), dim3(256), smem, s>>>((const T*)k, (const T*)v, parent, accept, st.S, st.z, (T*)st.win, st.pos,
-                                               path_out, commit_len, ctx->d_status, c.H, N, c.conv_taps, c.max_depth);
   ctx->launches += 1;
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(B * c.H * kCommitSplit), dim3(256), smem, s, (const T*)k, (const T*)v, parent, accept, st.S,
+                    st.z, (T*)st.win, st.pos, path_out, commit_len, ctx->d_status, c.H, N, c.conv_taps, c.max_depth);
 }
 
 template <typename T, int D>

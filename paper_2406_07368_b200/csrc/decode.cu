@@ -22,6 +22,8 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restr
 
   const int bh = blockIdx.x, h = bh % H, t = threadIdx.x;
   const size_t vec = (size_t)bh * D;
+  pdl_wait();                      // the kernel before this one in the stream may still be running until here
+  pdl_trigger();
   const int c4 = (t % TPR) * 4, rg = t / TPR;
   float* Sb = S + (size_t)bh * D * D;
 
@@ -81,14 +83,10 @@ static cudaError_t launch_decode_t(la_ctx* ctx, int B, const void* q, const void
                                    const la_state& st, void* o, cudaStream_t s) {
   const la_config& c = ctx->cfg;
   dim3 grid(B * c.H), block(256);
-  if (c.phi == LA_PHI_ELU1)
-    decode_kernel<T, D, LA_PHI_ELU1><<<grid, block, 0, s>>>((const T*)q, (const T*)k, (const T*)v, w, st.S, st.z,
-                                                            (T*)st.win, st.pos, (T*)o, c.H, c.conv_taps, c.eps);
-  else
-    decode_kernel<T, D, LA_PHI_RELU><<<grid, block, 0, s>>>((const T*)q, (const T*)k, (const T*)v, w, st.S, st.z,
-                                                            (T*)st.win, st.pos, (T*)o, c.H, c.conv_taps, c.eps);
+  auto kern = c.phi == LA_PHI_ELU1 ? decode_kernel<T, D, LA_PHI_ELU1> : decode_kernel<T, D, LA_PHI_RELU>;
   ctx->launches += 1;
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, block, 0, s, (const T*)q, (const T*)k, (const T*)v, w, st.S, st.z, (T*)st.win, st.pos,
+                    (T*)o, c.H, c.conv_taps, c.eps);
 }
 
 cudaError_t launch_decode(la_ctx* ctx, int B, const void* q, const void* k, const void* v, const float* w,

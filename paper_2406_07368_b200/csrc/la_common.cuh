@@ -23,6 +23,14 @@ template <int PHI> __device__ __forceinline__ float phi(float x) {
   return fmaxf(x, 0.f);
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// A kernel launched with launch_pdl() may start while its predecessor in the stream is still running (as SMs
+// become free), so that its launch latency and its set-up overlap the predecessor's tail.  Every thread calls
+// pdl_wait() before it touches global memory: it returns once the predecessor has completed and its writes are
+// visible.  pdl_trigger() then lets the successor start in the same way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- sticky device status ---------------------------------------------------------------
 __device__ __forceinline__ void report(int* status, int code) { atomicCAS(status, 0, code); }
 
@@ -59,6 +67,22 @@ struct la_ctx {
   void* ws;               // caller-provided device workspace (may be null)
   size_t ws_bytes;
 };
+
+// Launch with programmatic stream serialization allowed (see pdl_wait above).
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 // Kernel launchers (one per translation unit).  All return the cudaError_t of the launch.
 namespace la {

@@ -242,6 +242,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = ctl.tmem_base;
+  pdl_wait();                                // everything above touched shared memory and TMEM only
+  pdl_trigger();
 
   if (warp == kCtrlWarp) {
     // =============================== TMA and the tensor cores (one lane) ===============================
@@ -650,12 +652,12 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
   auto kern = c.phi == LA_PHI_ELU1 ? vtc::verify_tc_kernel<LA_PHI_ELU1> : vtc::verify_tc_kernel<LA_PHI_RELU>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vtc::kSmemBytes);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), vtc::kSmemBytes, s>>>(
-      ms, mv, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, parent, w, st.z, (const __nv_bfloat16*)st.win,
-      (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps, BH);
+  e = launch_pdl(kern, dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), vtc::kSmemBytes, s, ms, mv,
+                 (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, parent, w, (const float*)st.z,
+                 (const __nv_bfloat16*)st.win, (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps, BH);
   ctx->launches += 1;
   *handled = true;
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace la
