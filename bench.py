@@ -274,12 +274,67 @@ def verify_workload(W: wl.Workload, rank: int, device):
     return step, e2e_step, info
 
 
+def promptgen_workload(W: wl.Workload, rank: int, device):
+    """Prompt + generation: for every (P, G) pair a prefill of P tokens, then G decode steps, one sequence."""
+    from paper_2406_07368_b200 import binding
+    io, shapes = W.io, W.extra["shapes"]
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io, chunk=W.chunk)
+    w = dev(W.weights(), "f32", device)
+    tdt = binding.TORCH_DTYPE[io]
+    prompts, gens, outs_p, outs_g, states = [], [], [], [], []
+    for i, (P, G) in enumerate(shapes):
+        q, k, v = wl.qkv(W.seed + 100 * rank + i, (W.B, W.H, P + G, W.d), W.scale, io)
+        prompts.append([dev(x[:, :, :P], io, device) for x in (q, k, v)])
+        # generation tokens step-major, so that every step reads one contiguous [B, H, d] slab
+        gens.append([dev(np.ascontiguousarray(np.moveaxis(x[:, :, P:], 2, 0)), io, device) for x in (q, k, v)])
+        outs_p.append(torch.empty(W.B, W.H, P, W.d, dtype=tdt, device=device))
+        outs_g.append(torch.empty(G, W.B, W.H, W.d, dtype=tdt, device=device))
+        states.append(ctx.new_state(W.B))
+
+    def run_shape(i):
+        P, G = shapes[i]
+        ctx.la_prefill(prompts[i][0], prompts[i][1], prompts[i][2], w, states[i], init_state=False, out=outs_p[i])
+        for g in range(G):
+            ctx.la_decode_step(gens[i][0][g], gens[i][1][g], gens[i][2][g], w, states[i], out=outs_g[i][g])
+
+    def step():
+        for i in range(len(shapes)):
+            run_shape(i)
+
+    pinned = [[x.cpu().pin_memory() for x in prompts[i] + gens[i]] for i in range(len(shapes))]
+    host_out = [[torch.empty(o.shape, dtype=tdt).pin_memory() for o in (outs_p[i], outs_g[i])] for i in range(len(shapes))]
+
+    def e2e_step():
+        for i in range(len(shapes)):
+            for dst, src in zip(prompts[i] + gens[i], pinned[i]):
+                dst.copy_(src, non_blocking=True)
+            run_shape(i)
+            host_out[i][0].copy_(outs_p[i], non_blocking=True)
+            host_out[i][1].copy_(outs_g[i], non_blocking=True)
+
+    tokens = W.B * sum(P + G for P, G in shapes)
+    units = W.B * W.H
+    el = 2
+    dec_bytes = units * (8 * W.d * W.d + 2 * 4 * W.d + 4 * W.d * el + 2 * (W.W - 1) * W.d * el)
+    n_launch = sum(1 + G for _, G in shapes)
+    moved = 4 * tokens * W.H * W.d * el
+    info = {"ctx": ctx, "tokens_per_step": tokens, "alg_bytes_per_launch": dec_bytes, "launches_per_step": n_launch,
+            "h2d": 3 * tokens * W.H * W.d * el, "d2h": tokens * W.H * W.d * el, "kernel": "decode (one sequence: 32 units)",
+            "probe": lambda i: ctx.la_decode_step(gens[0][0][i % 16], gens[0][1][i % 16], gens[0][2][i % 16], w, states[0],
+                                                  out=outs_g[0][i % 16]),
+            "flops_per_launch": units * 4 * W.d * W.d, "period": 1, "shape_probe": run_shape, "shapes": shapes,
+            "l2": f"{moved / 2**20:.0f} MiB of tokens and {units * W.d * W.d * 4 / 2**20:.0f} MiB of state per shape: "
+                  "L2-resident by nature of the workload (a single sequence)"}
+    return step, e2e_step, info
+
+
 FACTORIES = {"llama7b_prefill": prefill_workload, "long_prefill": prefill_workload,
-             "batched_decode": decode_workload, "tree_verify": verify_workload}
+             "batched_decode": decode_workload, "tree_verify": verify_workload, "prompt_gen": promptgen_workload}
 METRICS = {"llama7b_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "long_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "batched_decode": ("decode_tokens_per_s_per_layer", "tokens/s"),
-           "tree_verify": ("verify_nodes_per_s_per_layer", "nodes/s")}
+           "tree_verify": ("verify_nodes_per_s_per_layer", "nodes/s"),
+           "prompt_gen": ("prompt_and_generation_tokens_per_s_per_layer", "tokens/s")}
 
 
 # ----------------------------------------------------------------------------------------
@@ -292,6 +347,16 @@ def oracle_sample(W: wl.Workload):
         w = W.weights()
         return (lambda: orc.prefill_quadratic(q, k, v, w, W.phi, W.eps), T,
                 f"quadratic definition, 1 of {W.B} sequences, all {W.H} heads, first {T} of {W.T} tokens")
+    if W.name == "prompt_gen":
+        P, G = min(W.extra["shapes"], key=lambda pg: pg[0] + pg[1])
+        q, k, v = wl.qkv(W.seed, (W.B, W.H, P + G, W.d), W.scale, W.io)
+        w = W.weights()
+
+        def fn():
+            _, st = orc.prefill_chunked(q[:, :, :P], k[:, :, :P], v[:, :, :P], w, W.phi, W.eps, W.chunk)
+            for g in range(G):
+                _, st = orc.decode_step(q[:, :, P + g], k[:, :, P + g], v[:, :, P + g], w, W.phi, W.eps, st)
+        return fn, W.B * (P + G), f"grouped prefill of {P} tokens then {G} recurrent steps: the ({P}, {G}) pair, all heads"
     if W.name == "batched_decode":
         B = 8
         q, k, v = W.prefill_inputs(B=B, T=64)
@@ -375,7 +440,7 @@ def main():
             run_reference(args, W)
         return 0
 
-    defaults = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000}
+    defaults = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
     args.steps = args.steps or defaults[W.name]
     args.warmup = 5 if args.warmup is None else max(3, args.warmup)
 
@@ -512,7 +577,7 @@ def main():
         roofline["second_kernel"] = second
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        reps = {"llama7b_prefill": 4, "long_prefill": 4, "batched_decode": 3, "tree_verify": 1}[W.name]
+        reps = {"llama7b_prefill": 4, "long_prefill": 4, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
         v, per, text = time_oracle(W, reps, warmup=0)
         cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text,
                "seconds": per * reps}
@@ -527,6 +592,24 @@ def main():
             "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
                     "d2h_bytes_per_step": info["d2h"], "steps": args.e2e_steps},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    if "shape_probe" in info:                    # latency of every (prompt, generation) pair on its own
+        line["shape_ms"] = {}
+        for i, (P, G) in enumerate(info["shapes"]):
+            fn = info["shape_probe"]
+            fn(i)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn(i)
+            g.replay()
+            torch.cuda.synchronize()
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            p0.record(stream)
+            for _ in range(5):
+                g.replay()
+            p1.record(stream)
+            torch.cuda.synchronize()
+            line["shape_ms"][f"({P}, {G})"] = p0.elapsed_time(p1) / 5
     if "accept_probe" in info:
         line["accept_kernel"] = {"kernel": "accept_greedy", "launch_ms": time_probe(info["accept_probe"]),
                                  "note": "integer kernel, one warp per sequence: latency, not bandwidth"}

@@ -161,7 +161,7 @@ def tree_batch(seed: int, rnd: int, B: int, N: int, max_depth: int = 5, max_fano
 
 
 # --------------------------------------------------------------------------
-# The five workload shapes
+# The workload shapes
 # --------------------------------------------------------------------------
 
 @dataclass
@@ -236,4 +236,12 @@ def long_prefill() -> Workload:
                     decode_steps=512)
 
 
-WORKLOADS = {w().name: w for w in (tiny_fp32, llama7b_prefill, batched_decode, tree_verify, long_prefill)}
+def prompt_gen() -> Workload:
+    """One sequence, H=32, d=128, bf16, elu+1, 3 taps: a prompt of P tokens is prefilled and G tokens are then
+    generated one by one, for the (P, G) pairs of the paper's table of inference latency at various prefill and
+    decode sizes: (340, 160), (60, 20), (7000, 200), (1700, 400).  Inputs N(0,1)."""
+    return Workload("prompt_gen", "bf16", 1, 32, 128, 7000, 3, 64, "elu1", 0.0, 5, 1.0,
+                    extra={"shapes": [(340, 160), (60, 20), (7000, 200), (1700, 400)]})
+
+
+WORKLOADS = {w().name: w for w in (tiny_fp32, llama7b_prefill, batched_decode, tree_verify, long_prefill, prompt_gen)}

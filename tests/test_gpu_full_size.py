@@ -152,3 +152,26 @@ def test_tree_verify_full_size_rounds():
         np.testing.assert_array_equal(host(st.win[sl]), ost[(b, h)].win)
         assert int(st.pos[b]) == int(ost[(b, h)].pos[0])
     assert ctx.la_last_device_status() == binding.LA_OK
+
+
+def test_prompt_gen_pairs_prefill_then_generate():
+    """The two shorter (prompt, generation) pairs end to end at full head count: every output token and the final
+    state against the oracle's quadratic definition over the whole P + G sequence."""
+    W = wl.prompt_gen()
+    w = W.weights()
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, W.io, chunk=W.chunk)
+    for i, (P, G) in enumerate(W.extra["shapes"]):
+        if P + G > 600:
+            continue
+        q, k, v = wl.qkv(W.seed + i, (W.B, W.H, P + G, W.d), W.scale, W.io)
+        st = ctx.new_state(W.B)
+        op = ctx.la_prefill(dev(q[:, :, :P]), dev(k[:, :, :P]), dev(v[:, :, :P]), dev(w, "f32"), st)
+        og = [ctx.la_decode_step(dev(q[:, :, P + g]), dev(k[:, :, P + g]), dev(v[:, :, P + g]), dev(w, "f32"), st)
+              for g in range(G)]
+        want, wst = orc.prefill_quadratic(q, k, v, w, W.phi, W.eps)
+        assert rel_err(host(op), want[:, :, :P]) < TOL["bf16"], (P, G)
+        assert rel_err(np.stack([host(o) for o in og], axis=2), want[:, :, P:]) < TOL["bf16"], (P, G)
+        assert rel_err(host(st.S), wst.S) < TOL["bf16"] and rel_err(host(st.z), wst.z) < TOL["bf16"]
+        np.testing.assert_array_equal(host(st.win), wst.win)
+        assert int(st.pos[0]) == P + G
+    assert ctx.la_last_device_status() == binding.LA_OK

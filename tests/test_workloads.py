@@ -48,4 +48,5 @@ def test_workload_shapes():
     assert abs(float(q.std()) - 128 ** -0.5) < 0.01
     cw = w.weights()
     assert cw.shape == (32, 128, 3) and abs(float(cw.var()) - 1 / 3) < 0.02
-    assert set(wl.WORKLOADS) == {"tiny_fp32", "llama7b_prefill", "batched_decode", "tree_verify", "long_prefill"}
+    assert set(wl.WORKLOADS) == {"tiny_fp32", "llama7b_prefill", "batched_decode", "tree_verify", "long_prefill",
+                                 "prompt_gen"}
