@@ -31,7 +31,7 @@ constexpr int kMaxTaps = 4;                        // longer tap windows are ser
 constexpr int kThreadsX = 256, kThreadsY = 256, kCtrlWarp = 16, kTreeWarp = 17, kThreads = 576;
 constexpr uint32_t S_BYTES = 128 * 128 * 4;        // the fp32 state of one unit, row-major
 constexpr uint32_t SB_BOX = 128 * 128;             // 128 rows x 64 bf16
-constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 32 fp32 (also: 64 rows x 64 bf16)
+constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 64 bf16
 constexpr uint32_t V_BOX = (NMAX + 16) * 128;      // 64 draft rows + 16 window rows x 64 bf16
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t P_COL = 64, G_COL = 128;                // G_j at G_COL + 64 j
