@@ -66,7 +66,13 @@ enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
-__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
+// Two halo buffers (the rows of v before a tile, for the convolution) while they fit; for the longest tap windows
+// one buffer for the first tile only, and later tiles take those rows from v in global memory.
+__host__ __device__ inline uint32_t smem_bytes2(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
+__host__ __device__ inline bool global_halo(int W) { return smem_bytes2(W) > 227u * 1024u; }
+__host__ __device__ inline uint32_t smem_bytes(int W) {
+  return global_halo(W) ? off_halo(W) + (uint32_t)(W - 1) * D * 2 + 1024 : smem_bytes2(W);
+}
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -289,7 +295,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                   const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
                   const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
-                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int* status, int H, int Ttot, int W, float eps, int init, int nseg,
+                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, const __nv_bfloat16* __restrict__ vg,
+                  int* status, int H, int Ttot, int W, float eps, int init, int nseg,
                   int seg_len) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -299,6 +306,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   // two halo buffers [W-1][128], oldest row first: tile n reads buffer n&1 and writes buffer (n+1)&1
   __nv_bfloat16* halo0 = reinterpret_cast<__nv_bfloat16*>(smem + off_halo(W));
   const int halo_elems = (W > 1 ? W - 1 : 1) * D;
+  const bool gh = global_halo(W);
   volatile int* abort = &sm.abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -608,11 +616,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       const uint32_t par = n & 1;
       const int valid = min(TILE, T - n * TILE);
       const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
-      const __nv_bfloat16* halo = halo0 + par * halo_elems;         // rows before this tile
+      // rows before this tile, addressed so that row -1 is the last of W-1 rows
+      const __nv_bfloat16* halo = !gh      ? halo0 + par * halo_elems
+                                  : n == 0 ? halo0
+                                           : vg + ((size_t)bh * Ttot + y0 + (size_t)n * TILE - (W - 1)) * D;
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
       ok = ok && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && tid < D) {
+      if (ok && tid < D && !gh) {
         // next halo <- last W-1 rows of (halo ++ valid rows of V)
         const unsigned char* Vc = Vt + (tid >> 6) * BOX_BYTES;
         const int cw = tid & 63;
@@ -679,8 +690,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     }
     if (tid == 0) tma_wait_all();                 // the last stores are complete before the CTA exits
     if (ok && tid < D) {
+      // the window to carry on: the last W-1 values of (incoming window ++ this unit's v)
       const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
-      for (int i = 0; i < W - 1; ++i) win[((size_t)u * (W - 1) + i) * D + tid] = halo[i * D + tid];
+      for (int i = 0; i < W - 1; ++i) {
+        const int t = T - (W - 1) + i;
+        win[((size_t)u * (W - 1) + i) * D + tid] =
+            !gh ? halo[i * D + tid] : t >= 0 ? vg[((size_t)bh * Ttot + y0 + t) * D + tid] : halo0[(t + W - 1) * D + tid];
+      }
       if (tid == 0 && h == 0 && nseg == 1) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
   }
@@ -930,10 +946,11 @@ static bool make_map(CUtensorMap* m, const void* base, int BH, int T) {
 template <int PHI>
 static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
-                            __nv_bfloat16* win, int64_t* pos, int* status, int nseg, int seg_len, cudaStream_t s) {
+                            __nv_bfloat16* win, int64_t* pos, const void* vg, int* status, int nseg, int seg_len,
+                            cudaStream_t s) {
   const size_t smem = tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               int*, int, int, int, float, int, int, int);
+               const __nv_bfloat16*, int*, int, int, int, float, int, int, int);
   switch (c.conv_taps) {     // unrolled tap loops for the common small widths
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
@@ -944,8 +961,8 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, status, c.H, T, c.conv_taps, c.eps,
-                                                     init, nseg, seg_len);
+  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, (const __nv_bfloat16*)vg, status, c.H, T,
+                                                     c.conv_taps, c.eps, init, nseg, seg_len);
   return cudaGetLastError();
 }
 
@@ -980,7 +997,7 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   const la_config& c = ctx->cfg;
   *handled = false;
   if (c.io_dtype != LA_BF16 || c.d != tc::D) return cudaSuccess;
-  if (tc::smem_bytes(c.conv_taps) > 227u * 1024u) return cudaSuccess;   // very long tap windows: CUDA-core kernel
+  if (tc::smem_bytes(c.conv_taps) > 227u * 1024u) return cudaSuccess;   // (does not happen up to LA_MAX_TAPS)
   const int BH = B * c.H;
   CUtensorMap mq, mk, mv, mo;
   if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
@@ -992,9 +1009,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   const bool elu = c.phi == LA_PHI_ELU1;
   cudaError_t e;
   if (nseg == 1) {
-    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
+    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
                                     ctx->d_status, 1, T, s)
-            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
+            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
                                     ctx->d_status, 1, T, s);
     ctx->launches += 1;
     *handled = true;
@@ -1012,9 +1029,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   tc::prefix_kernel<<<dim3(BH, tc::D * tc::D / 1024), dim3(256), 0, s>>>(S_seg, z_seg, win_seg, (const __nv_bfloat16*)v, st.S,
                                                                           st.z, (__nv_bfloat16*)st.win, st.pos, c.H, T,
                                                                           c.conv_taps, nseg, seg_len, init);
-  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
+  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
                                   seg_len, s)
-          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
+          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
                                   seg_len, s);
   ctx->launches += 3;
   *handled = true;
