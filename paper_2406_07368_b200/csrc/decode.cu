@@ -8,7 +8,7 @@
 
 namespace la {
 
-template <typename T, int D, int PHI>
+template <typename T, int D, int PHI, int WCAP>
 __global__ void __launch_bounds__(256)
 decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
               const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z, T* __restrict__ win,
@@ -31,6 +31,22 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restr
   float4 s[PASSES];
 #pragma unroll
   for (int m = 0; m < PASSES; ++m) s[m] = __ldcs(reinterpret_cast<const float4*>(Sb + (size_t)(rg + RPP * m) * D + c4));
+
+  // ... and, for short tap windows (W <= WCAP; WCAP = 0: any W, handled at the end), so are the window and the taps
+  // of this channel: in registers before they are needed, so that the shift at the end is stores only
+  constexpr int NW = WCAP > 0 ? WCAP - 1 : 1;
+  T wr[NW];
+  float wc[NW], w0 = 0.f;                        // wc[i]: the tap that meets window row i (W-1-i steps back)
+  T* wb = win + (size_t)bh * (W - 1) * D;
+  if (WCAP > 0 && t < D) {
+#pragma unroll
+    for (int i = 0; i < WCAP - 1; ++i)
+      if (i < W - 1) wr[i] = wb[(size_t)i * D + t];
+    w0 = w[((size_t)h * D + t) * W];
+#pragma unroll
+    for (int i = 0; i < WCAP - 1; ++i)
+      if (i < W - 1) wc[i] = w[((size_t)h * D + t) * W + (W - 1 - i)];
+  }
 
   float den_part = 0.f;
   if (t < D) {
@@ -67,11 +83,37 @@ decode_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restr
     float num = 0.f;
 #pragma unroll
     for (int g = 0; g < RPP; ++g) num += red[g][t];
-    const float* wc = w + ((size_t)h * D + t) * W;
-    float conv = wc[0] * vv[t];
-    T* wb = win + (size_t)bh * (W - 1) * D;
-    for (int tap = 1; tap < W; ++tap) conv = fmaf(wc[tap], to_f32(wb[(size_t)(W - 1 - tap) * D + t]), conv);
-    for (int i = 0; i + 2 < W; ++i) wb[(size_t)i * D + t] = wb[(size_t)(i + 1) * D + t];
+    float conv;
+    if (WCAP > 0) {
+      conv = w0 * vv[t];
+#pragma unroll
+      for (int i = 0; i < WCAP - 1; ++i)                   // window row i holds the value W-1-i steps back
+        if (i < W - 1) conv = fmaf(wc[i], to_f32(wr[i]), conv);
+#pragma unroll
+      for (int i = 0; i < WCAP - 2; ++i)
+        if (i + 2 < W) wb[(size_t)i * D + t] = wr[i + 1];
+    } else {
+      // one pass over the window in batches of eight rows: all loads of a batch are in flight together; row i is
+      // used for its tap and then stored one place down (a batch only overwrites rows it or an earlier one has read)
+      const float* wg = w + ((size_t)h * D + t) * W;
+      conv = wg[0] * vv[t];
+      for (int base = 0; base < W - 1; base += 8) {
+        T r[8];
+        float g[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (base + i < W - 1) {
+            r[i] = wb[(size_t)(base + i) * D + t];
+            g[i] = wg[W - 1 - (base + i)];
+          }
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (base + i < W - 1) {
+            conv = fmaf(g[i], to_f32(r[i]), conv);
+            if (base + i >= 1) wb[(size_t)(base + i - 1) * D + t] = r[i];
+          }
+      }
+    }
     if (W > 1) wb[(size_t)(W - 2) * D + t] = v[vec + t];
     o[vec + t] = from_f32<T>(num / (den + eps) + conv);
   }
@@ -83,7 +125,10 @@ static cudaError_t launch_decode_t(la_ctx* ctx, int B, const void* q, const void
                                    const la_state& st, void* o, cudaStream_t s) {
   const la_config& c = ctx->cfg;
   dim3 grid(B * c.H), block(256);
-  auto kern = c.phi == LA_PHI_ELU1 ? decode_kernel<T, D, LA_PHI_ELU1> : decode_kernel<T, D, LA_PHI_RELU>;
+  const bool elu = c.phi == LA_PHI_ELU1;
+  auto kern = c.conv_taps <= 4   ? (elu ? decode_kernel<T, D, LA_PHI_ELU1, 4> : decode_kernel<T, D, LA_PHI_RELU, 4>)
+              : c.conv_taps <= 8 ? (elu ? decode_kernel<T, D, LA_PHI_ELU1, 8> : decode_kernel<T, D, LA_PHI_RELU, 8>)
+                                 : (elu ? decode_kernel<T, D, LA_PHI_ELU1, 0> : decode_kernel<T, D, LA_PHI_RELU, 0>);
   ctx->launches += 1;
   return launch_pdl(kern, grid, block, 0, s, (const T*)q, (const T*)k, (const T*)v, w, st.S, st.z, (T*)st.win, st.pos,
                     (T*)o, c.H, c.conv_taps, c.eps);

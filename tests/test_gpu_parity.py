@@ -50,6 +50,8 @@ def make(io, B, H, d, T, W, seed, scale=1.0):
     ("bf16", 128, "relu", 1e-6, 5, 333),
     ("bf16", 64, "elu1", 0.0, 3, 200),
     ("bf16", 128, "elu1", 0.0, 32, 150),
+    ("bf16", 128, "elu1", 0.0, 26, 300),
+    ("bf16", 128, "relu", 1e-6, 27, 300),
     ("bf16", 128, "elu1", 0.0, 1, 150),
 ])
 def test_prefill_matches_oracle(kernel, io, d, phi, eps, W, T):
@@ -82,6 +84,27 @@ def test_prefill_continuation(kernel, io, T1, T2):
                         init_state=True)
     want, wst = orc.prefill_quadratic(q, k, v, w, "elu1", 0.0)
     assert rel_err(np.concatenate([host(o1), host(o2)], axis=2), want) < TOL[io]
+    check_state(st, wst, TOL[io])
+
+
+@pytest.mark.parametrize("T1,T2,T3", [(20, 300, 9), (140, 17, 130)])
+def test_prefill_continuation_with_the_longest_tap_window(T1, T2, T3):
+    """32 taps: the window carried between calls is longer than some of the pieces, and tiles after the first take
+    the rows before them from v in global memory."""
+    io, B, H, d, W = "bf16", 2, 2, 128, 32
+    T = T1 + T2 + T3
+    q, k, v, w = make(io, B, H, d, T, W, seed=15, scale=0.5)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    st = ctx.new_state(B)
+    cut = lambda x, a, b: dev(x[:, :, a:b], io)
+    outs, a = [], 0
+    for i, n in enumerate((T1, T2, T3)):
+        outs.append(ctx.la_prefill(cut(q, a, a + n), cut(k, a, a + n), cut(v, a, a + n), dev(w, "f32"), st,
+                                   init_state=i > 0))
+        a += n
+    want, wst = orc.prefill_quadratic(q, k, v, w, "elu1", 0.0)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    assert rel_err(np.concatenate([host(o) for o in outs], axis=2), want) < TOL[io]
     check_state(st, wst, TOL[io])
 
 
@@ -139,7 +162,10 @@ def test_prefill_is_causal_bitwise():
 # ------------------------------------------------------------------ decode
 @pytest.mark.parametrize("io,d,phi,eps,W", [("f32", 64, "elu1", 0.0, 3), ("bf16", 128, "elu1", 0.0, 3),
                                             ("bf16", 128, "relu", 1e-6, 5), ("bf16", 64, "elu1", 0.0, 1),
-                                            ("f32", 128, "elu1", 0.0, 32)])
+                                            ("f32", 128, "elu1", 0.0, 32), ("bf16", 128, "elu1", 0.0, 2),
+                                            ("bf16", 128, "elu1", 0.0, 4), ("bf16", 128, "relu", 1e-6, 8),
+                                            ("bf16", 128, "elu1", 0.0, 9), ("bf16", 128, "elu1", 0.0, 17),
+                                            ("bf16", 128, "elu1", 0.0, 32)])
 def test_decode_matches_oracle(io, d, phi, eps, W):
     B, H, T0, steps = 3, 2, 40, 12
     q, k, v, w = make(io, B, H, d, T0, W, seed=21 + W, scale=0.7)
