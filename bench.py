@@ -166,6 +166,8 @@ def prefill_workload(W: wl.Workload, rank: int, device):
     info = {"ctx": ctx, "tokens_per_step": tokens, "alg_bytes_per_launch": alg_bytes, "launches_per_step": 1,
             "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill" + (" (sequence split: 3 launches)" if ws_bytes else ""),
             "flops_per_launch": units * 4 * W.d * (W.chunk + W.d),
+            # causal-strict count: the masked upper triangle of every group is not counted
+            "flops_strict_per_launch": units * (2 * W.d * (W.chunk + 1) + 4 * W.d * W.d),
             "period": nsets,
             "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
     return step, e2e_step, info
@@ -639,6 +641,11 @@ def main():
                 "tensor_frac_of_sustained": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
                 / peaks["bf16_tflops_sustained"]}
     roofline["frac_of_nominal_7700"] = achieved / NOMINAL_HBM_GBS
+    if roofline["traffic"] is not None:          # the same fraction from the DRAM bytes ncu counted, not the algorithmic ones
+        roofline["achieved_from_traffic"] = roofline["traffic"] / (kernel_ms * 1e-3) / 1e9
+        roofline["frac_from_traffic"] = roofline["achieved_from_traffic"] / peaks["hbm_gbs"]
+    if "flops_strict_per_launch" in info:
+        roofline["tensor_tflops_strict"] = info["flops_strict_per_launch"] / (kernel_ms * 1e-3) / 1e12
     if info["launches_per_step"] > 1:
         roofline["step_ms"] = ms / args.steps      # all kernels of the step; launch_ms is the dominant one alone
     if second is not None:
