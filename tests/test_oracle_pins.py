@@ -488,3 +488,13 @@ def test_pins_catch_planted_mistakes(monkeypatch):
                                           orc.empty_state(1, 1, 2, 2))[0] for i in range(3)], axis=2), None)) > 1e-6
     # (c) reversed taps
     assert off(lambda: orc.prefill_quadratic(q, k, v, w[:, :, ::-1], "relu", 0.0)) > 1e-6
+    # (d) acceptance: the verifier's predictions attached to the wrong nodes (shifted by one) change the hand-worked
+    #     result, and the tie of that example (nodes 5 and 6, both at depth 3) goes to the smaller index
+    g = json.load(open(os.path.join(GOLD, "hand_example_accept.json")))
+    parent = np.array([g["parent"]], dtype=np.int32)
+    draft = np.array([g["draft_token"]], dtype=np.int32)
+    pred = np.array([g["pred"]], dtype=np.int32)
+    node, length, _ = orc.accept_greedy(parent, draft, np.array([g["pred_root"]]), np.roll(pred, 1, axis=1))
+    assert (int(node[0]), int(length[0])) != (g["accept_node"], g["accept_len"])
+    node, _, _ = orc.accept_greedy(parent, draft, np.array([g["pred_root"]]), pred)
+    assert int(node[0]) == 5
