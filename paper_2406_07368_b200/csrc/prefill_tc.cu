@@ -861,15 +861,15 @@ prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat1
               __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, int H, int Ttot, int W, int nseg, int seg_len,
               int init) {
   const int bh = blockIdx.x, e4 = (blockIdx.y * 256 + threadIdx.x) * 4;
-  // Loads in batches of eight segments, all in flight at once; only the additions are sequential.
+  // Loads in batches of sixteen segments, all in flight at once; only the additions are sequential.
   float4 run = init ? *reinterpret_cast<const float4*>(S + (size_t)bh * D * D + e4) : make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int sg0 = 0; sg0 < nseg; sg0 += 8) {
-    float4 d[8];
+  for (int sg0 = 0; sg0 < nseg; sg0 += 16) {
+    float4 d[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < 16; ++j)
       if (sg0 + j < nseg) d[j] = *reinterpret_cast<const float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4);
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < 16; ++j)
       if (sg0 + j < nseg) {
         *reinterpret_cast<float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4) = run;
         run.x += d[j].x; run.y += d[j].y; run.z += d[j].z; run.w += d[j].w;
