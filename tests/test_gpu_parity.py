@@ -87,6 +87,23 @@ def test_prefill_continuation(kernel, io, T1, T2):
     check_state(st, wst, TOL[io])
 
 
+def test_prefill_more_chains_than_sms():
+    """160 chains on 148 SMs: the chains of the second wave start when CTAs of the first one have left."""
+    io, B, H, d, W, T = "bf16", 5, 32, 128, 3, 300
+    q, k, v, w = make(io, B, H, d, T, W, seed=77, scale=d ** -0.5)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    st = ctx.new_state(B)
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    for b, h in ((0, 0), (2, 17), (4, 19), (4, 31)):                     # (4, 19) and (4, 31): chains 147 and 159
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        want, wst = orc.prefill_quadratic(q[sl], k[sl], v[sl], w[h:h + 1], "elu1", 0.0)
+        assert rel_err(host(o[sl]), want) < TOL[io], (b, h)
+        assert rel_err(host(st.S[sl]), wst.S) < TOL[io] and rel_err(host(st.z[sl]), wst.z) < TOL[io]
+        np.testing.assert_array_equal(host(st.win[sl]), wst.win)
+    assert st.pos.tolist() == [T] * B
+
+
 @pytest.mark.parametrize("T1,T2,T3", [(20, 300, 9), (140, 17, 130)])
 def test_prefill_continuation_with_the_longest_tap_window(T1, T2, T3):
     """32 taps: the window carried between calls is longer than some of the pieces, and tiles after the first take
@@ -109,7 +126,8 @@ def test_prefill_continuation_with_the_longest_tap_window(T1, T2, T3):
 
 
 @pytest.mark.parametrize("T,W,phi,eps,init", [(2500, 3, "elu1", 0.0, False), (4099, 5, "relu", 1e-6, False),
-                                              (3000, 4, "elu1", 0.0, True), (2048, 1, "elu1", 0.0, False)])
+                                              (3000, 4, "elu1", 0.0, True), (2048, 1, "elu1", 0.0, False),
+                                              (2300, 32, "elu1", 0.0, True), (2200, 27, "relu", 1e-6, False)])
 def test_prefill_sequence_split_with_workspace(T, W, phi, eps, init):
     """Few chains and a long sequence: with a workspace the sequence is cut into segments run as separate CTAs."""
     io, B, H, d = "bf16", 1, 2, 128
