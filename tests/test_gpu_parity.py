@@ -247,6 +247,35 @@ def test_verify_matches_oracle_and_leaves_state_untouched(kernel, io, d, N, W, p
         assert torch.equal(a, b)
 
 
+def test_verify_every_tree_size():
+    """N = 1 .. 64 on the tensor-core path (rows past N are padding inside the kernel)."""
+    io, B, H, d, W = "bf16", 1, 2, 128, 3
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=64, max_depth=64)
+    ost, q, k, v, _, w = tree_case(io, B, H, d, 64, W, seed=123)
+    st = oracle_state_to_dev(ost, io)
+    for N in range(1, 65):
+        parent = np.stack([wl.random_tree(wl.rng(123, 4, N, 0), N, 6, 3)]).astype(np.int32)
+        qn, kn, vn = (np.ascontiguousarray(x[:, :, :N]) for x in (q, k, v))
+        o = ctx.la_verify_tree(dev(qn, io), dev(kn, io), dev(vn, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+        want = orc.verify_tree(qn, kn, vn, parent, w, "elu1", 0.0, ost)
+        assert rel_err(host(o), want) < TOL[io], N
+    assert ctx.la_last_device_status() == binding.LA_OK
+
+
+def test_prefill_lengths_around_the_tile_edges():
+    io, B, H, d, W = "bf16", 1, 2, 128, 3
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    q, k, v, w = make(io, B, H, d, 400, W, seed=321, scale=d ** -0.5)
+    for T in (1, 2, 3, 63, 64, 65, 126, 127, 128, 129, 130, 255, 256, 257, 383, 384, 385):
+        st = ctx.new_state(B)
+        cut = lambda x: dev(x[:, :, :T], io)
+        o = ctx.la_prefill(cut(q), cut(k), cut(v), dev(w, "f32"), st)
+        want, wst = orc.prefill_quadratic(q[:, :, :T], k[:, :, :T], v[:, :, :T], w, "elu1", 0.0)
+        assert rel_err(host(o), want) < TOL[io], T
+        check_state(st, wst, TOL[io])
+    assert ctx.la_last_device_status() == binding.LA_OK
+
+
 def test_verify_more_units_than_sms_with_one_bad_tree():
     """Several units per persistent CTA; one sequence in the middle carries an invalid tree."""
     io, B, H, d, N, W = "bf16", 48, 8, 128, 64, 4
