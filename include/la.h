@@ -175,6 +175,15 @@ la_status la_accept_greedy(la_ctx* ctx, int32_t B, int32_t N, const int32_t* par
                            const int32_t* pred_root, const int32_t* pred, int32_t* accept_node, int32_t* accept_len,
                            int32_t* next_token, void* stream);
 
+/* Self-test of the bounded waits.  (No counterpart in the paper.)  Every wait of a kernel of this library on a
+ * shared-memory barrier has a time limit, after which the kernel records LA_ERR_TIMEOUT in the status word and
+ * returns instead of hanging the GPU.  This call launches a one-CTA kernel that waits, through the same helper, on a
+ * barrier nobody arrives on, with a limit of limit_us microseconds (1 .. 1 000 000).  Afterwards
+ * la_last_device_status returns LA_ERR_TIMEOUT, *waited_ns (device pointer to one int64, may be null) holds the time
+ * the wait took, and the context is as usable as before (la_clear_device_status resets the status word).
+ */
+la_status la_selftest_wait_timeout(la_ctx* ctx, uint32_t limit_us, int64_t* waited_ns /*device*/, void* stream);
+
 /* Tree verification for callers that cannot allocate device memory.  (The paper has no
  * counterpart to this entry point; it exists for the way the library is embedded.)
  *

@@ -24,7 +24,7 @@ LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
-           "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy",
+           "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy", "la_selftest_wait_timeout",
            "la_prefill_workspace_bytes"]
 
 
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
         L.la_accept_greedy.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.la_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp, vp]
         L.la_verify_tree_noalloc.argtypes = [C.POINTER(la_config), i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state),
                                              vp, vp, vp]
         L.la_last_device_status.argtypes = [vp, vp]
@@ -229,6 +230,13 @@ class Context:
             _ptr(accept_len, torch.int32, (B,), "accept_len"), _ptr(next_token, torch.int32, (B,), "next_token"),
             _stream(stream)))
         return accept_node, accept_len, next_token
+
+    def la_selftest_wait_timeout(self, limit_us: int, stream=None) -> int:
+        """Runs the bounded-wait self-test; returns the nanoseconds the wait took (see include/la.h)."""
+        waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+        _check("la_selftest_wait_timeout", lib().la_selftest_wait_timeout(self._h, int(limit_us), waited.data_ptr(),
+                                                                          _stream(stream)))
+        return int(waited.item())
 
     def la_last_device_status(self, stream=None) -> int:
         return int(lib().la_last_device_status(self._h, _stream(stream)))

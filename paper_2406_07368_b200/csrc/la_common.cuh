@@ -23,6 +23,43 @@ template <int PHI> __device__ __forceinline__ float phi(float x) {
   return fmaxf(x, 0.f);
 }
 
+// ---- bounded waits on shared-memory barriers -------------------------------------------------
+// Every wait of a kernel on an mbarrier goes through mbar_wait: it returns false once `limit_ns` nanoseconds of
+// %globaltimer have passed (and raises the CTA's abort flag, so that every other waiter of the CTA gives up at its
+// next check), never spins without bound and never traps.  The kernel then records LA_ERR_TIMEOUT and leaves.
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second per wait
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+#pragma unroll 1
+    for (int it = 0; it < 64; ++it)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (global_ns() - t0 > limit_ns) {
+      *abort = 1;
+      return false;
+    }
+  }
+}
+
 // ---- programmatic dependent launch ----------------------------------------------------------
 // A kernel launched with launch_pdl() may start while its predecessor in the stream is still running (as SMs
 // become free), so that its launch latency and its set-up overlap the predecessor's tail.  Every thread calls

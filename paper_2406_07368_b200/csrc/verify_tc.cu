@@ -36,7 +36,6 @@ constexpr uint32_t V_BOX = (NMAX + 16) * 128;      // 64 draft rows + 16 window 
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t P_COL = 64, G_COL = 128;                // G_j at G_COL + 64 j
 __host__ __device__ constexpr uint32_t acc_col(int t) { return (t & 1) ? 384u : 0u; }   // acc of unit t
-constexpr unsigned long long kWaitLimitNs = 1000000000ull;
 
 // Small tables.  Those that group X writes and group Y reads exist twice (unit parity).
 struct alignas(16) Tab {
@@ -72,37 +71,6 @@ static_assert(offsetof(Tab, rden) % 16 == 0, "rden is read four at a time");
 static_assert(OFF_V % 1024 == 0 && V_BOX % 1024 == 0 && OFF_TAB % 16 == 0, "swizzled regions are 1024-byte aligned");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: false after one second (the CTA's abort flag is raised) or when another thread gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int it = 0; it < 64; ++it)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
-    if (global_ns() - t0 > kWaitLimitNs) {
-      *abort = 1;
-      return false;
-    }
-  }
-}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }

@@ -91,3 +91,19 @@ def test_repeated_calls_give_the_same_bits():
         results.append((o, ov, od, path, clen, st.S.clone(), st.z.clone(), st.win.clone(), st.pos.clone()))
     for a, b in zip(*results):
         assert torch.equal(a, b)
+
+
+def test_a_wait_that_nobody_ends_runs_out_and_reports_it():
+    """The bounded wait of the kernels, on a barrier nobody arrives on: it gives up after the limit, the status word
+    says so, and the context keeps working."""
+    ctx = binding.Context(2, 128, 3, "elu1", 0.0, "bf16")
+    assert ctx.la_last_device_status() == binding.LA_OK
+    waited = ctx.la_selftest_wait_timeout(20000)                     # 20 ms
+    assert ctx.la_last_device_status() == binding.LA_ERR_TIMEOUT
+    assert 20e6 <= waited < 200e6                                    # at least the limit, and not much more
+    ctx.la_clear_device_status()
+    assert ctx.la_last_device_status() == binding.LA_OK
+    st = ctx.new_state(1)
+    x = torch.randn(1, 2, 130, 128, device="cuda").bfloat16() * 0.1
+    o = ctx.la_prefill(x, x, x, torch.ones(2, 128, 3, device="cuda"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK and torch.isfinite(o.float()).all()
