@@ -125,7 +125,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// phi on two packed bf16 values, in packed arithmetic; the results are bf16 (and so exact as tf32 too).  elu + 1:
+// phi on two packed bf16 values, in packed arithmetic; the results are bf16.  elu + 1:
 // x + 1 where x > 0, 2^(x log2 e) elsewhere, merged with a lane mask.  ReLU: packed max.
 // 8 consecutive TMEM columns of this thread's lane; the caller waits once for all the loads it has issued.
 __device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, uint32_t* r) {
