@@ -225,8 +225,7 @@ la_status la_last_device_status(la_ctx* ctx, void* stream);
 la_status la_clear_device_status(la_ctx* ctx, void* stream);
 
 /* Selects the kernels of la_prefill and la_verify_tree: 0 = automatic (tensor-core kernels where
- * they apply: bf16 io, d = 128; for la_verify_tree also at most 4 live taps), 1 = always the fp32
- * CUDA-core kernels.  For testing one kernel against the other. */
+ * they apply: bf16 io, d = 128), 1 = always the fp32 CUDA-core kernels.  For testing one kernel against the other. */
 la_status la_set_prefill_kernel(la_ctx* ctx, int32_t which);
 
 /* Optional workspace for la_prefill.  With few (batch, head) chains and a long sequence -- fewer chains

@@ -1,4 +1,4 @@
-// Draft-tree verification on the tensor cores (bf16 io, d = 128, N <= 64, W <= 4).
+// Draft-tree verification on the tensor cores (bf16 io, d = 128, N <= 64).
 //
 // Sec. 4.2 / Sec. 5.3: all N draft nodes of a sequence share the committed state and attend, among the draft
 // tokens, to their ancestors and themselves only.  Per (sequence, head) unit everything that is a contraction
@@ -14,8 +14,9 @@
 //                                                                    that tap j of the causal convolution reads)
 // and the CUDA cores are left with phi, the tree walk, the mask, the denominators and
 //     o[n][c] = acc[c][n] / (phi(q_n) . z + sum_m Pm[n][m] + eps) + sum_j w[j][c] G_j[c][n].
-// Nothing of the state is written.  CTAs are persistent: group X prepares unit t + 1 while group Y finishes
-// unit t, and one thread feeds TMA and the tensor cores.
+// Taps beyond the fourth (W > 4) are added by the CUDA cores in the epilogue, from the same shared-memory copy of V
+// and a table of the rows they read.  Nothing of the state is written.  CTAs are persistent: group X prepares
+// unit t + 1 while group Y finishes unit t, and one thread feeds TMA and the tensor cores.
 #include <cuda.h>
 
 #include <algorithm>
@@ -27,12 +28,13 @@ namespace la {
 namespace vtc {
 
 constexpr int D = 128, NMAX = LA_MAX_NODES;
-constexpr int kMaxTaps = 4;                        // longer tap windows are served by the CUDA-core kernel
+constexpr int kMaxTaps = 4;                        // taps whose gathers run as tensor-core products
+constexpr int kExtTaps = LA_MAX_TAPS - kMaxTaps;   // the others: gathered by the CUDA cores in the epilogue
 constexpr int kThreadsX = 256, kThreadsY = 256, kCtrlWarp = 16, kTreeWarp = 17, kThreads = 576;
 constexpr uint32_t S_BYTES = 128 * 128 * 4;        // the fp32 state of one unit, row-major
 constexpr uint32_t SB_BOX = 128 * 128;             // 128 rows x 64 bf16
 constexpr uint32_t Q_BOX = NMAX * 128;             // 64 rows x 64 bf16
-constexpr uint32_t V_BOX = (NMAX + 16) * 128;      // 64 draft rows + 16 window rows x 64 bf16
+constexpr uint32_t V_BOX = (NMAX + 32) * 128;      // 64 draft rows + 32 window rows (newest first) x 64 bf16
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t P_COL = 64, G_COL = 128;                // G_j at G_COL + 64 j
 __host__ __device__ constexpr uint32_t acc_col(int t) { return (t & 1) ? 384u : 0u; }   // acc of unit t
@@ -46,6 +48,7 @@ struct alignas(16) Tab {
   float den_part[2][NMAX];                         // masked row sums of P, one per column half
   float rden[NMAX];                                // 1 / (denominator + eps)
   int par[NMAX];                                   // the parent array (private to the tree warp)
+  unsigned char ext[2][kExtTaps][NMAX];            // row of the V copy that tap 4 + j of node n reads (W > 4 only)
 };
 struct alignas(16) Ctl {
   unsigned long long bars[12];
@@ -160,7 +163,7 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 //   warp 17              unit t: walks the tree; writes the tree masks, the selection matrices and the window rows;
 //   warp 16 (one lane)   TMA of S and V; every tcgen05.mma;
 //   group Y (warps 8-15) masks the scores, forms the denominators, and writes the outputs.
-template <int PHI>
+template <int PHI, bool EXT>   // EXT: more than kMaxTaps live taps
 __global__ void __launch_bounds__(kThreads, 1)
 verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__ CUtensorMap mv,
                  const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -198,8 +201,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
   // selection matrices and masked scores start as zeros; so do the 16 window rows below the draft rows of V
   for (uint32_t i = tid; i < (OFF_TAB - OFF_SEL) / 16; i += kThreads)
     *reinterpret_cast<uint4*>(smem + OFF_SEL + i * 16) = make_uint4(0u, 0u, 0u, 0u);
-  for (uint32_t i = tid; i < 2 * 16 * 128 / 16; i += kThreads)
-    *reinterpret_cast<uint4*>(smem + OFF_V + (i >> 7) * V_BOX + NMAX * 128 + (i & 127) * 16) = make_uint4(0u, 0u, 0u, 0u);
+  for (uint32_t i = tid; i < 2 * 32 * 128 / 16; i += kThreads)
+    *reinterpret_cast<uint4*>(smem + OFF_V + (i >> 8) * V_BOX + NMAX * 128 + (i & 255) * 16) = make_uint4(0u, 0u, 0u, 0u);
   if (warp == kCtrlWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl.tmem_base)),
                  "r"(TMEM_COLS)
@@ -268,7 +271,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         if (good) {
           // G_j[c][n], the value tap j reads for node n, for all taps at once: the selection matrices lie one after
           // the other, so they form one operand of 64 W rows and the products land in 64 W consecutive columns
-          const uint32_t idG = idesc(true, false, 64u * (uint32_t)W);
+          const uint32_t idG = idesc(true, false, 64u * (uint32_t)min(W, kMaxTaps));
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)       // 16 draft rows per step
             mma(tmem + G_COL, smem_desc(sbase + OFF_V + kk * 2048u, V_BOX, 1024u, 2u),
@@ -287,7 +290,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
                 smem_desc(sbase + OFF_PM + kk * 32u, 16u, 1024u, 2u), kIdV, true);
         }
         mma_commit(bar[B_O]);
-        if (!mbar_wait(bar[B_O], par, abort)) break;       // V has been read
+        if (!mbar_wait(bar[B_O], par, abort)) break;       // V has been read by the tensor cores
+        // with more than four taps the epilogue of this unit reads V too
+        if (EXT && !mbar_wait(bar[B_EPI], par, abort)) break;
         if (t + 1 < nloc) load_v(t + 1);
       }
     }
@@ -303,11 +308,12 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       const int u = (int)blockIdx.x + t * (int)gridDim.x, b = u / H, par = t & 1;
       tab.par[lane] = lane < N ? parent[(size_t)b * N + lane] : -1;
       tab.par[lane + 32] = lane + 32 < N ? parent[(size_t)b * N + lane + 32] : -1;
-      uint32_t wv[6];                                       // the committed window: (W - 1) rows of 128 channels
+      uint32_t wv[6];                                       // the committed window (up to three rows: W <= 4) in flight early
 #pragma unroll
       for (int i = 0; i < 6; ++i) {
         const int idx = lane + 32 * i;
-        wv[i] = idx < 64 * (W - 1) ? *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx) : 0u;
+        wv[i] = (!EXT && idx < 64 * (W - 1)) ? *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx)
+                                                      : 0u;
       }
       __syncwarp();
       // ---- each lane follows the parents of its two nodes (integer work) ----
@@ -337,6 +343,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       // ---- the selection matrices and the window rows of unit t - 1 have been consumed (and with them everything
       //      issued before: this parity's tables were last read two units ago) ----
       if (t >= 1) ok = ok && mbar_wait(bar[B_SG], (t - 1) & 1, abort);
+      // with more than four taps the epilogue of unit t - 1 reads the window rows and the V copy as well
+      if (EXT && t >= 1) ok = ok && mbar_wait(bar[B_EPI], (t - 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         if (lane == 0) tab.bad[par] = bad_any ? 1 : 0;
@@ -353,18 +361,41 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
               if (j < depth[s2]) {
                 const int a = anc[s2][j - 1];
                 pv = OFF_SEL + j * Q_BOX + swz(n, a >> 3) + (a & 7) * 2;
-              } else {                                      // behind the chain: the committed window, newest row last
-                pv = OFF_SELW + selw_offset(64 * j + n, (W - 2) - (j - depth[s2]));
+              } else {                                      // behind the chain: the committed window, newest row first
+                pv = OFF_SELW + selw_offset(64 * j + n, j - depth[s2]);
               }
               *reinterpret_cast<unsigned short*>(smem + pv) = 0x3F80;
             }
           }
         }
+        // the window below the draft rows of both channel halves, newest row first: row NMAX + p holds the value
+        // p + 1 steps behind the first draft token
+        if (!EXT) {
 #pragma unroll
-        for (int i = 0; i < 6; ++i) {                        // window row r of both channel halves, below the draft rows
-          const int idx = lane + 32 * i, r = idx >> 6, c2 = (idx & 63) * 2;
-          if (idx < 64 * (W - 1))
-            *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + r, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv[i];
+          for (int i = 0; i < 6; ++i) {
+            const int idx = lane + 32 * i, p = (W - 2) - (idx >> 6), c2 = (idx & 63) * 2;
+            if (idx < 64 * (W - 1))
+              *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + p, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv[i];
+          }
+        } else {
+          for (int idx = lane; idx < 64 * (W - 1); idx += 32) {
+            const int p = (W - 2) - (idx >> 6), c2 = (idx & 63) * 2;
+            *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + p, (c2 & 63) >> 3) + (c2 & 7) * 2) =
+                *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx);
+          }
+          // rows that the taps beyond the fourth read: a second walk, now that this parity's table is free
+          for (int s2 = 0; s2 < 2; ++s2) {
+            const int n = lane + 32 * s2;
+            if (n < N && !bad_any) {
+              int m = n, kk = 0;
+              for (; m >= 0 && kk < W; ++kk) {
+                if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned char)m;
+                m = tab.par[m];
+              }
+              for (; kk < W; ++kk)                         // behind the chain: window rows, newest first
+                if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned char)(NMAX + kk - depth[s2]);
+            }
+          }
         }
       }
       proxy_fence();
@@ -532,6 +563,19 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
 #pragma unroll
               for (int i = 0; i < 8; ++i) out[i] = fmaf(wt[j], __uint_as_float(rg[j][i]), out[i]);
             }
+          // taps beyond the fourth: the value comes straight from the shared-memory copy of V (draft rows, then
+          // window rows), at the row the tree warp tabulated
+          for (int j = kMaxTaps; EXT && j < W; ++j) {
+            const float wj = w[((size_t)h * D + c) * W + j];
+            const unsigned char* vcol = smem + OFF_V + (c >> 6) * V_BOX + (c & 7) * 2;
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              if (nb + i < N) {
+                const int row = tab.ext[par][j - kMaxTaps][nb + i];
+                const __nv_bfloat16 x = *reinterpret_cast<const __nv_bfloat16*>(vcol + swz(row, (c & 63) >> 3));
+                out[i] = fmaf(wj, __bfloat162float(x), out[i]);
+              }
+          }
           // Two neighbouring lanes trade values so that each stores two adjacent channels of one node: the even
           // lane takes node nb + i, the odd lane node nb + i + 1.
 #pragma unroll
@@ -592,7 +636,7 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
                              bool* handled) {
   const la_config& c = ctx->cfg;
   *handled = false;
-  if (c.io_dtype != LA_BF16 || c.d != vtc::D || c.conv_taps > vtc::kMaxTaps) return cudaSuccess;
+  if (c.io_dtype != LA_BF16 || c.d != vtc::D) return cudaSuccess;
   vtc::EncodeTiledFn fn = vtc::encode_fn();
   if (!fn) return cudaSuccess;
   const int BH = B * c.H;
@@ -617,7 +661,10 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return cudaSuccess;
   }
-  auto kern = c.phi == LA_PHI_ELU1 ? vtc::verify_tc_kernel<LA_PHI_ELU1> : vtc::verify_tc_kernel<LA_PHI_RELU>;
+  const bool elu = c.phi == LA_PHI_ELU1;
+  auto kern = c.conv_taps <= vtc::kMaxTaps
+                  ? (elu ? vtc::verify_tc_kernel<LA_PHI_ELU1, false> : vtc::verify_tc_kernel<LA_PHI_RELU, false>)
+                  : (elu ? vtc::verify_tc_kernel<LA_PHI_ELU1, true> : vtc::verify_tc_kernel<LA_PHI_RELU, true>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vtc::kSmemBytes);
   if (e != cudaSuccess) return e;
   e = launch_pdl(kern, dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), vtc::kSmemBytes, s, ms, mv,

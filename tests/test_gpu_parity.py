@@ -230,7 +230,9 @@ def tree_case(io, B, H, d, N, W, seed, phi="elu1", eps=0.0, chain=False):
     ("bf16", 128, 1, 3, "elu1", 0.0, False), ("f32", 128, 64, 9, "elu1", 0.0, False),
     ("bf16", 128, 20, 32, "elu1", 0.0, True), ("bf16", 128, 16, 1, "elu1", 0.0, False),
     ("bf16", 128, 64, 4, "relu", 1e-6, True), ("bf16", 128, 37, 2, "relu", 1e-6, False),
-    ("bf16", 128, 50, 4, "elu1", 0.0, False), ("bf16", 128, 33, 4, "elu1", 1e-6, True)])
+    ("bf16", 128, 50, 4, "elu1", 0.0, False), ("bf16", 128, 33, 4, "elu1", 1e-6, True),
+    ("bf16", 128, 64, 8, "elu1", 0.0, False), ("bf16", 128, 64, 32, "elu1", 1e-6, False),
+    ("bf16", 128, 3, 6, "relu", 1e-6, True), ("bf16", 128, 64, 17, "relu", 0.0, True)])
 @pytest.mark.parametrize("kernel", [0, 1])
 def test_verify_matches_oracle_and_leaves_state_untouched(kernel, io, d, N, W, phi, eps, chain):
     B, H = 3, 2
@@ -276,9 +278,10 @@ def test_prefill_lengths_around_the_tile_edges():
     assert ctx.la_last_device_status() == binding.LA_OK
 
 
-def test_verify_more_units_than_sms_with_one_bad_tree():
+@pytest.mark.parametrize("W", [4, 7])
+def test_verify_more_units_than_sms_with_one_bad_tree(W):
     """Several units per persistent CTA; one sequence in the middle carries an invalid tree."""
-    io, B, H, d, N, W = "bf16", 48, 8, 128, 64, 4
+    io, B, H, d, N = "bf16", 48, 8, 128, 64
     ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=97, phi="relu", eps=1e-6)
     ctx = binding.Context(H, d, W, "relu", 1e-6, io, max_nodes=64, max_depth=64)
     st = oracle_state_to_dev(ost, io)
