@@ -3,19 +3,19 @@
 // Sec. 4.1: the sequence is cut into non-overlapping groups; inside a group the causally
 // masked product phi(Q) phi(K)^T V is formed in parallel, between groups only the cumulative
 // sums S = sum phi(k) v^T and z = sum phi(k) are carried.  One CTA walks one (batch, head)
-// chain in tiles of 128 tokens.  The normaliser rides along on the tensor cores: V is
-// extended by a column of ones and S by the column z, so that
-//     [O | den] = phi(Q) [S | z]_prev + (P o M) [V | 1],     [S | z] += phi(K)^T [V | 1].
-// Per tile n:
+// chain in tiles of 128 tokens:
+//     O = phi(Q) S_prev + (P o M) V,   den = phi(Q) . z_prev + rowsum(P o M),   S += phi(K)^T V,   z += colsum phi(K).
+// The four matrix products run on the tensor cores; the normaliser (two vectors per tile) is formed by the
+// threads that hold phi(Q), phi(K) and P in registers anyway.  Per tile n:
 //
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
-//   group A  phi applied in place on Q and K (packed bf16x2 arithmetic, fp32 exp)
+//   group A  phi applied in place on Q and K (packed bf16x2 arithmetic); phi(q) . z_prev; z += colsum phi(K)
 //   tcgen05  P = phi(Q) phi(K)^T
-//            [S | z] += phi(K)^T [V | 1]     (fp32 in TMEM for the whole chain)
-//            [O | den] = phi(Q) [S | z]_prev  ([S | z]_prev is a bf16 copy in shared memory)
-//   group A  P -> causal mask, bf16 -> TMEM (the A operand of the next product);
-//            phi on K of tile n+1 (K is double-buffered);  [S | z] -> bf16 copy for tile n+1
-//   tcgen05  [O | den] += (P o M) [V | 1]
+//            S += phi(K)^T V                 (fp32 in TMEM for the whole chain)
+//            O = phi(Q) S_prev               (S_prev is a bf16 copy in shared memory)
+//   group A  P -> causal mask, row sums, bf16 -> TMEM (the A operand of the next product);
+//            phi on K of tile n+1 (K is double-buffered);  S -> bf16 copy for tile n+1
+//   tcgen05  O += (P o M) V
 //   group B  o = O / (den + eps) + conv(V) -> global memory
 //
 // Three roles run concurrently: group A (warps 8-15), group B (warps 0-7) and warp 16, whose
@@ -39,29 +39,36 @@ constexpr int kCtrlWarp = 16;
 constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns: P, O, S (128 each, fp32), two 16-column blocks whose first column is den and z, and the
-// masked P as packed bf16 pairs (64 columns).
-constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, DEN_COL = 384, Z_COL = 400, P16_COL = 416, TMEM_COLS = 512;
+// TMEM columns (all 512): P, two O accumulators (tiles alternate, so that the epilogue of one tile runs beside the
+// products of the next) and S, 128 fp32 columns each.  The masked P goes back as packed bf16 pairs into the columns
+// its own fp32 values came from: each thread overwrites only columns of its own row that it has already read
+// (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
+constexpr uint32_t P_COL = 0, O_COL = 128 /* and 256 */, S_COL = 384, TMEM_COLS = 512;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0, OFF_K0 = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
                    OFF_K1 = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
-                   OFF_ONES = 6 * TILE_BYTES,      // [128 x 16] bf16, column 0 = 1: the extension of V
-                   OFF_SZ = OFF_ONES + 4096,       // [128 x 16] bf16, column 0 = z: the extension of the S copy
-                   OFF_SMALL = OFF_SZ + 4096;
+                   OFF_ZBUF = 6 * TILE_BYTES,      // [2][128] fp32: z before even / odd tiles
+                   OFF_KPART = OFF_ZBUF + 1024,    // [8][128] fp32: column sums of phi(K), one row per warp
+                   OFF_DEN = OFF_KPART + 4096,     // [4][2][128] fp32: halves of the denominators of tile n in slot n & 3
+                   OFF_SMALL = OFF_DEN + 4096;
 
 struct Small {
-  unsigned long long bars[16];
+  unsigned long long bars[20];
   uint32_t tmem_base;
   int abort;
   int pad[2];
 };
-// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI: arrivals of group B (O has been read).
-// VFREE: the outputs staged in a V buffer have left it (one arrival by the thread that issued the TMA store).
-// MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T[V|1] (K buffer free);
-// after [O|den] = phi(Q)[S|z] (Q buffer free); after [O|den] += P[V|1].
-enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O = 5, B_PHI = 6, B_PDONE = 7,
-       B_SB = 8, B_EPI = 9, B_MMA_Q = 10, B_FULL_Q = 11, B_FULL_K1 = 12, B_VFREE = 13, kNumBars = 14 };
+// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI0 / EPI1: arrivals of group B (that O
+// accumulator has been read).
+// STAGED0 / STAGED1: group B has written a tile's outputs into that V buffer (the control lane stores them).
+// MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after S += phi(K)^T V (K buffer free);
+// after O = phi(Q) S (Q buffer free); after O += P V (MMA_O0 / MMA_O1, one per accumulator).
+// A barrier that one role waits on while another role can run a tile ahead exists once per accumulator, so that a
+// waiter is never more than one phase behind.
+enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O0 = 5, B_MMA_O1 = 6, B_PHI = 7,
+       B_PDONE = 8, B_SB = 9, B_EPI0 = 10, B_EPI1 = 11, B_MMA_Q = 12, B_FULL_Q = 13, B_FULL_K1 = 14, B_STAGED0 = 15,
+       B_STAGED1 = 16, kNumBars = 17 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
@@ -89,6 +96,11 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void sync_group_b() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
+__device__ __forceinline__ void sync_group_a() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void sync_half_b(int hf) {
+  if (hf) asm volatile("bar.sync 4, 128;" ::: "memory");
+  else asm volatile("bar.sync 3, 128;" ::: "memory");
+}
 
 __device__ __forceinline__ void tma_load(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
   asm volatile(
@@ -192,6 +204,16 @@ __device__ __forceinline__ uint64_t desc_ext(uint32_t tile, int ks) {
 __device__ __forceinline__ uint32_t ext_offset(int k, int n) {   // byte offset of element (k, n) in such a block
   return (uint32_t)(k >> 3) * 256u + (uint32_t)(n >> 3) * 128u + (uint32_t)(k & 7) * 16u + (uint32_t)(n & 7) * 2u;
 }
+// The same descriptors split into their two 32-bit words: the steps of a product differ only in the start-address
+// field of the low word (by a constant, and the field cannot overflow below 256 KB), so the issuing lane forms the
+// words of step 0 once per tile and adds a constant per step.
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+constexpr uint32_t kDescHiSw128 = ((1024u >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
+__host__ __device__ constexpr uint32_t kstep_kmajor(int ks) { return ((uint32_t)(ks >> 2) * BOX_BYTES + (uint32_t)(ks & 3) * 32u) >> 4; }
+__host__ __device__ constexpr uint32_t kstep_mnmajor(int ks) { return ((uint32_t)ks * 2048u) >> 4; }
+__device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n.
 __host__ __device__ constexpr uint32_t idesc(bool a_mn, bool b_mn, uint32_t n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
@@ -282,26 +304,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const int u = blockIdx.x, bh = u / nseg, h = bh % H;
   const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
   const int nchunks = (T + TILE - 1) / TILE;
-  uint32_t bar[kNumBars];
-#pragma unroll
-  for (int i = 0; i < kNumBars; ++i) bar[i] = smem_u32(&sm.bars[i]);
+  const uint32_t bar0 = smem_u32(&sm.bars[0]);    // barrier i lives at bar0 + 8 i
 
   // ---- set-up ----
   if (tid == 0) {
-    mbar_init(bar[B_FULL_K0], 1);
-    mbar_init(bar[B_FULL_K1], 1);
-    mbar_init(bar[B_FULL_Q], 1);
-    mbar_init(bar[B_FULL_V0], 1);
-    mbar_init(bar[B_FULL_V1], 1);
-    mbar_init(bar[B_MMA_P], 1);
-    mbar_init(bar[B_MMA_S], 1);
-    mbar_init(bar[B_MMA_O], 1);
-    mbar_init(bar[B_PHI], kThreadsA);
-    mbar_init(bar[B_PDONE], kThreadsA);
-    mbar_init(bar[B_SB], kThreadsA);
-    mbar_init(bar[B_EPI], kThreadsB);
-    mbar_init(bar[B_MMA_Q], 1);
-    mbar_init(bar[B_VFREE], 1);
+    mbar_init((bar0 + 8u * (B_FULL_K0)), 1);
+    mbar_init((bar0 + 8u * (B_FULL_K1)), 1);
+    mbar_init((bar0 + 8u * (B_FULL_Q)), 1);
+    mbar_init((bar0 + 8u * (B_FULL_V0)), 1);
+    mbar_init((bar0 + 8u * (B_FULL_V1)), 1);
+    mbar_init((bar0 + 8u * (B_MMA_P)), 1);
+    mbar_init((bar0 + 8u * (B_MMA_S)), 1);
+    mbar_init((bar0 + 8u * (B_MMA_O0)), 1);
+    mbar_init((bar0 + 8u * (B_MMA_O1)), 1);
+    mbar_init((bar0 + 8u * (B_PHI)), kThreadsA);
+    mbar_init((bar0 + 8u * (B_PDONE)), kThreadsA);
+    mbar_init((bar0 + 8u * (B_SB)), kThreadsA);
+    mbar_init((bar0 + 8u * (B_EPI0)), kThreadsB);
+    mbar_init((bar0 + 8u * (B_EPI1)), kThreadsB);
+    mbar_init((bar0 + 8u * (B_MMA_Q)), 1);
+    mbar_init((bar0 + 8u * (B_STAGED0)), kThreadsB);
+    mbar_init((bar0 + 8u * (B_STAGED1)), kThreadsB);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -314,14 +337,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
     halo0[idx] = init ? win[(size_t)u * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
-  for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
-    reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
-  __syncthreads();
-  if (tid < TILE) {
-    *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
-    if (init)
-      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)u * D + tid]);
-  }
+  float* zbuf = reinterpret_cast<float*>(smem + OFF_ZBUF);      // zbuf[m & 1]: z before tile m
+  float* kpart = reinterpret_cast<float*>(smem + OFF_KPART);
+  float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
+  if (tid < D) zbuf[tid] = init ? z[(size_t)u * D + tid] : 0.f;
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -332,109 +351,115 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     // =============================== TMA + MMA issue (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx(bar[B_FULL_K0], TILE_BYTES);
-      tma_load(sbase + OFF_K0, &mk, 0, y0, bh, bar[B_FULL_K0]);
-      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, y0, bh, bar[B_FULL_K0]);
+      mbar_expect_tx((bar0 + 8u * (B_FULL_K0)), TILE_BYTES);
+      tma_load(sbase + OFF_K0, &mk, 0, y0, bh, (bar0 + 8u * (B_FULL_K0)));
+      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, y0, bh, (bar0 + 8u * (B_FULL_K0)));
       if (nchunks > 1) {
-        mbar_expect_tx(bar[B_FULL_K1], TILE_BYTES);
-        tma_load(sbase + OFF_K1, &mk, 0, y0 + TILE, bh, bar[B_FULL_K1]);
-        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, y0 + TILE, bh, bar[B_FULL_K1]);
+        mbar_expect_tx((bar0 + 8u * (B_FULL_K1)), TILE_BYTES);
+        tma_load(sbase + OFF_K1, &mk, 0, y0 + TILE, bh, (bar0 + 8u * (B_FULL_K1)));
+        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, y0 + TILE, bh, (bar0 + 8u * (B_FULL_K1)));
       }
-      mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
-      tma_load(sbase + OFF_Q, &mq, 0, y0, bh, bar[B_FULL_Q]);
-      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0, bh, bar[B_FULL_Q]);
+      mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
+      tma_load(sbase + OFF_Q, &mq, 0, y0, bh, (bar0 + 8u * (B_FULL_Q)));
+      tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0, bh, (bar0 + 8u * (B_FULL_Q)));
       for (int n = 0; n < 2 && n < nchunks; ++n) {
-        mbar_expect_tx(bar[B_FULL_V0 + n], TILE_BYTES);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, bar[B_FULL_V0 + n]);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, bar[B_FULL_V0 + n]);
+        mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + n)), TILE_BYTES);
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
       }
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
         const uint32_t vbuf = sbase + OFF_V0 + par * TILE_BYTES;
         const uint32_t kbuf = sbase + (par ? OFF_K1 : OFF_K0);
-        const uint32_t kbar = bar[par ? B_FULL_K1 : B_FULL_K0];
+        const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
         const bool has_state = init || n > 0;
-        ok = mbar_wait(bar[B_PHI], par, abort);                 // phi(Q), phi(K) of tile n are in place
+        const uint32_t ocol = tmem + O_COL + par * 128u;        // this tile's accumulator
+        // low descriptor words of step 0: Q and K read along their rows (K-major), K, V and the S copy down their rows
+        const uint32_t q_km = desc_lo(sbase + OFF_Q, 16u), k_km = desc_lo(kbuf, 16u);
+        const uint32_t k_mn = desc_lo(kbuf, BOX_BYTES), v_mn = desc_lo(vbuf, BOX_BYTES), s_mn = desc_lo(sbase + OFF_S, BOX_BYTES);
+        ok = mbar_wait((bar0 + 8u * (B_PHI)), par, abort);                 // phi(Q), phi(K) of tile n are in place
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T
-          mma_bf16(tmem + P_COL, desc_kmajor(sbase + OFF_Q, ks), desc_kmajor(kbuf, ks),
+          mma_bf16(tmem + P_COL, desc64(q_km + kstep_kmajor(ks)), desc64(k_km + kstep_kmajor(ks)),
                    idesc(false, false, 128), ks > 0);
-        mma_commit(bar[B_MMA_P]);
-        // the bf16 copy of [S|z] before tile n is complete (and S itself has been read) after n + 1 arrivals
-        ok = mbar_wait(bar[B_SB], par, abort) && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
+        mma_commit((bar0 + 8u * (B_MMA_P)));
+        // the bf16 copy of S before tile n is complete (and S itself has been read) after n + 1 arrivals; the
+        // accumulator is free once the epilogue of tile n-2 has read it
+        ok = mbar_wait((bar0 + 8u * (B_SB)), par, abort);
+        if (ok && n >= 2) ok = mbar_wait((bar0 + 8u * (B_EPI0 + par)), ((n >> 1) - 1) & 1, abort);
         if (!ok) break;
         tc_fence_after();
-        // Two chains decide the pace: the epilogue of tile n-1 -> [O|den] = phi(Q)[S|z] -> [O|den] += P[V|1] -> the
-        // epilogue of tile n; and the last read of the Q buffer -> its reload -> phi -> the products of tile n+1.
-        // Both start with the product on phi(Q), which has to wait for the epilogue of tile n-1; the state update
-        // [S|z] += phi(K)^T[V|1] is needed much later, so its steps only fill the time until that epilogue is done.
-        int s_steps = 0;
-        auto issue_s = [&](int upto) {
-          for (; s_steps < upto; ++s_steps) {
-            const uint64_t kd = desc_mnmajor(kbuf, s_steps);
-            mma_bf16(tmem + S_COL, kd, desc_mnmajor(vbuf, s_steps), idesc(true, true, 128), has_state || s_steps > 0);
-            mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, s_steps), idesc(true, true, 16), has_state || s_steps > 0);
-          }
-        };
-        if (n >= 1) {
-          while (!mbar_try_wait(bar[B_EPI], (n - 1) & 1)) {
-            if (s_steps < 8) {
-              issue_s(s_steps + 1);
-            } else {
-              ok = mbar_wait(bar[B_EPI], (n - 1) & 1, abort);
-              break;
-            }
-          }
-          if (!ok) break;
-          tc_fence_after();
-        }
         if (has_state) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {   // [O | den] = phi(Q) [S | z]_prev
-            const uint64_t qd = desc_kmajor(sbase + OFF_Q, ks);
-            mma_bf16(tmem + O_COL, qd, desc_mnmajor(sbase + OFF_S, ks), idesc(false, true, 128), ks > 0);
-            mma_bf16(tmem + DEN_COL, qd, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
-          }
+          for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
+            mma_bf16(ocol, desc64(q_km + kstep_kmajor(ks)), desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128),
+                     ks > 0);
         }
-        mma_commit(bar[B_MMA_Q]);
-        ok = mbar_wait(bar[B_PDONE], par, abort);               // masked P of tile n is in TMEM
+        mma_commit((bar0 + 8u * (B_MMA_Q)));
+        // The single Q buffer sets the pace (last read -> reload -> phi -> products of the next tile), so its reload
+        // goes out as soon as the two products that read it are complete, ahead of the state update.
+        if (n + 1 < nchunks) {
+          ok = mbar_wait((bar0 + 8u * (B_MMA_Q)), par, abort);             // the Q buffer is free
+          if (!ok) break;
+          mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
+          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
+          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
+        }
+        ok = mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
+        if (!ok) break;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)       // S += phi(K)^T V
+          mma_bf16(tmem + S_COL, desc64(k_mn + kstep_mnmajor(ks)), desc64(v_mn + kstep_mnmajor(ks)), idesc(true, true, 128),
+                   has_state || ks > 0);
+        mma_commit((bar0 + 8u * (B_MMA_S)));
+        ok = mbar_wait((bar0 + 8u * (B_PDONE)), par, abort);               // masked P of tile n is in TMEM
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {     // [O | den] += (P o M) [V | 1]
-          const uint32_t pa = tmem + P16_COL + 8 * ks;       // 16 values of every row = 8 columns
-          mma_bf16_ts(tmem + O_COL, pa, desc_mnmajor(vbuf, ks), idesc(false, true, 128), has_state || ks > 0);
-          mma_bf16_ts(tmem + DEN_COL, pa, desc_ext(sbase + OFF_ONES, ks), idesc(false, true, 16), has_state || ks > 0);
-        }
-        mma_commit(bar[B_MMA_O]);
-        if (n + 1 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_Q], par, abort);             // the Q buffer is free
-          if (!ok) break;
-          mbar_expect_tx(bar[B_FULL_Q], TILE_BYTES);
-          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
-          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_Q]);
-        }
-        issue_s(8);                          // the rest of [S | z] += phi(K)^T [V | 1]
-        mma_commit(bar[B_MMA_S]);
-        if (n >= 1 && n + 1 < nchunks) {
-          // the outputs of tile n-1, staged in its V buffer, have left: the buffer takes tile n+1
-          ok = mbar_wait(bar[B_VFREE], (n - 1) & 1, abort);
-          if (!ok) break;
-          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
-          mbar_expect_tx(bar[B_FULL_V0 + (par ^ 1)], TILE_BYTES);
-          tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-          tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, bar[B_FULL_V0 + (par ^ 1)]);
-        }
+        for (int ks = 0; ks < 8; ++ks)       // O += (P o M) V; 16 tokens of every row of P = 8 columns
+          mma_bf16_ts(ocol, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
+                      idesc(false, true, 128), has_state || ks > 0);
+        mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
         if (n + 2 < nchunks) {
-          ok = mbar_wait(bar[B_MMA_S], par, abort);             // this K buffer is free: it takes tile n+2
+          ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);             // this K buffer is free: it takes tile n+2
           if (!ok) break;
           mbar_expect_tx(kbar, TILE_BYTES);
           tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
           tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
         }
+        if (n >= 1) {
+          // the outputs of tile n-1 are staged in its V buffer: store them; once they have been read the buffer
+          // takes tile n+1
+          ok = mbar_wait((bar0 + 8u * (B_STAGED0 + (par ^ 1))), ((n - 1) >> 1) & 1, abort);
+          if (!ok) break;
+          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
+          tma_store(&mo, 0, y0 + (n - 1) * TILE, bh, vnext);    // rows past the end of the sequence are clipped
+          tma_store(&mo, 64, y0 + (n - 1) * TILE, bh, vnext + BOX_BYTES);
+          tma_commit();
+          if (n + 1 < nchunks) {
+            tma_wait_read();
+            mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + (par ^ 1))), TILE_BYTES);
+            tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + (par ^ 1))));
+            tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + (par ^ 1))));
+          }
+        }
+        // P of the next tile overwrites the columns that the last product of this tile reads
+        ok = mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);
+        if (!ok) break;
       }
+      if (ok) {   // the outputs of the last tile
+        const int n = nchunks - 1;
+        ok = mbar_wait((bar0 + 8u * (B_STAGED0 + (n & 1))), (n >> 1) & 1, abort);
+        if (ok) {
+          const uint32_t src = sbase + OFF_V0 + (n & 1) * TILE_BYTES;
+          tma_store(&mo, 0, y0 + n * TILE, bh, src);
+          tma_store(&mo, 64, y0 + n * TILE, bh, src + BOX_BYTES);
+          tma_commit();
+        }
+      }
+      tma_wait_all();                             // every store is complete before the CTA exits
     }
   } else if (warp >= 8) {
     // =============================== group A: phi, P, [S|z] snapshot (256 threads) ===============================
@@ -448,7 +473,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     float* Sg = S + (size_t)u * D * D + (size_t)r * D + 64 * hf;
     bool ok = true;
 
-    if (init) {   // [S|z] -> TMEM (fp32); S -> bf16 copy in shared memory (z was copied during set-up)
+    if (init) {   // S -> TMEM (fp32) and bf16 copy in shared memory (z was copied during set-up)
 #pragma unroll
       for (int qq = 0; qq < 2; ++qq) {
         uint32_t v[32];
@@ -462,52 +487,88 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
         for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
       }
-      if (hf == 0) {
-        tmem_st1(tmem + lane_addr + Z_COL, __float_as_uint(z[(size_t)u * D + r]));
-#pragma unroll
-        for (int c = 1; c < 16; ++c) tmem_st1(tmem + lane_addr + Z_COL + c, 0u);
-      }
       tmem_wait_st();
     }
     fence_proxy_async();
     tc_fence_before();
-    mbar_arrive(bar[B_SB]);                       // phase 0: the state before tile 0 is in place
+    mbar_arrive((bar0 + 8u * (B_SB)));                       // phase 0: the state before tile 0 is in place
 
-    // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero
-    auto phi_k = [&](int m) {
-      const int valid = min(TILE, T - m * TILE);
+    // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero.  The column
+    // sums of the result advance z: zbuf[(m+1) & 1] = zbuf[m & 1] + colsum (eight rows per thread, the two row
+    // groups of a warp by shuffle, the eight warps through shared memory).
+    // Every warp of the group calls it, also after a wait has run out (go = false: no work, same barrier).
+    auto phi_k = [&](int m, bool go) {
+      const int valid = go ? min(TILE, T - m * TILE) : 0;
       const int ct = ta & 15, rg = ta >> 4;                     // chunk column 0..15, row group 0..15
       unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * BOX_BYTES;
+      float cs[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) cs[e] = 0.f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int j = rg + 16 * i;
         uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-        *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+        const uint4 x = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+        if (go) *p = x;
+        cs[0] += lo_f(x.x); cs[1] += hi_f(x.x); cs[2] += lo_f(x.y); cs[3] += hi_f(x.y);
+        cs[4] += lo_f(x.z); cs[5] += hi_f(x.z); cs[6] += lo_f(x.w); cs[7] += hi_f(x.w);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], 16);
+      if (lane < 16) {
+        float4* dst = reinterpret_cast<float4*>(kpart + wa * D + 8 * ct);
+        dst[0] = make_float4(cs[0], cs[1], cs[2], cs[3]);
+        dst[1] = make_float4(cs[4], cs[5], cs[6], cs[7]);
+      }
+      sync_group_a();
+      if (ta < D) {
+        float acc = zbuf[(m & 1) * D + ta];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc += kpart[i * D + ta];
+        zbuf[((m + 1) & 1) * D + ta] = acc;
       }
     };
-    ok = mbar_wait(bar[B_FULL_K0], 0, abort);
+    ok = mbar_wait((bar0 + 8u * (B_FULL_K0)), 0, abort);
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) phi_k(0);
+    phi_k(0, ok);
 
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
       const bool last = n + 1 == nchunks;
 
       // ---- phi on Q in place (phi on K of this tile was done one iteration earlier) ----
-      ok = ok && mbar_wait(bar[B_FULL_Q], par, abort);
+      ok = ok && mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
+      uint4 fq[8];                                // phi(q) of row r, this thread's 64 channels
       if (ok) {
 #pragma unroll
         for (int cc = 0; cc < 8; ++cc) {
           uint4* p = reinterpret_cast<uint4*>(Qb + swz(r, cc));
-          *p = phi8<PHI>(*p);
+          fq[cc] = phi8<PHI>(*p);
+          *p = fq[cc];
         }
       }
       fence_proxy_async();
-      mbar_arrive(bar[B_PHI]);
+      mbar_arrive((bar0 + 8u * (B_PHI)));
+      // this half of phi(q) . z_prev, while the tensor cores form P
+      float dpart = 0.f;
+      if (ok) {
+        const float* zp = zbuf + par * D + 64 * hf;
+        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < 8; ++cc) {
+          const float4 z0 = *reinterpret_cast<const float4*>(zp + 8 * cc);
+          const float4 z1 = *reinterpret_cast<const float4*>(zp + 8 * cc + 4);
+          d0 = fmaf(lo_f(fq[cc].x), z0.x, d0); d1 = fmaf(hi_f(fq[cc].x), z0.y, d1);
+          d2 = fmaf(lo_f(fq[cc].y), z0.z, d2); d3 = fmaf(hi_f(fq[cc].y), z0.w, d3);
+          d0 = fmaf(lo_f(fq[cc].z), z1.x, d0); d1 = fmaf(hi_f(fq[cc].z), z1.y, d1);
+          d2 = fmaf(lo_f(fq[cc].w), z1.z, d2); d3 = fmaf(hi_f(fq[cc].w), z1.w, d3);
+        }
+        dpart = (d0 + d1) + (d2 + d3);
+      }
 
       // ---- P: causal mask, packed bf16 -> TMEM ----
-      ok = ok && mbar_wait(bar[B_MMA_P], par, abort);
+      ok = ok && mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
@@ -515,34 +576,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         for (int qq = 0; qq < 2; ++qq) {
           const int col0 = 64 * hf + 32 * qq;
           uint32_t v[32], pk[16];
+          float ps0 = 0.f, ps1 = 0.f;
           if (col0 <= 32 * (wa & 3) + 31) {                     // warp-uniform: some row of this warp reaches col0
             LA_TMEM_LD32(tmem + P_COL + lane_addr + col0, v);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 16; ++e)
-              pk[e] = pack2(col0 + 2 * e <= r ? __uint_as_float(v[2 * e]) : 0.f,
-                            col0 + 2 * e + 1 <= r ? __uint_as_float(v[2 * e + 1]) : 0.f);
+            for (int e = 0; e < 16; ++e) {
+              const float p0 = col0 + 2 * e <= r ? __uint_as_float(v[2 * e]) : 0.f;
+              const float p1 = col0 + 2 * e + 1 <= r ? __uint_as_float(v[2 * e + 1]) : 0.f;
+              pk[e] = pack2(p0, p1);
+              ps0 += p0;
+              ps1 += p1;
+            }
+            dpart += ps0 + ps1;
           } else {
 #pragma unroll
             for (int e = 0; e < 16; ++e) pk[e] = 0u;
           }
-          LA_TMEM_ST16(tmem + P16_COL + lane_addr + (col0 >> 1), pk);
+          LA_TMEM_ST16(tmem + P_COL + lane_addr + 64 * hf + 16 * qq, pk);
         }
+        denbuf[((n & 3) * 2 + hf) * D + r] = dpart;   // half of den: phi(q) . z_prev + row sum of the masked P
         tmem_wait_st();
       }
       tc_fence_before();
-      mbar_arrive(bar[B_PDONE]);
+      mbar_arrive((bar0 + 8u * (B_PDONE)));
 
       // ---- phi on K of the next tile while the tensor cores work on this one ----
       if (!last) {
-        ok = ok && mbar_wait(bar[((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0], ((n + 1) >> 1) & 1, abort);
+        ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
         ok = __all_sync(0xffffffffu, ok);
-        if (ok) phi_k(n + 1);
+        phi_k(n + 1, ok);
       }
 
-      // ---- [S|z]_n: bf16 copy for the next tile, or the final state to global memory ----
-      // S_n is final after MMA_S; the old copy may be overwritten once [O|den] = phi(Q)[S|z]_prev has read it
-      ok = ok && mbar_wait(bar[B_MMA_S], par, abort) && mbar_wait(bar[B_MMA_Q], par, abort);
+      // ---- S_n: bf16 copy for the next tile, or the final state to global memory ----
+      // S_n is final after MMA_S; the old copy may be overwritten once O = phi(Q) S_prev has read it
+      ok = ok && mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort) && mbar_wait((bar0 + 8u * (B_MMA_Q)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
@@ -562,16 +630,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
             for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
           }
         }
-        if (hf == 0) {
-          const float zz = __uint_as_float(tmem_ld1(tmem + lane_addr + Z_COL));
-          tmem_wait_ld();
-          if (last) z[(size_t)u * D + r] = zz;
-          else *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(r, 0)) = __float2bfloat16_rn(zz);
-        }
+        if (last && hf == 0) z[(size_t)u * D + r] = zbuf[(nchunks & 1) * D + r];   // r == ta: this thread wrote it
       }
       fence_proxy_async();
       tc_fence_before();
-      mbar_arrive(bar[B_SB]);
+      mbar_arrive((bar0 + 8u * (B_SB)));
     }
   } else {
     // =============================== group B: epilogue (256 threads) ===============================
@@ -588,74 +651,65 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                                   : n == 0 ? halo0
                                            : vg + ((size_t)bh * Ttot + y0 + (size_t)n * TILE - (W - 1)) * D;
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
-      ok = ok && mbar_wait(bar[B_FULL_V0 + par], (n >> 1) & 1, abort);
+      ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && tid < D && !gh) {
-        // next halo <- last W-1 rows of (halo ++ valid rows of V)
-        const unsigned char* Vc = Vt + (tid >> 6) * BOX_BYTES;
-        const int cw = tid & 63;
+      if (ok && (tid & 127) < 64 && !gh) {
+        // next halo <- last W-1 rows of (halo ++ valid rows of V); each half of the group copies its own channels
+        const unsigned char* Vc = Vt + hf * BOX_BYTES;
+        const int cw = tid & 63, ch = 64 * hf + cw;
         for (int i = 0; i < W - 1; ++i) {
           const int src = valid + i;
           __nv_bfloat16 x;
-          if (src < W - 1) x = halo[src * D + tid];
+          if (src < W - 1) x = halo[src * D + ch];
           else x = *reinterpret_cast<const __nv_bfloat16*>(Vc + swz(src - (W - 1), cw >> 3) + (cw & 7) * 2);
-          halo_next[i * D + tid] = x;
+          halo_next[i * D + ch] = x;
         }
       }
-      ok = ok && mbar_wait(bar[B_MMA_O], par, abort);
+      ok = ok && mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);   // also: every product that reads V is done
       ok = __all_sync(0xffffffffu, ok);
-      uint4 outp[8];                              // this thread's 64 channels of row r, packed
+      // The outputs leave through the V buffer of this tile, 16-byte column by column: a column is overwritten (same
+      // swizzled layout) once every thread of this half has taken its taps from it, so that a thread holds one
+      // column of outputs at a time; the control lane then stores whole rows with one TMA store per box.  The two
+      // halves of the group (64 channels each) share nothing and synchronise separately.
+      sync_half_b(hf);                            // the next halo is complete before any row of V is overwritten
+      float rden = 0.f;
       if (ok) {
         tc_fence_after();
-        const float den = __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
-        tmem_wait_ld();
-        const float rden = 1.f / (den + eps);
+        const float den = denbuf[((n & 3) * 2) * D + r] + denbuf[((n & 3) * 2 + 1) * D + r];
+        rden = 1.f / (den + eps);
+      }
+      unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
 #pragma unroll
-        for (int qq = 0; qq < 2; ++qq) {
-          uint32_t v[32];
-          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32 * qq, v);
+      for (int qq = 0; qq < 2; ++qq) {
+        uint32_t v[32];
+        if (ok) {
+          LA_TMEM_LD32(tmem + lane_addr + O_COL + par * 128u + 64 * hf + 32 * qq, v);
           tmem_wait_ld();
+        }
+        if (qq == 1) {
+          tc_fence_before();
+          mbar_arrive((bar0 + 8u * (B_EPI0 + par)));         // this accumulator has been read
+        }
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const int cc = 4 * qq + c;                          // chunk inside this half's box
-            const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
+        for (int c = 0; c < 4; ++c) {
+          const int cc = 4 * qq + c;                            // chunk inside this half's box
+          const int ch0 = 64 * hf + 8 * cc;                     // first channel of the chunk
+          uint4 outp = make_uint4(0u, 0u, 0u, 0u);
+          if (ok) {
             float acc[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
             conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
-            outp[cc] = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+            outp = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
           }
+          sync_half_b(hf);                        // column cc of this half has been read by all of its rows
+          if (ok) *reinterpret_cast<uint4*>(Ob + swz(r, cc)) = outp;
         }
-      }
-      // the state update, issued after the products of this tile's outputs, reads V too: it must be complete before
-      // the outputs overwrite the buffer (it is, long since; the wait comes before the arrival below so that the
-      // next completion of that barrier cannot overtake it)
-      ok = ok && mbar_wait(bar[B_MMA_S], par, abort);
-      ok = __all_sync(0xffffffffu, ok);
-      tc_fence_before();
-      mbar_arrive(bar[B_EPI]);                    // O has been read
-      // The outputs leave through the V buffer of this tile: once every thread has taken its taps from it, each row
-      // is overwritten with its outputs (same swizzled layout) and one TMA store per box writes whole rows.
-      sync_group_b();                             // V and the old halo have been read; the next halo is complete
-      if (ok) {
-        unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) *reinterpret_cast<uint4*>(Ob + swz(r, cc)) = outp[cc];
       }
       fence_proxy_async();
-      sync_group_b();
-      if (tid == 0) {
-        if (ok) {
-          const uint32_t src = sbase + OFF_V0 + par * TILE_BYTES;
-          tma_store(&mo, 0, y0 + n * TILE, bh, src);            // rows past the end of the sequence are clipped
-          tma_store(&mo, 64, y0 + n * TILE, bh, src + BOX_BYTES);
-          tma_commit();
-          tma_wait_read();                                      // the buffer has been read
-        }
-        mbar_arrive(bar[B_VFREE]);
-      }
+      mbar_arrive((bar0 + 8u * (B_STAGED0 + par)));
     }
-    if (tid == 0) tma_wait_all();                 // the last stores are complete before the CTA exits
+    sync_group_b();                               // both halves of the last halo are complete
     if (ok && tid < D) {
       // the window to carry on: the last W-1 values of (incoming window ++ this unit's v)
       const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
@@ -707,14 +761,12 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
   const int u = blockIdx.x, bh = u / nseg;
   const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
   const int nchunks = (T + TILE - 1) / TILE;
-  uint32_t bar[kStateBars];
-#pragma unroll
-  for (int i = 0; i < kStateBars; ++i) bar[i] = smem_u32(&bars[i]);
+  const uint32_t bar0 = smem_u32(&bars[0]);       // barrier i lives at bar0 + 8 i
 
   if (tid == 0) {
-    for (int i = 0; i < 4; ++i) mbar_init(bar[i], 1);
-    mbar_init(bar[SB_PHI], 256);
-    mbar_init(bar[SB_MMA], 1);
+    for (int i = 0; i < 4; ++i) mbar_init((bar0 + 8u * (i)), 1);
+    mbar_init((bar0 + 8u * (SB_PHI)), 256);
+    mbar_init((bar0 + 8u * (SB_MMA)), 1);
     *abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -738,17 +790,17 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
     if (lane == 0) {
       auto load_tile = [&](int n) {
         const uint32_t b2 = n & 1;
-        mbar_expect_tx(bar[SB_FULL_K0 + b2], TILE_BYTES);
-        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES, &mk, 0, y0 + n * TILE, bh, bar[SB_FULL_K0 + b2]);
-        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES + BOX_BYTES, &mk, 64, y0 + n * TILE, bh, bar[SB_FULL_K0 + b2]);
-        mbar_expect_tx(bar[SB_FULL_V0 + b2], TILE_BYTES);
-        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, bar[SB_FULL_V0 + b2]);
-        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, bar[SB_FULL_V0 + b2]);
+        mbar_expect_tx((bar0 + 8u * (SB_FULL_K0 + b2)), TILE_BYTES);
+        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES, &mk, 0, y0 + n * TILE, bh, (bar0 + 8u * (SB_FULL_K0 + b2)));
+        tma_load(sbase + ST_OFF_K + b2 * TILE_BYTES + BOX_BYTES, &mk, 64, y0 + n * TILE, bh, (bar0 + 8u * (SB_FULL_K0 + b2)));
+        mbar_expect_tx((bar0 + 8u * (SB_FULL_V0 + b2)), TILE_BYTES);
+        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, (bar0 + 8u * (SB_FULL_V0 + b2)));
+        tma_load(sbase + ST_OFF_V + b2 * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, (bar0 + 8u * (SB_FULL_V0 + b2)));
       };
       for (int n = 0; n < 2 && n < nchunks; ++n) load_tile(n);
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t b2 = n & 1;
-        if (!mbar_wait(bar[SB_PHI], n & 1, abort) || !mbar_wait(bar[SB_FULL_V0 + b2], (n >> 1) & 1, abort)) break;
+        if (!mbar_wait((bar0 + 8u * (SB_PHI)), n & 1, abort) || !mbar_wait((bar0 + 8u * (SB_FULL_V0 + b2)), (n >> 1) & 1, abort)) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {     // [dS | dz] += phi(K)^T [V | 1]
@@ -756,8 +808,8 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
           mma_bf16(tmem + SCOL, kd, desc_mnmajor(sbase + ST_OFF_V + b2 * TILE_BYTES, ks), idesc(true, true, 128), n > 0 || ks > 0);
           mma_bf16(tmem + ZCOL, kd, desc_ext(sbase + ST_OFF_ONES, ks), idesc(true, true, 16), n > 0 || ks > 0);
         }
-        mma_commit(bar[SB_MMA]);
-        if (!mbar_wait(bar[SB_MMA], n & 1, abort)) break;       // both buffers of this tile are free
+        mma_commit((bar0 + 8u * (SB_MMA)));
+        if (!mbar_wait((bar0 + 8u * (SB_MMA)), n & 1, abort)) break;       // both buffers of this tile are free
         if (n + 2 < nchunks) load_tile(n + 2);
       }
     }
@@ -765,7 +817,7 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
     bool ok = true;
     for (int n = 0; n < nchunks; ++n) {
       const int valid = min(TILE, T - n * TILE);
-      ok = ok && mbar_wait(bar[SB_FULL_K0 + (n & 1)], (n >> 1) & 1, abort);
+      ok = ok && mbar_wait((bar0 + 8u * (SB_FULL_K0 + (n & 1))), (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         const int ct = tid & 15, rg = tid >> 4;
@@ -778,11 +830,11 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
         }
       }
       fence_proxy_async();
-      mbar_arrive(bar[SB_PHI]);
+      mbar_arrive((bar0 + 8u * (SB_PHI)));
     }
     // Wait for the last two products in turn (tile L was loaded only after product L-2 had completed, so the
     // barrier is at phase L-1 or later here and a parity wait cannot be fooled by an older phase).
-    for (int n = max(0, nchunks - 2); n < nchunks; ++n) ok = ok && mbar_wait(bar[SB_MMA], n & 1, abort);
+    for (int n = max(0, nchunks - 2); n < nchunks; ++n) ok = ok && mbar_wait((bar0 + 8u * (SB_MMA)), n & 1, abort);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
