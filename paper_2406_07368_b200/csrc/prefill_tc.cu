@@ -39,11 +39,12 @@ constexpr int kCtrlWarp = 16;
 constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns (all 512): P, two O accumulators (tiles alternate, so that the epilogue of one tile runs beside the
-// products of the next) and S, 128 fp32 columns each.  The masked P goes back as packed bf16 pairs into the columns
-// its own fp32 values came from: each thread overwrites only columns of its own row that it has already read
-// (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
-constexpr uint32_t P_COL = 0, O_COL = 128 /* and 256 */, S_COL = 384, TMEM_COLS = 512;
+// TMEM columns: P, O and S, 128 fp32 columns each, and phi(Q) as packed bf16 pairs (64 columns): phi(Q) is the A
+// operand of two products and goes from the registers that computed it straight to TMEM, so that the Q buffer in
+// shared memory is free for the next tile as soon as it has been read.  The masked P goes back as packed bf16 pairs
+// into the columns its own fp32 values came from: each thread overwrites only columns of its own row that it has
+// already read (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
+constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, FQ_COL = 384 /* 64 columns */, TMEM_COLS = 512;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0, OFF_K0 = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
@@ -373,40 +374,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         const uint32_t kbuf = sbase + (par ? OFF_K1 : OFF_K0);
         const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
         const bool has_state = init || n > 0;
-        const uint32_t ocol = tmem + O_COL + par * 128u;        // this tile's accumulator
-        // low descriptor words of step 0: Q and K read along their rows (K-major), K, V and the S copy down their rows
-        const uint32_t q_km = desc_lo(sbase + OFF_Q, 16u), k_km = desc_lo(kbuf, 16u);
+        // low descriptor words of step 0: K read along its rows (K-major), K, V and the S copy down their rows
+        const uint32_t k_km = desc_lo(kbuf, 16u);
         const uint32_t k_mn = desc_lo(kbuf, BOX_BYTES), v_mn = desc_lo(vbuf, BOX_BYTES), s_mn = desc_lo(sbase + OFF_S, BOX_BYTES);
-        ok = mbar_wait((bar0 + 8u * (B_PHI)), par, abort);                 // phi(Q), phi(K) of tile n are in place
+        ok = mbar_wait((bar0 + 8u * (B_PHI)), par, abort);   // phi(Q) of tile n is in TMEM, phi(K) in place
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T
-          mma_bf16(tmem + P_COL, desc64(q_km + kstep_kmajor(ks)), desc64(k_km + kstep_kmajor(ks)),
-                   idesc(false, false, 128), ks > 0);
-        mma_commit((bar0 + 8u * (B_MMA_P)));
-        // the bf16 copy of S before tile n is complete (and S itself has been read) after n + 1 arrivals; the
-        // accumulator is free once the epilogue of tile n-2 has read it
-        ok = mbar_wait((bar0 + 8u * (B_SB)), par, abort);
-        if (ok && n >= 2) ok = mbar_wait((bar0 + 8u * (B_EPI0 + par)), ((n >> 1) - 1) & 1, abort);
-        if (!ok) break;
-        tc_fence_after();
-        if (has_state) {
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
-            mma_bf16(ocol, desc64(q_km + kstep_kmajor(ks)), desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128),
-                     ks > 0);
-        }
-        mma_commit((bar0 + 8u * (B_MMA_Q)));
-        // The single Q buffer sets the pace (last read -> reload -> phi -> products of the next tile), so its reload
-        // goes out as soon as the two products that read it are complete, ahead of the state update.
+        // The Q buffer has been read by then (phi(Q) lives in TMEM): its reload, which sets the pace, goes out first.
         if (n + 1 < nchunks) {
-          ok = mbar_wait((bar0 + 8u * (B_MMA_Q)), par, abort);             // the Q buffer is free
-          if (!ok) break;
           mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
           tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
         }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T; 16 channels of every row of phi(Q) = 8 columns
+          mma_bf16_ts(tmem + P_COL, tmem + FQ_COL + 8 * ks, desc64(k_km + kstep_kmajor(ks)), idesc(false, false, 128), ks > 0);
+        mma_commit((bar0 + 8u * (B_MMA_P)));
+        // The state update needs nothing from the previous tile's epilogue: it fills the time until that epilogue
+        // has read the accumulator.
         ok = mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
 #pragma unroll
@@ -414,12 +399,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16(tmem + S_COL, desc64(k_mn + kstep_mnmajor(ks)), desc64(v_mn + kstep_mnmajor(ks)), idesc(true, true, 128),
                    has_state || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_S)));
+        // the bf16 copy of S before tile n is complete after n + 1 arrivals; the accumulator is free once the
+        // epilogue of tile n-1 has read it
+        ok = mbar_wait((bar0 + 8u * (B_SB)), par, abort);
+        if (ok && n >= 1) ok = mbar_wait((bar0 + 8u * (B_EPI0 + (par ^ 1))), ((n - 1) >> 1) & 1, abort);
+        if (!ok) break;
+        tc_fence_after();
+        if (has_state) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
+            mma_bf16_ts(tmem + O_COL, tmem + FQ_COL + 8 * ks, desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128), ks > 0);
+        }
+        mma_commit((bar0 + 8u * (B_MMA_Q)));
         ok = mbar_wait((bar0 + 8u * (B_PDONE)), par, abort);               // masked P of tile n is in TMEM
         if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)       // O += (P o M) V; 16 tokens of every row of P = 8 columns
-          mma_bf16_ts(ocol, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
+          mma_bf16_ts(tmem + O_COL, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
                       idesc(false, true, 128), has_state || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
         if (n + 2 < nchunks) {
@@ -539,16 +536,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       // ---- phi on Q in place (phi on K of this tile was done one iteration earlier) ----
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
-      uint4 fq[8];                                // phi(q) of row r, this thread's 64 channels
+      // phi(q) of row r, this thread's 64 channels: 32 packed pairs = 32 TMEM columns of lane r.  (The products of
+      // tile n-1 that read these columns are complete: the snapshot above waited for them.)
+      uint32_t fq[32];
       if (ok) {
 #pragma unroll
         for (int cc = 0; cc < 8; ++cc) {
-          uint4* p = reinterpret_cast<uint4*>(Qb + swz(r, cc));
-          fq[cc] = phi8<PHI>(*p);
-          *p = fq[cc];
+          const uint4 f = phi8<PHI>(*reinterpret_cast<const uint4*>(Qb + swz(r, cc)));
+          fq[4 * cc] = f.x; fq[4 * cc + 1] = f.y; fq[4 * cc + 2] = f.z; fq[4 * cc + 3] = f.w;
         }
+        LA_TMEM_ST32(tmem + lane_addr + FQ_COL + 32 * hf, fq);
+        tmem_wait_st();
       }
-      fence_proxy_async();
+      fence_proxy_async();                        // (phi(K) of this tile, written one iteration earlier)
+      tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PHI)));
       // this half of phi(q) . z_prev, while the tensor cores form P
       float dpart = 0.f;
@@ -559,10 +560,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         for (int cc = 0; cc < 8; ++cc) {
           const float4 z0 = *reinterpret_cast<const float4*>(zp + 8 * cc);
           const float4 z1 = *reinterpret_cast<const float4*>(zp + 8 * cc + 4);
-          d0 = fmaf(lo_f(fq[cc].x), z0.x, d0); d1 = fmaf(hi_f(fq[cc].x), z0.y, d1);
-          d2 = fmaf(lo_f(fq[cc].y), z0.z, d2); d3 = fmaf(hi_f(fq[cc].y), z0.w, d3);
-          d0 = fmaf(lo_f(fq[cc].z), z1.x, d0); d1 = fmaf(hi_f(fq[cc].z), z1.y, d1);
-          d2 = fmaf(lo_f(fq[cc].w), z1.z, d2); d3 = fmaf(hi_f(fq[cc].w), z1.w, d3);
+          d0 = fmaf(lo_f(fq[4 * cc]), z0.x, d0); d1 = fmaf(hi_f(fq[4 * cc]), z0.y, d1);
+          d2 = fmaf(lo_f(fq[4 * cc + 1]), z0.z, d2); d3 = fmaf(hi_f(fq[4 * cc + 1]), z0.w, d3);
+          d0 = fmaf(lo_f(fq[4 * cc + 2]), z1.x, d0); d1 = fmaf(hi_f(fq[4 * cc + 2]), z1.y, d1);
+          d2 = fmaf(lo_f(fq[4 * cc + 3]), z1.z, d2); d3 = fmaf(hi_f(fq[4 * cc + 3]), z1.w, d3);
         }
         dpart = (d0 + d1) + (d2 + d3);
       }
@@ -683,7 +684,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       for (int qq = 0; qq < 2; ++qq) {
         uint32_t v[32];
         if (ok) {
-          LA_TMEM_LD32(tmem + lane_addr + O_COL + par * 128u + 64 * hf + 32 * qq, v);
+          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32 * qq, v);
           tmem_wait_ld();
         }
         if (qq == 1) {
