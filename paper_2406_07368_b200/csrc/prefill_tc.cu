@@ -5,11 +5,12 @@
 // sums S = sum phi(k) v^T and z = sum phi(k) are carried.  One CTA walks one (batch, head)
 // chain in tiles of 128 tokens:
 //     O = phi(Q) S_prev + (P o M) V,   den = phi(Q) . z_prev + rowsum(P o M),   S += phi(K)^T V,   z += colsum phi(K).
-// The four matrix products run on the tensor cores; the normaliser (two vectors per tile) is formed by the
-// threads that hold phi(Q), phi(K) and P in registers anyway.  Per tile n:
+// The matrix products run on the tensor cores, and z rides along with S: V is extended by a column of ones and the
+// copy of S by the column z ([S | z] += phi(K)^T [V | 1], [O | phi(q) . z] = phi(Q) [S | z]_prev; 16-column,
+// unswizzled operand blocks).  The row sums of the masked P are taken by the threads that mask it.  Per tile n:
 //
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
-//   group A  phi applied in place on Q and K (packed bf16x2 arithmetic); phi(q) . z_prev; z += colsum phi(K)
+//   group A  phi(Q) -> TMEM and phi(K) in place (packed bf16x2 arithmetic)
 //   tcgen05  P = phi(Q) phi(K)^T
 //            S += phi(K)^T V                 (fp32 in TMEM for the whole chain)
 //            O = phi(Q) S_prev               (S_prev is a bf16 copy in shared memory)
@@ -44,15 +45,16 @@ constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
 // shared memory is free for the next tile as soon as it has been read.  The masked P goes back as packed bf16 pairs
 // into the columns its own fp32 values came from: each thread overwrites only columns of its own row that it has
 // already read (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
-constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, FQ_COL = 384 /* 64 columns */, TMEM_COLS = 512;
+constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, FQ_COL = 384 /* 64 columns */, DEN_COL = 448, Z_COL = 464,
+                   TMEM_COLS = 512;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0, OFF_K0 = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
                    OFF_K1 = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
-                   OFF_ZBUF = 6 * TILE_BYTES,      // [2][128] fp32: z before even / odd tiles
-                   OFF_KPART = OFF_ZBUF + 1024,    // [8][128] fp32: column sums of phi(K), one row per warp
-                   OFF_DEN = OFF_KPART + 4096,     // [4][2][128] fp32: halves of the denominators of tile n in slot n & 3
-                   OFF_SMALL = OFF_DEN + 4096;
+                   OFF_ONES = 6 * TILE_BYTES,      // [128 x 16] bf16, column 0 = 1: the extension of V
+                   OFF_SZ = OFF_ONES + 4096,       // [128 x 16] bf16, column 0 = z: the extension of the S copy
+                   OFF_DEN = OFF_SZ + 4096,        // [2][2][128] fp32: halves of the row sums of the masked P of tile n in slot n & 1
+                   OFF_SMALL = OFF_DEN + 2048;
 
 struct Small {
   unsigned long long bars[20];
@@ -97,7 +99,6 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void sync_group_b() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
-__device__ __forceinline__ void sync_group_a() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void sync_half_b(int hf) {
   if (hf) asm volatile("bar.sync 4, 128;" ::: "memory");
   else asm volatile("bar.sync 3, 128;" ::: "memory");
@@ -338,10 +339,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
     halo0[idx] = init ? win[(size_t)u * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
-  float* zbuf = reinterpret_cast<float*>(smem + OFF_ZBUF);      // zbuf[m & 1]: z before tile m
-  float* kpart = reinterpret_cast<float*>(smem + OFF_KPART);
   float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
-  if (tid < D) zbuf[tid] = init ? z[(size_t)u * D + tid] : 0.f;
+  for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
+    reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  __syncthreads();
+  if (tid < TILE) {
+    *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
+    if (init)
+      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)u * D + tid]);
+  }
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -395,9 +401,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         ok = mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)       // S += phi(K)^T V
-          mma_bf16(tmem + S_COL, desc64(k_mn + kstep_mnmajor(ks)), desc64(v_mn + kstep_mnmajor(ks)), idesc(true, true, 128),
-                   has_state || ks > 0);
+        for (int ks = 0; ks < 8; ++ks) {     // [S | z] += phi(K)^T [V | 1]
+          const uint64_t kd = desc64(k_mn + kstep_mnmajor(ks));
+          mma_bf16(tmem + S_COL, kd, desc64(v_mn + kstep_mnmajor(ks)), idesc(true, true, 128), has_state || ks > 0);
+          mma_bf16(tmem + Z_COL, kd, desc_ext(sbase + OFF_ONES, ks), idesc(true, true, 16), has_state || ks > 0);
+        }
         mma_commit((bar0 + 8u * (B_MMA_S)));
         // the bf16 copy of S before tile n is complete after n + 1 arrivals; the accumulator is free once the
         // epilogue of tile n-1 has read it
@@ -407,8 +415,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tc_fence_after();
         if (has_state) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
+          for (int ks = 0; ks < 8; ++ks) {   // [O | phi(q) . z] = phi(Q) [S | z]_prev
             mma_bf16_ts(tmem + O_COL, tmem + FQ_COL + 8 * ks, desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128), ks > 0);
+            mma_bf16_ts(tmem + DEN_COL, tmem + FQ_COL + 8 * ks, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
+          }
         }
         mma_commit((bar0 + 8u * (B_MMA_Q)));
         ok = mbar_wait((bar0 + 8u * (B_PDONE)), par, abort);               // masked P of tile n is in TMEM
@@ -484,45 +494,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
         for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
       }
+      if (hf == 0) {
+        tmem_st1(tmem + lane_addr + Z_COL, __float_as_uint(z[(size_t)u * D + r]));
+#pragma unroll
+        for (int c = 1; c < 16; ++c) tmem_st1(tmem + lane_addr + Z_COL + c, 0u);
+      }
       tmem_wait_st();
     }
     fence_proxy_async();
     tc_fence_before();
     mbar_arrive((bar0 + 8u * (B_SB)));                       // phase 0: the state before tile 0 is in place
 
-    // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero.  The column
-    // sums of the result advance z: zbuf[(m+1) & 1] = zbuf[m & 1] + colsum (eight rows per thread, the two row
-    // groups of a warp by shuffle, the eight warps through shared memory).
-    // Every warp of the group calls it, also after a wait has run out (go = false: no work, same barrier).
+    // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero
     auto phi_k = [&](int m, bool go) {
-      const int valid = go ? min(TILE, T - m * TILE) : 0;
+      if (!go) return;
+      const int valid = min(TILE, T - m * TILE);
       const int ct = ta & 15, rg = ta >> 4;                     // chunk column 0..15, row group 0..15
       unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * BOX_BYTES;
-      float cs[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) cs[e] = 0.f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int j = rg + 16 * i;
         uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-        const uint4 x = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
-        if (go) *p = x;
-        cs[0] += lo_f(x.x); cs[1] += hi_f(x.x); cs[2] += lo_f(x.y); cs[3] += hi_f(x.y);
-        cs[4] += lo_f(x.z); cs[5] += hi_f(x.z); cs[6] += lo_f(x.w); cs[7] += hi_f(x.w);
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], 16);
-      if (lane < 16) {
-        float4* dst = reinterpret_cast<float4*>(kpart + wa * D + 8 * ct);
-        dst[0] = make_float4(cs[0], cs[1], cs[2], cs[3]);
-        dst[1] = make_float4(cs[4], cs[5], cs[6], cs[7]);
-      }
-      sync_group_a();
-      if (ta < D) {
-        float acc = zbuf[(m & 1) * D + ta];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) acc += kpart[i * D + ta];
-        zbuf[((m + 1) & 1) * D + ta] = acc;
+        *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
       }
     };
     ok = mbar_wait((bar0 + 8u * (B_FULL_K0)), 0, abort);
@@ -551,22 +544,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       fence_proxy_async();                        // (phi(K) of this tile, written one iteration earlier)
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PHI)));
-      // this half of phi(q) . z_prev, while the tensor cores form P
-      float dpart = 0.f;
-      if (ok) {
-        const float* zp = zbuf + par * D + 64 * hf;
-        float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-#pragma unroll
-        for (int cc = 0; cc < 8; ++cc) {
-          const float4 z0 = *reinterpret_cast<const float4*>(zp + 8 * cc);
-          const float4 z1 = *reinterpret_cast<const float4*>(zp + 8 * cc + 4);
-          d0 = fmaf(lo_f(fq[4 * cc]), z0.x, d0); d1 = fmaf(hi_f(fq[4 * cc]), z0.y, d1);
-          d2 = fmaf(lo_f(fq[4 * cc + 1]), z0.z, d2); d3 = fmaf(hi_f(fq[4 * cc + 1]), z0.w, d3);
-          d0 = fmaf(lo_f(fq[4 * cc + 2]), z1.x, d0); d1 = fmaf(hi_f(fq[4 * cc + 2]), z1.y, d1);
-          d2 = fmaf(lo_f(fq[4 * cc + 3]), z1.z, d2); d3 = fmaf(hi_f(fq[4 * cc + 3]), z1.w, d3);
-        }
-        dpart = (d0 + d1) + (d2 + d3);
-      }
+      float dpart = 0.f;                          // this half of the row sum of the masked P
 
       // ---- P: causal mask, packed bf16 -> TMEM ----
       ok = ok && mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
@@ -596,7 +574,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
           LA_TMEM_ST16(tmem + P_COL + lane_addr + 64 * hf + 16 * qq, pk);
         }
-        denbuf[((n & 3) * 2 + hf) * D + r] = dpart;   // half of den: phi(q) . z_prev + row sum of the masked P
+        // (slot n & 1 was last read by the epilogue of tile n-2, before the arrival that released the accumulator to
+        // tile n-1, whose products were complete before P of this tile was issued)
+        denbuf[(par * 2 + hf) * D + r] = dpart;
         tmem_wait_st();
       }
       tc_fence_before();
@@ -631,7 +611,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
             for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Sb + swz(r, 4 * qq + c)) = pack8(v + 8 * c);
           }
         }
-        if (last && hf == 0) z[(size_t)u * D + r] = zbuf[(nchunks & 1) * D + r];   // r == ta: this thread wrote it
+        if (hf == 0) {
+          const float zz = __uint_as_float(tmem_ld1(tmem + lane_addr + Z_COL));
+          tmem_wait_ld();
+          if (last) z[(size_t)u * D + r] = zz;
+          else *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(r, 0)) = __float2bfloat16_rn(zz);
+        }
       }
       fence_proxy_async();
       tc_fence_before();
@@ -676,7 +661,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       float rden = 0.f;
       if (ok) {
         tc_fence_after();
-        const float den = denbuf[((n & 3) * 2) * D + r] + denbuf[((n & 3) * 2 + 1) * D + r];
+        float den = denbuf[(par * 2) * D + r] + denbuf[(par * 2 + 1) * D + r];   // row sum of the masked P
+        if (init || n > 0) {                      // + phi(q) . z_prev, formed beside O on the tensor cores
+          den += __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
+          tmem_wait_ld();
+        }
         rden = 1.f / (den + eps);
       }
       unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
