@@ -681,19 +681,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mbar_arrive((bar0 + 8u * (B_EPI0 + par)));         // this accumulator has been read
         }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int cc = 4 * qq + c;                            // chunk inside this half's box
-          const int ch0 = 64 * hf + 8 * cc;                     // first channel of the chunk
-          uint4 outp = make_uint4(0u, 0u, 0u, 0u);
-          if (ok) {
-            float acc[8];
+        for (int c2 = 0; c2 < 2; ++c2) {          // two columns per barrier
+          uint4 outp[2];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
-            conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
-            outp = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+          for (int j = 0; j < 2; ++j) {
+            const int c = 2 * c2 + j;
+            const int cc = 4 * qq + c;                          // chunk inside this half's box
+            const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
+            outp[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (ok) {
+              float acc[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
+              conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
+              outp[j] = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+            }
           }
-          sync_half_b(hf);                        // column cc of this half has been read by all of its rows
-          if (ok) *reinterpret_cast<uint4*>(Ob + swz(r, cc)) = outp;
+          sync_half_b(hf);                        // these two columns of this half have been read by all of its rows
+          if (ok) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) *reinterpret_cast<uint4*>(Ob + swz(r, 4 * qq + 2 * c2 + j)) = outp[j];
+          }
         }
       }
       fence_proxy_async();
