@@ -256,9 +256,11 @@ template <int PHI> __device__ __forceinline__ uint4 phi8(uint4 u) {
 __device__ __forceinline__ uint32_t swz(int row, int cc) { return (uint32_t)row * 128u + (uint32_t)((cc ^ (row & 7)) << 4); }
 
 // ---- the kernel ------------------------------------------------------------------------------------
-// Convolution part of the epilogue for one 8-channel chunk: acc[e] += sum_t w[t][ch] v_{row-t}[ch].
+// Convolution part of the epilogue for one 8-channel chunk: acc[e] += sum_t w[t][ch] v_{row-t}[ch], two channels per
+// packed fp32 multiply-add (each half is the IEEE fused multiply-add of the scalar instruction).
+__device__ __forceinline__ float2 bf2(uint32_t u) { return make_float2(lo_f(u), hi_f(u)); }
 template <int WT>
-__device__ __forceinline__ void conv8(float* acc, int W, int r, int cc, int ch0, const unsigned char* Vbox,
+__device__ __forceinline__ void conv8(float2* acc, int W, int r, int cc, int ch0, const unsigned char* Vbox,
                                       const __nv_bfloat16* halo, const float* wsm) {
   const int taps = WT > 0 ? WT : W;
 #pragma unroll
@@ -269,10 +271,10 @@ __device__ __forceinline__ void conv8(float* acc, int W, int r, int cc, int ch0,
     else u = *reinterpret_cast<const uint4*>(halo + (W - 1 + row) * D + ch0);
     const float4 w0 = *reinterpret_cast<const float4*>(wsm + t * D + ch0);
     const float4 w1 = *reinterpret_cast<const float4*>(wsm + t * D + ch0 + 4);
-    acc[0] = fmaf(w0.x, lo_f(u.x), acc[0]); acc[1] = fmaf(w0.y, hi_f(u.x), acc[1]);
-    acc[2] = fmaf(w0.z, lo_f(u.y), acc[2]); acc[3] = fmaf(w0.w, hi_f(u.y), acc[3]);
-    acc[4] = fmaf(w1.x, lo_f(u.z), acc[4]); acc[5] = fmaf(w1.y, hi_f(u.z), acc[5]);
-    acc[6] = fmaf(w1.z, lo_f(u.w), acc[6]); acc[7] = fmaf(w1.w, hi_f(u.w), acc[7]);
+    acc[0] = __ffma2_rn(make_float2(w0.x, w0.y), bf2(u.x), acc[0]);
+    acc[1] = __ffma2_rn(make_float2(w0.z, w0.w), bf2(u.y), acc[1]);
+    acc[2] = __ffma2_rn(make_float2(w1.x, w1.y), bf2(u.z), acc[2]);
+    acc[3] = __ffma2_rn(make_float2(w1.z, w1.w), bf2(u.w), acc[3]);
   }
 }
 
@@ -690,11 +692,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
             const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
             outp[j] = make_uint4(0u, 0u, 0u, 0u);
             if (ok) {
-              float acc[8];
+              float2 acc[4];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) acc[e] = __uint_as_float(v[8 * c + e]) * rden;
+              for (int e = 0; e < 4; ++e)
+                acc[e] = __fmul2_rn(make_float2(__uint_as_float(v[8 * c + 2 * e]), __uint_as_float(v[8 * c + 2 * e + 1])),
+                                    make_float2(rden, rden));
               conv8<WT>(acc, W, r, cc, ch0, Vt + hf * BOX_BYTES, halo, wsm);
-              outp[j] = make_uint4(pack2(acc[0], acc[1]), pack2(acc[2], acc[3]), pack2(acc[4], acc[5]), pack2(acc[6], acc[7]));
+              outp[j] = make_uint4(pack2(acc[0].x, acc[0].y), pack2(acc[1].x, acc[1].y), pack2(acc[2].x, acc[2].y),
+                                   pack2(acc[3].x, acc[3].y));
             }
           }
           sync_half_b(hf);                        // these two columns of this half have been read by all of its rows
