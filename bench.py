@@ -35,7 +35,7 @@ L2_BYTES = 126 * 2 ** 20
 NOMINAL_HBM_GBS = 7700.0        # HGX B200 data-sheet figure, printed beside the measured copy bandwidth
 # DRAM bytes (read + written) per launch of the dominant kernel, from the ncu captures summarised under
 # profiles/; None where no capture of the current kernel exists.
-NCU_TRAFFIC = {"llama7b_prefill": 245.9e6, "batched_decode": 218.6e6, "tree_verify": 61.5e6, "long_prefill": 1643.5e6}
+NCU_TRAFFIC = {"llama7b_prefill": 245.9e6, "batched_decode": 218.6e6, "tree_verify": 61.5e6, "long_prefill": 1648.9e6}
 
 
 # ----------------------------------------------------------------------------------------
