@@ -12,16 +12,16 @@
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
 //   group A  phi(Q) -> TMEM and phi(K) in place (packed bf16x2 arithmetic)
 //   tcgen05  P = phi(Q) phi(K)^T
-//            S += phi(K)^T V                 (fp32 in TMEM for the whole chain)
-//            O = phi(Q) S_prev               (S_prev is a bf16 copy in shared memory)
+//            [S | z] += phi(K)^T [V | 1]               (fp32 in TMEM for the whole chain)
+//            [O | phi(q) . z] = phi(Q) [S | z]_prev    ([S | z]_prev is a bf16 copy in shared memory)
 //   group A  P -> causal mask, row sums, bf16 -> TMEM (the A operand of the next product);
-//            phi on K of tile n+1 (K is double-buffered);  S -> bf16 copy for tile n+1
+//            phi on K of tile n+1 (K is double-buffered);  [S | z] -> bf16 copy for tile n+1
 //   tcgen05  O += (P o M) V
-//   group B  o = O / (den + eps) + conv(V) -> global memory
+//   group B  o = O / (den + eps) + conv(V) -> the tile's V buffer;  TMA stores it to global memory
 //
 // Three roles run concurrently: group A (warps 8-15), group B (warps 0-7) and warp 16, whose
-// elected lane issues every TMA load and every MMA.  While group B finishes tile n, group A
-// already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
+// elected lane issues every TMA load, every TMA store and every MMA.  While group B finishes tile n,
+// group A already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
 // records LA_ERR_TIMEOUT, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
@@ -40,9 +40,10 @@ constexpr int kCtrlWarp = 16;
 constexpr int kThreads = 544;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns: P, O and S, 128 fp32 columns each, and phi(Q) as packed bf16 pairs (64 columns): phi(Q) is the A
-// operand of two products and goes from the registers that computed it straight to TMEM, so that the Q buffer in
-// shared memory is free for the next tile as soon as it has been read.  The masked P goes back as packed bf16 pairs
+// TMEM columns: P, O and S, 128 fp32 columns each; phi(Q) as packed bf16 pairs (64 columns); two 16-column blocks
+// whose first column is phi(q) . z and z.  phi(Q) is the A operand of two products and goes from the registers
+// that computed it straight to TMEM, so that the Q buffer in shared memory is free for the next tile as soon as it
+// has been read.  The masked P goes back as packed bf16 pairs
 // into the columns its own fp32 values came from: each thread overwrites only columns of its own row that it has
 // already read (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
 constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, FQ_COL = 384 /* 64 columns */, DEN_COL = 448, Z_COL = 464,
@@ -62,12 +63,12 @@ struct Small {
   int abort;
   int pad[2];
 };
-// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI0 / EPI1: arrivals of group B (that O
-// accumulator has been read).
+// full_*: TMA landed.  PHI / PDONE / SB: arrivals of group A.  EPI0 / EPI1: arrivals of group B (the accumulator
+// has been read; tiles alternate between the two).
 // STAGED0 / STAGED1: group B has written a tile's outputs into that V buffer (the control lane stores them).
-// MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after S += phi(K)^T V (K buffer free);
-// after O = phi(Q) S (Q buffer free); after O += P V (MMA_O0 / MMA_O1, one per accumulator).
-// A barrier that one role waits on while another role can run a tile ahead exists once per accumulator, so that a
+// MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T [V|1] (K buffer free);
+// after [O | phi(q).z] = phi(Q) [S|z]; after O += P V (MMA_O0 / MMA_O1, tiles alternate).
+// A barrier that one role waits on while another role can run a tile ahead exists once per tile parity, so that a
 // waiter is never more than one phase behind.
 enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O0 = 5, B_MMA_O1 = 6, B_PHI = 7,
        B_PDONE = 8, B_SB = 9, B_EPI0 = 10, B_EPI1 = 11, B_MMA_Q = 12, B_FULL_Q = 13, B_FULL_K1 = 14, B_STAGED0 = 15,
@@ -532,7 +533,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
       // phi(q) of row r, this thread's 64 channels: 32 packed pairs = 32 TMEM columns of lane r.  (The products of
-      // tile n-1 that read these columns are complete: the snapshot above waited for them.)
+      // tile n-1 that read these columns are complete: the snapshot at the end of the previous iteration waited for them.)
       uint32_t fq[32];
       if (ok) {
 #pragma unroll
