@@ -29,10 +29,16 @@
  *     status word.
  *   - Every entry point returns an la_status.  Problems the host can see (null or
  *     misaligned pointers, sizes out of range, unsupported head dimension) are rejected
- *     before anything is launched.  Problems only the device can see (a malformed tree, an
- *     accepted node outside the tree, a bounded wait that ran out) make the kernel skip the
- *     affected sequence, leave its outputs and state unwritten, and record a sticky code in
- *     the status word, which la_last_device_status returns.  Nothing ever traps.
+ *     before anything is launched.  Problems only the device can see record a sticky code in
+ *     the status word, which la_last_device_status returns; nothing ever traps.  A malformed
+ *     tree or an accepted node outside the tree (LA_ERR_BAD_TREE) makes the kernel skip the
+ *     affected sequence and leave its outputs and state unwritten.  A bounded wait that ran out
+ *     (LA_ERR_TIMEOUT) ends the thread block where it stands: outputs of that call may be
+ *     partly written and the state buffers it was updating are undefined afterwards -- restore
+ *     them from a copy or restart the sequence.
+ *   - LA_ERR_UNSUPPORTED from la_prefill / la_verify_tree means that the shape belongs to the
+ *     tensor-core kernels but the driver cannot encode TMA tensor maps; the library does not
+ *     fall back to a slower kernel behind the caller's back.
  */
 #ifndef LA_B200_LA_H_
 #define LA_B200_LA_H_
@@ -110,6 +116,11 @@ const char* la_status_str(la_status s);
  *   init_state  0: start from an empty state (st is output only); 1: continue from st
  *   st          in-out; on return holds S, z, the window and pos after the T tokens
  *   o           [B, H, T, d] io type
+ *
+ * Kernels: bf16 io with d = 128 runs grouped on the tensor cores (128-token tiles).  fp32 io, and
+ * d = 64 in either type, take a CUDA-core kernel that walks the tokens in order -- the cumulative
+ * sum taken literally, every product an fp32 multiply-add, which is what the fp32 tolerance
+ * needs; it is correct for any T but far slower per token.
  */
 la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
                      const float* conv_w, int32_t init_state, la_state* st /*host struct*/, void* o,
@@ -193,9 +204,12 @@ la_status la_selftest_wait_timeout(la_ctx* ctx, uint32_t limit_us, int64_t* wait
  * allocation's implicit synchronisation would stall other streams.  Such a caller cannot
  * use la_create, because the context allocates its status word.
  *
- * It computes exactly what la_verify_tree computes, from the same arguments, with the
- * configuration passed directly instead of a context, on the device that is current at the
- * call.  It calls no allocating routine.  Its only scratch memory, one status word per
+ * It computes what la_verify_tree computes, from the same arguments, with the configuration
+ * passed directly instead of a context, on the device that is current at the call.  It always
+ * runs the fp32 CUDA-core kernel, so for bf16 io with d = 128 its results agree with
+ * la_verify_tree (which rounds S and the scores to bf16 for the tensor cores) within the io
+ * tolerance rather than bit for bit, and it is several times slower for that shape.  It calls
+ * no allocating routine.  Its only scratch memory, one status word per
  * sequence, is a fixed array inside the library image; each GPU that loads the library
  * carries those LA_NOALLOC_MAX_SEQ * 4 bytes until the process ends.
  *
@@ -207,8 +221,9 @@ la_status la_selftest_wait_timeout(la_ctx* ctx, uint32_t limit_us, int64_t* wait
  *   other arguments as for la_verify_tree; cfg->max_nodes, max_depth and chunk are ignored
  *   (N is limited by LA_MAX_NODES).
  *
- * The first call on each device looks up the device address of the fixed array; make that
- * first call outside any stream capture.  All calls share the array, which still holds the
+ * The first call on each device looks up the device address of the fixed array (and, as the
+ * first use of the library on that device, makes the CUDA runtime load the kernel image); make
+ * that first call outside any stream capture.  All calls share the array, which still holds the
  * previous call's codes on entry, so every call first clears the B words it uses, on
  * `stream`.  Two calls that overlap on the GPU (different streams, no ordering between
  * them) race on those words: keep calls to this entry point ordered on one device. */

@@ -7,6 +7,11 @@
 
 namespace {
 
+// A launcher's error as a status: a shape the tensor-core path covers on a driver that cannot encode tensor maps is
+// LA_ERR_UNSUPPORTED (there is no silent detour over the CUDA-core kernels), everything else LA_ERR_CUDA.
+inline la_status cuda_status(cudaError_t e) {
+  return e == cudaSuccess ? LA_OK : e == cudaErrorNotSupported ? LA_ERR_UNSUPPORTED : LA_ERR_CUDA;
+}
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool good(const void* p) { return p != nullptr && aligned16(p); }
 
@@ -114,7 +119,7 @@ la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const voi
   if (ctx->prefill_kernel == 0) {
     bool handled = false;
     cudaError_t e = la::launch_prefill_tc(ctx, B, T, q, k, v, conv_w, init_state, *st, o, s, &handled);
-    if (e != cudaSuccess) return LA_ERR_CUDA;
+    if (e != cudaSuccess) return cuda_status(e);
     if (handled) return LA_OK;
   }
   return la::launch_prefill_simt(ctx, B, T, q, k, v, conv_w, init_state, *st, o, s) == cudaSuccess ? LA_OK
@@ -143,7 +148,8 @@ la_status la_verify_tree(la_ctx* ctx, int32_t B, int32_t N, const void* q, const
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (ctx->prefill_kernel == 0) {
     bool handled = false;
-    if (la::launch_verify_tc(ctx, B, N, q, k, v, parent, conv_w, *st, o, s, &handled) != cudaSuccess) return LA_ERR_CUDA;
+    const cudaError_t e = la::launch_verify_tc(ctx, B, N, q, k, v, parent, conv_w, *st, o, s, &handled);
+    if (e != cudaSuccess) return cuda_status(e);
     if (handled) return LA_OK;
   }
   return la::launch_verify(ctx, B, N, q, k, v, parent, conv_w, *st, o, s) == cudaSuccess ? LA_OK : LA_ERR_CUDA;

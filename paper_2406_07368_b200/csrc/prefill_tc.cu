@@ -1025,7 +1025,7 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   CUtensorMap mq, mk, mv, mo;
   if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
       !tc::make_map(&mo, o, BH, T))
-    return cudaSuccess;   // no tensor-map support: the CUDA-core kernel takes over
+    return cudaErrorNotSupported;   // the driver cannot encode tensor maps: reported, never a silent slow path
   int nseg, seg_len;
   plan_split(ctx, BH, T, &nseg, &seg_len);
   if (nseg > 1 && (ctx->ws == nullptr || ctx->ws_bytes < split_bytes(c, BH, nseg) || T < c.conv_taps)) nseg = 1, seg_len = T;

@@ -638,7 +638,7 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
   *handled = false;
   if (c.io_dtype != LA_BF16 || c.d != vtc::D) return cudaSuccess;
   vtc::EncodeTiledFn fn = vtc::encode_fn();
-  if (!fn) return cudaSuccess;
+  if (!fn) return cudaErrorNotSupported;   // the driver cannot encode tensor maps: reported, never a silent slow path
   const int BH = B * c.H;
   const cuuint32_t es[3] = {1, 1, 1};
   CUtensorMap ms;   // S viewed as [BH * 128 rows, 128 columns] fp32; one unit per box, no swizzle
@@ -649,7 +649,7 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
     if (fn(&ms, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, st.S, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaSuccess;
+      return cudaErrorNotSupported;
   }
   CUtensorMap mv;   // V viewed as [BH][N][128] bf16; boxes of 64 channels x 64 nodes (nodes past N read as zeros)
   {
@@ -659,7 +659,7 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
     if (fn(&mv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(v), dims, strides, box, es,
            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaSuccess;
+      return cudaErrorNotSupported;
   }
   const bool elu = c.phi == LA_PHI_ELU1;
   auto kern = c.conv_taps <= vtc::kMaxTaps

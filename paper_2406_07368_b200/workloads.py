@@ -31,6 +31,7 @@ _STREAM_DRAFT = 5
 _STREAM_ACCEPT = 6
 _STREAM_STATE = 7
 _STREAM_TOKENS = 8
+_STREAM_PROMPT = 9
 
 
 def rng(seed: int, stream: int, a: int = 0, b: int = 0) -> np.random.Generator:
@@ -63,9 +64,13 @@ def gaussian(gen: np.random.Generator, shape, scale: float, io: str) -> np.ndarr
     return store(x, io)
 
 
-def qkv(seed: int, shape, scale: float, io: str, stream: int = _STREAM_QKV, a: int = 0):
-    """Three independent Gaussian tensors of the same shape."""
-    return tuple(gaussian(rng(seed, stream, a, i), shape, scale, io) for i in range(3))
+def qkv(seed: int, shape, scale: float, io: str, stream: int = _STREAM_QKV, a: int = 0, v_mean: float = 0.0):
+    """Three independent Gaussian tensors of the same shape.  `v_mean` shifts the values v: with a non-zero mean the
+    attention term (a weighted mean of values) keeps its size at late positions instead of averaging out."""
+    q, k, v = (gaussian(rng(seed, stream, a, i), shape, scale, io) for i in range(3))
+    if v_mean != 0.0:
+        v = store(v + np.float32(v_mean), io)
+    return q, k, v
 
 
 def conv_weights(seed: int, H: int, d: int, W: int) -> np.ndarray:
@@ -191,6 +196,11 @@ class Workload:
         """q, k, v [B, H, T, d]; sub-sampling B/H/T draws a smaller tensor of the same law."""
         shape = (B or self.B, H or self.H, T or self.T, self.d)
         return qkv(self.seed, shape, self.scale, self.io)
+
+    def prompt_of_sequence(self, b: int, T: int | None = None):
+        """q, k, v [1, H, T, d] of sequence b alone, keyed by b: for batches whose prompts are too large to draw as
+        one array, the prompt is built sequence by sequence."""
+        return qkv(self.seed, (1, self.H, T or self.T, self.d), self.scale, self.io, stream=_STREAM_PROMPT, a=b)
 
     def decode_inputs(self, step: int, B: int | None = None, H: int | None = None):
         shape = (B or self.B, H or self.H, self.d)

@@ -1,0 +1,159 @@
+"""Parity cases in which the attention term is the whole output, or a large part of it.
+
+With zero-mean values and convolution taps of unit scale the convolution branch carries almost all of the output's
+energy, and an error metric floored at the tensor's RMS then says little about the attention term.  Two variants of
+every mode remove that cover: `w0` sets the taps to zero, so that o = la exactly, and `vmean` draws the values around
+1 instead of 0, so that la (a weighted mean of values) stays of order one at late positions.  Same oracle, same
+metric, same tolerances as the other parity tests; the last 128 positions of a prefill are also checked on their own.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import la_oracle as orc
+from paper_2406_07368_b200 import binding, workloads as wl
+from tests._util import TOL, rel_err
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = {"w0": (True, 0.0), "vmean": (False, 1.0), "w0_vmean": (True, 1.0)}
+
+
+def dev(x, io):
+    return torch.from_numpy(np.ascontiguousarray(x)).to(binding.TORCH_DTYPE[io]).cuda()
+
+
+def host(t):
+    return t.detach().float().cpu().numpy().astype(np.float64) if t.is_floating_point() else t.cpu().numpy()
+
+
+def oracle_state_to_dev(st, io):
+    return binding.State(torch.from_numpy(st.S).float().cuda(), torch.from_numpy(st.z).float().cuda(),
+                         dev(st.win.astype(np.float32), io), torch.from_numpy(st.pos).cuda())
+
+
+def make(io, shape, W, seed, scale, variant):
+    zero_w, v_mean = VARIANTS[variant]
+    q, k, v = wl.qkv(seed, shape, scale, io, v_mean=v_mean)
+    w = wl.conv_weights(seed, shape[1], shape[-1], W)
+    if zero_w:
+        w = np.zeros_like(w)
+    return q, k, v, w
+
+
+def check_prefill(o, want, st, wst, io):
+    assert rel_err(host(o), want) < TOL[io]
+    assert rel_err(host(o)[:, :, -128:], want[:, :, -128:]) < TOL[io]      # the late positions on their own
+    assert rel_err(host(st.S), wst.S) < TOL[io] and rel_err(host(st.z), wst.z) < TOL[io]
+    np.testing.assert_array_equal(host(st.win), wst.win)
+    np.testing.assert_array_equal(host(st.pos), wst.pos)
+
+
+@pytest.mark.parametrize("variant", ["w0", "vmean"])
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("io,d,phi,eps,W,T", [
+    ("bf16", 128, "elu1", 0.0, 3, 700), ("bf16", 128, "relu", 1e-6, 5, 333), ("f32", 64, "elu1", 0.0, 3, 256),
+    ("bf16", 64, "elu1", 0.0, 3, 200), ("bf16", 128, "elu1", 0.0, 32, 300), ("bf16", 128, "elu1", 0.0, 3, 2048)])
+def test_prefill_attention_term(variant, kernel, io, d, phi, eps, W, T):
+    B, H = 2, 3
+    scale = 1.0 if io == "f32" else d ** -0.5
+    q, k, v, w = make(io, (B, H, T, d), W, 1000 + T + W, scale, variant)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want, wst = orc.prefill_quadratic(q, k, v, w, phi, eps)
+    check_prefill(o, want, st, wst, io)
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("io,T1,T2,variant", [("bf16", 130, 129, "w0"), ("f32", 50, 77, "vmean"),
+                                              ("bf16", 300, 500, "w0_vmean")])
+def test_prefill_continuation_attention_term(kernel, io, T1, T2, variant):
+    B, H, d, W = 1, 2, 128, 4
+    q, k, v, w = make(io, (B, H, T1 + T2, d), W, 1005, 0.5, variant)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    cut = lambda x, a, b: dev(x[:, :, a:b], io)
+    o1 = ctx.la_prefill(cut(q, 0, T1), cut(k, 0, T1), cut(v, 0, T1), dev(w, "f32"), st, init_state=False)
+    o2 = ctx.la_prefill(cut(q, T1, T1 + T2), cut(k, T1, T1 + T2), cut(v, T1, T1 + T2), dev(w, "f32"), st,
+                        init_state=True)
+    want, wst = orc.prefill_quadratic(q, k, v, w, "elu1", 0.0)
+    assert rel_err(host(o2), want[:, :, T1:]) < TOL[io]                    # the continued part on its own
+    check_prefill(torch.cat([o1, o2], dim=2), want, st, wst, io)
+
+
+@pytest.mark.parametrize("T,W,phi,eps,init,variant", [(2500, 3, "elu1", 0.0, False, "w0"),
+                                                      (4099, 5, "relu", 1e-6, False, "vmean"),
+                                                      (3000, 4, "elu1", 0.0, True, "w0_vmean"),
+                                                      (8192, 5, "relu", 1e-6, False, "w0")])
+def test_prefill_sequence_split_attention_term(T, W, phi, eps, init, variant):
+    io, B, H, d = "bf16", 1, 2, 128
+    q, k, v, w = make(io, (B, H, T, d), W, 2000 + T, d ** -0.5, variant)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    need = ctx.la_prefill_workspace_bytes(B, T)
+    assert need > 0
+    ctx.la_set_workspace(torch.empty(need, dtype=torch.uint8, device="cuda"))
+    st, ost = ctx.new_state(B), None
+    if init:
+        q0, k0, v0, _ = make(io, (B, H, 70, d), W, 2001, d ** -0.5, variant)
+        _, ost = orc.prefill_quadratic(q0, k0, v0, w, phi, eps)
+        st = oracle_state_to_dev(ost, io)
+    n0 = ctx.la_launch_count()
+    o = ctx.la_prefill(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st, init_state=init)
+    assert ctx.la_launch_count() - n0 >= 1
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want, wst = orc.prefill_chunked(q, k, v, w, phi, eps, 256, ost)
+    check_prefill(o, want, st, wst, io)
+    for lo in range(0, T - 127, 1024):                                     # segment by segment
+        assert rel_err(host(o)[:, :, lo:lo + 1024], want[:, :, lo:lo + 1024]) < TOL[io], lo
+
+
+@pytest.mark.parametrize("variant", ["w0", "vmean"])
+@pytest.mark.parametrize("io,d,phi,eps,W", [("f32", 64, "elu1", 0.0, 3), ("bf16", 128, "elu1", 0.0, 3),
+                                            ("bf16", 128, "relu", 1e-6, 5), ("bf16", 128, "elu1", 0.0, 17)])
+def test_decode_attention_term(variant, io, d, phi, eps, W):
+    B, H, T0, steps = 3, 2, 200, 12
+    q, k, v, w = make(io, (B, H, T0, d), W, 1021 + W, 0.7, variant)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    _, ost = orc.prefill_quadratic(q, k, v, w, phi, eps)
+    st = oracle_state_to_dev(ost, io)
+    for s in range(steps):
+        qs, ks, vs = wl.qkv(1100 + s, (B, H, d), 0.7, io, v_mean=VARIANTS[variant][1])
+        o = ctx.la_decode_step(dev(qs, io), dev(ks, io), dev(vs, io), dev(w, "f32"), st)
+        want, ost = orc.decode_step(qs, ks, vs, w, phi, eps, ost)
+        assert rel_err(host(o), want) < TOL[io], s
+    assert rel_err(host(st.S), ost.S) < TOL[io] and rel_err(host(st.z), ost.z) < TOL[io]
+
+
+def tree_case(io, B, H, d, N, W, seed, phi, eps, variant, chain=False, T0=200):
+    q0, k0, v0, w = make(io, (B, H, T0, d), W, seed, 0.7, variant)
+    _, ost = orc.prefill_quadratic(q0, k0, v0, w, phi, eps)
+    q, k, v = wl.qkv(seed + 1, (B, H, N, d), 0.7, io, v_mean=VARIANTS[variant][1])
+    if chain:
+        parent = np.stack([wl.chain_tree(N)] * B)
+    else:
+        parent = np.stack([wl.random_tree(wl.rng(seed, 4, 0, b), N, 5, 4) for b in range(B)]).astype(np.int32)
+    return ost, q, k, v, parent, w
+
+
+@pytest.mark.parametrize("variant", ["w0", "vmean"])
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("io,d,N,W,phi,eps,chain", [
+    ("bf16", 128, 64, 3, "elu1", 0.0, False), ("bf16", 128, 37, 5, "relu", 1e-6, False),
+    ("f32", 64, 10, 3, "elu1", 0.0, False), ("bf16", 128, 64, 8, "elu1", 0.0, True),
+    ("bf16", 128, 64, 4, "relu", 1e-6, True)])
+def test_verify_attention_term(variant, kernel, io, d, N, W, phi, eps, chain):
+    B, H = 3, 2
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, 1041 + N, phi, eps, variant, chain)
+    ctx = binding.Context(H, d, W, phi, eps, io, max_nodes=64, max_depth=64)
+    ctx.la_set_prefill_kernel(kernel)
+    st = oracle_state_to_dev(ost, io)
+    o = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want = orc.verify_tree(q, k, v, parent, w, phi, eps, ost)
+    assert rel_err(host(o), want) < TOL[io]
+    for b in range(B):                                                     # per sequence, so that one unit cannot hide
+        assert rel_err(host(o[b]), want[b]) < TOL[io], b

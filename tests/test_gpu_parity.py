@@ -335,8 +335,6 @@ def test_commit_matches_oracle_and_paths_are_exact(io, d, N, W):
     check_state(st, wst, TOL[io])
     # and it equals decoding the path token by token on the GPU
     st2 = oracle_state_to_dev(ost, io)
-    for b in range(B):
-        pass
     ctx1 = binding.Context(H, d, W, "elu1", 0.0, io)
     for b in range(B):
         sb = binding.State(st2.S[b:b + 1].clone(), st2.z[b:b + 1].clone(), st2.win[b:b + 1].clone(),
