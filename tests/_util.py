@@ -19,4 +19,31 @@ def rel_err(x, y) -> float:
     return float(np.max(np.abs(x - y) / np.maximum(np.abs(y), tau)))
 
 
+def position_octaves(T: int):
+    """[0, 1), [1, 2), [2, 4), [4, 8), ... up to T: ranges of positions within which the attention term of a fresh
+    sequence keeps its scale to within a factor of about sqrt(2)."""
+    out, lo = [(0, 1)], 1
+    while lo < T:
+        out.append((lo, min(2 * lo, T)))
+        lo *= 2
+    return out
+
+
+def rel_err_octaves(x, y, axis: int = 2) -> float:
+    """rel_err taken octave by octave along the position axis, each octave against its own RMS; the largest.
+
+    With zero taps and zero-mean values the output is a running weighted mean of the values: of the values' own
+    size in the first rows and about 1/sqrt(i) of it at row i.  One RMS over the whole tensor is then several
+    times smaller than the early rows and several times larger than the late ones, so it is neither a fair floor
+    for the former nor a strict one for the latter; an octave of positions shares one scale.
+    """
+    x, y = np.asarray(x), np.asarray(y)
+    worst = 0.0
+    for lo, hi in position_octaves(y.shape[axis]):
+        sl = [slice(None)] * y.ndim
+        sl[axis] = slice(lo, hi)
+        worst = max(worst, rel_err(x[tuple(sl)], y[tuple(sl)]))
+    return worst
+
+
 TOL = {"f32": 1e-4, "bf16": 2e-2}

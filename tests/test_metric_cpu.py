@@ -37,3 +37,17 @@ def test_v_mean_shifts_only_the_values():
     np.testing.assert_array_equal(q0, q1)
     np.testing.assert_array_equal(k0, k1)
     np.testing.assert_array_equal(v1, wl.round_to_bf16(v0 + np.float32(1.0)))
+
+
+def test_octaves_tile_the_positions_and_see_the_fault_at_late_rows():
+    from tests._util import position_octaves, rel_err_octaves
+    for T in (1, 2, 3, 128, 700):
+        cuts = position_octaves(T)
+        assert cuts[0] == (0, 1) and cuts[-1][1] == T or T == 1
+        assert all(a[1] == b[0] for a, b in zip(cuts, cuts[1:]))
+    # a fault confined to the last rows of a decaying signal is invisible to one RMS over the tensor, not to octaves
+    T = 4096
+    y = np.random.default_rng(0).standard_normal((1, 1, T, 8)) / np.sqrt(np.arange(1, T + 1))[None, None, :, None]
+    x = y.copy()
+    x[:, :, -256:] *= 0.9
+    assert rel_err(x, y) < 0.03 and rel_err_octaves(x, y) > 0.09
