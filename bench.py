@@ -2,13 +2,20 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
-One step is one pass of the hot path over one batch of synthetic input.  The default
+One step is one pass of the hot path over one batch of synthetic input.  The headline
 workload is the LLaMA-2-7B-shaped prefill (B=4, H=32, d=128, T=2048, bf16, elu+1, 3 taps);
---workload batched_decode / tree_verify / long_prefill time the other shapes with the same
-machinery.  Rank 0 prints one JSON line.  With N > 1 (launched by torch.distributed.run) every
-rank processes its own batch -- (sequence, head) units are independent, so there is no
-collective on the data path -- and the value is the total over ranks divided by the slowest
-rank's time.
+on one GPU the same run also times the other shapes (batched decode, tree verification with its
+commit, long-context prefill) and reports them under "others".  --workload NAME makes another
+shape the headline.  Rank 0 prints one JSON line.
+
+With N > 1 every rank processes its own batch -- (sequence, head) units are independent, so
+there is no collective on the data path -- and the value is the total over ranks divided by the
+slowest rank's time.  The ranks come from torch.distributed.run (RANK / WORLD_SIZE in the
+environment); started plainly with --gpus N > 1, this program starts the N ranks itself.
+
+Timing: W warm-up steps, then R regions of exactly K steps each, every region bracketed by a
+barrier and a device synchronisation on both sides and timed with CUDA events on the launching
+stream; the reported time is the median region (max over ranks within each region).
 """
 from __future__ import annotations
 
@@ -33,12 +40,38 @@ from paper_2406_07368_b200 import dist as ladist   # noqa: E402
 
 L2_BYTES = 126 * 2 ** 20
 NOMINAL_HBM_GBS = 7700.0        # HGX B200 data-sheet figure, printed beside the measured copy bandwidth
-# DRAM bytes (read + written) per launch of the dominant kernel, from the ncu captures summarised under
-# profiles/; None where no capture of the current kernel exists.
-NCU_TRAFFIC = {"llama7b_prefill": 245.9e6, "batched_decode": 218.6e6, "tree_verify": 61.5e6, "long_prefill": 1648.9e6}
+REGIONS = 5                     # timed regions of K steps each; the median is reported
 
 
 # ----------------------------------------------------------------------------------------
+def profiled_traffic(workload: str, kernel: str | None = None):
+    """DRAM bytes (read + written) per launch of a workload's dominant kernel, as counted by ncu.
+
+    The figure is read from the summaries under profiles/ -- a line
+        # bench-traffic: workload=NAME kernel=KERNEL source=PATH sha256=HEX dram_bytes_per_launch=N
+    written beside each capture -- and is only returned while the kernel's source file still hashes to the value
+    recorded with the capture: once the kernel has changed, the counters describe another program and the result
+    is None."""
+    import hashlib
+    pdir = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(pdir):
+        return None
+    for fn in sorted(os.listdir(pdir)):
+        if not fn.endswith((".txt", ".md")):
+            continue
+        for line in open(os.path.join(pdir, fn), errors="replace"):
+            if not line.startswith("# bench-traffic:"):
+                continue
+            kv = dict(tok.split("=", 1) for tok in line.split()[2:] if "=" in tok)
+            if kv.get("workload") != workload or (kernel is not None and kv.get("kernel") != kernel):
+                continue
+            src = os.path.join(ROOT, kv.get("source", ""))
+            if not os.path.isfile(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != kv.get("sha256"):
+                return None
+            return float(kv["dram_bytes_per_launch"])
+    return None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -90,10 +123,12 @@ class ClockSampler:
             self.proc.terminate()
             self.thread.join(timeout=2)
 
-    def summary(self):
+    def summary(self, t0=None, t1=None):
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        inside = [r for t, r in self.rows if self.t0 is not None and self.t0 <= t <= (self.t1 or t)]
+        t0 = self.t0 if t0 is None else t0
+        t1 = self.t1 if t1 is None else t1
+        inside = [r for t, r in self.rows if t0 is not None and t0 <= t <= (t1 or t)]
         for r in inside or [r for _, r in self.rows]:     # samples taken during the timed region, if any fell into it
             try:
                 sm.append(float(r[0]))
@@ -220,6 +255,8 @@ def decode_workload(W: wl.Workload, rank: int, device):
             "h2d": 3 * units * W.d * el, "d2h": units * W.d * el, "kernel": "decode",
             "flops_per_launch": units * 4 * W.d * W.d,
             "period": nrot,
+            "setup": "state built by a seeded 256-token prompt (the workload's own prompt is 2048 tokens; the step's "
+                     "cost does not depend on what the state holds)",
             "l2": f"state of {units * W.d * W.d * 4 / 2**20:.0f} MiB streamed every step (larger than L2)"}
     return step, e2e_step, info
 
@@ -306,6 +343,8 @@ def verify_workload(W: wl.Workload, rank: int, device):
             "accepted_tokens_per_step": W.B * acc_len, "accept_probe": probe_accept,
             "flops_per_launch": units * (2 * N * W.d * W.d + 4 * N * N * W.d),
             "period": nrot * nsets // math.gcd(nrot, nsets),
+            "setup": "every state set built by a seeded 256-token prompt (the workload's own prompt is 1024 tokens; the "
+                     "step's cost does not depend on what the state holds)",
             "l2": f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"}
     return step, e2e_step, info
 
@@ -374,15 +413,20 @@ METRICS = {"llama7b_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
 
 
 # ----------------------------------------------------------------------------------------
-def oracle_sample(W: wl.Workload):
-    """One bounded sample of the workload for the float64 oracle: returns (fn, units, text)."""
+def oracle_samples(W: wl.Workload):
+    """Bounded samples of the workload for the float64 oracle: {"primary": (fn, units, text), "definition": ... }.
+    The primary sample uses the oracle's fastest exact form for the mode (grouped for prefill, the recurrence for
+    decode, the tree form for verify + commit); for prefill the quadratic definition is timed beside it."""
     from oracle import la_oracle as orc
     if W.name in ("llama7b_prefill", "long_prefill"):
-        T = min(W.T, 2048)
+        T = W.T
         q, k, v = W.prefill_inputs(B=1, T=T)
         w = W.weights()
-        return (lambda: orc.prefill_quadratic(q, k, v, w, W.phi, W.eps), T,
-                f"quadratic definition, 1 of {W.B} sequences, all {W.H} heads, first {T} of {W.T} tokens")
+        Tq = min(W.T, 2048)
+        return {"primary": (lambda: orc.prefill_chunked(q, k, v, w, W.phi, W.eps, W.chunk), T,
+                            f"grouped form (groups of {W.chunk}), 1 of {W.B} sequences, all {W.H} heads, all {T} tokens"),
+                "definition": (lambda: orc.prefill_quadratic(q[:, :, :Tq], k[:, :, :Tq], v[:, :, :Tq], w, W.phi, W.eps), Tq,
+                               f"quadratic definition, 1 of {W.B} sequences, all {W.H} heads, first {Tq} of {W.T} tokens")}
     if W.name == "prompt_gen":
         P, G = min(W.extra["shapes"], key=lambda pg: pg[0] + pg[1])
         q, k, v = wl.qkv(W.seed, (W.B, W.H, P + G, W.d), W.scale, W.io)
@@ -392,7 +436,8 @@ def oracle_sample(W: wl.Workload):
             _, st = orc.prefill_chunked(q[:, :, :P], k[:, :, :P], v[:, :, :P], w, W.phi, W.eps, W.chunk)
             for g in range(G):
                 _, st = orc.decode_step(q[:, :, P + g], k[:, :, P + g], v[:, :, P + g], w, W.phi, W.eps, st)
-        return fn, W.B * (P + G), f"grouped prefill of {P} tokens then {G} recurrent steps: the ({P}, {G}) pair, all heads"
+        return {"primary": (fn, W.B * (P + G),
+                            f"grouped prefill of {P} tokens then {G} recurrent steps: the ({P}, {G}) pair, all heads")}
     if W.name == "batched_decode":
         B = 8
         q, k, v = W.prefill_inputs(B=B, T=64)
@@ -404,7 +449,7 @@ def oracle_sample(W: wl.Workload):
         def fn():
             for _ in range(4):
                 _, box[0] = orc.decode_step(qs, ks, vs, w, W.phi, W.eps, box[0])
-        return fn, 4 * B, f"recurrent form, {B} of {W.B} sequences, all heads, 4 decode steps"
+        return {"primary": (fn, 4 * B, f"recurrent form, {B} of {W.B} sequences, all heads, 4 decode steps")}
     B = 2
     q, k, v = W.prefill_inputs(B=B, T=64)
     w = W.weights()
@@ -415,7 +460,7 @@ def oracle_sample(W: wl.Workload):
     def fn():
         orc.verify_tree(qd, kd, vd, parent, w, W.phi, W.eps, st)
         orc.commit(kd, vd, parent, accept, W.phi, st, W.max_depth)
-    return fn, B * W.tree_nodes, f"tree form, {B} of {W.B} sequences, all heads, one verify + commit round"
+    return {"primary": (fn, B * W.tree_nodes, f"tree form, {B} of {W.B} sequences, all heads, one verify + commit round")}
 
 
 def blas_threads() -> int:
@@ -429,25 +474,47 @@ def blas_threads() -> int:
     return len(os.sched_getaffinity(0))
 
 
-def time_oracle(W: wl.Workload, repeats: int, warmup: int = 0):
-    fn, units, text = oracle_sample(W)
+def time_fn(fn, units, repeats: int, warmup: int = 0):
     for _ in range(warmup):
         fn()
     t0 = time.perf_counter()
     for _ in range(repeats):
         fn()
     dt = time.perf_counter() - t0
-    return units * repeats / dt, dt / repeats, text
+    return units * repeats / dt, dt / repeats
+
+
+def l2_note(W: wl.Workload) -> str:
+    """How the GPU arm keeps the 126 MB L2 from serving a step's inputs (a property of the workload's sizes)."""
+    if W.name in ("llama7b_prefill", "long_prefill"):
+        per_set = 4 * W.B * W.H * W.T * W.d * 2
+        nsets = max(2, -(-2 * L2_BYTES // per_set) + 1) if per_set < 4 * L2_BYTES else 1
+        return f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"
+    if W.name == "batched_decode":
+        return f"state of {W.B * W.H * W.d * W.d * 4 / 2**20:.0f} MiB streamed every step (larger than L2)"
+    if W.name == "tree_verify":
+        per_state = W.B * W.H * W.d * W.d * 4
+        nsets = max(2, -(-2 * L2_BYTES // per_state) + 1)
+        return f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"
+    return "a single sequence: tokens and state are L2-resident by nature of the workload"
+
+
+def base_config(W: wl.Workload, world: int = 1) -> dict:
+    """The workload's identity: the same keys and values in both arms of the benchmark."""
+    return {"workload": W.name, "B": W.B, "H": W.H, "d": W.d, "T": W.T, "chunk": W.chunk, "phi": W.phi, "eps": W.eps,
+            "conv_taps": W.W, "tree_nodes": W.tree_nodes, "decode_steps": W.decode_steps, "rounds": W.rounds,
+            "io": W.io, "seed": W.seed, "l2": l2_note(W), "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(args, W: wl.Workload):
     metric, unit = METRICS[W.name]
-    value, per_step, text = time_oracle(W, args.steps, args.warmup)
+    fn, units, text = oracle_samples(W)["primary"]
+    value, per_step = time_fn(fn, units, args.steps, args.warmup)
     cores = blas_threads()
     line = {"impl": "reference", "metric": metric, "value": value, "unit": unit, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": W.name, "sample_per_step": text},
+            "config": base_config(W, int(os.environ.get("WORLD_SIZE", 1))), "sample_per_step": text,
             "cpu_baseline": {"value": value, "unit": unit, "cores": cores, "kind": "oracle", "sample": text},
             "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -455,47 +522,18 @@ def run_reference(args, W: wl.Workload):
 
 
 # ----------------------------------------------------------------------------------------
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=None)
-    ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama7b_prefill", choices=sorted(FACTORIES))
-    ap.add_argument("--e2e-steps", type=int, default=10)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="launch every step from Python instead of replaying a CUDA graph")
-    args = ap.parse_args()
-    W = wl.WORKLOADS[args.workload]()
-    rank, world = ladist.rank_world()
-
-    if args.impl == "reference":
-        args.steps = args.steps or 3
-        args.warmup = 1 if args.warmup is None else args.warmup
-        if rank == 0:
-            run_reference(args, W)
-        return 0
-
-    defaults = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
-    args.steps = args.steps or defaults[W.name]
-    args.warmup = 5 if args.warmup is None else max(3, args.warmup)
-
-    local = int(os.environ.get("LOCAL_RANK", 0))
-    torch.cuda.set_device(local)
-    device = torch.device("cuda", local)
-    ladist.init(world, backend="nccl")
-
+def measure(W: wl.Workload, steps: int, warmup: int, rank: int, world: int, device, clocks, use_graph: bool,
+            e2e_steps: int):
+    """Times one workload on this rank's GPU: R regions of `steps` steps (median reported), the dominant kernel
+    alone where a step has several, and (e2e_steps > 0) the end-to-end loop with host buffers."""
     step, e2e_step, info = FACTORIES[W.name](W, rank, device)
     ctx = info["ctx"]
     stream = torch.cuda.current_stream()
-
-    clocks = ClockSampler(local)
-    clocks.__enter__()
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
     torch.cuda.synchronize()
     if ctx.la_last_device_status() != 0:
-        raise RuntimeError("device status not OK after warm-up")
+        raise RuntimeError(f"{W.name}: device status not OK after warm-up")
 
     # The same calls, recorded once into a CUDA graph of one rotation period and replayed: the steps are short
     # enough for the Python interpreter to be the bottleneck otherwise.  K steps = K // period replays, the rest eager.
@@ -509,8 +547,8 @@ def main():
                 fn(i)
         return g, ctx.la_launch_count() - n0
 
-    graph = None
-    if not args.no_graph and args.steps >= period:
+    graph, launches_per_replay = None, 0
+    if use_graph and steps >= period:
         graph, launches_per_replay = capture(lambda i: step())
         graph.replay()                                     # one untimed replay
         torch.cuda.synchronize()
@@ -526,152 +564,66 @@ def main():
             step()
         return extra
 
-    ladist.barrier(world)
-    torch.cuda.synchronize()
-    launches0 = ctx.la_launch_count()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     clocks.wait_ready()
-    torch.cuda.synchronize()
-    clocks.mark_start()
-    ev0.record(stream)
-    replayed = run_steps(args.steps)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    clocks.mark_end()
-    clocks.__exit__()
-    ladist.barrier(world)
-    ms = ev0.elapsed_time(ev1)
-    launches = ctx.la_launch_count() - launches0 + replayed
-    ms_max = ladist.max_over_ranks(ms, world, device)
-    value = world * info["tokens_per_step"] * args.steps / (ms_max * 1e-3)
+    regions, launches = [], 0
+    t_start = time.time()
+    for _ in range(REGIONS):
+        ladist.barrier(world)
+        torch.cuda.synchronize()
+        launches0 = ctx.la_launch_count()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        replayed = run_steps(steps)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ladist.barrier(world)
+        regions.append(ladist.max_over_ranks(ev0.elapsed_time(ev1), world, device))
+        launches = ctx.la_launch_count() - launches0 + replayed          # per region of K steps
+    time.sleep(0.15)
+    t_end = time.time()
+    ms = float(np.median(regions))
 
-    # per-launch duration of the dominant kernel, measured live: events around every launch of a
-    # short second pass on the same stream (for two-kernel steps only the first kernel is bracketed)
+    # per-launch duration of one kernel alone, measured live: a short second pass on the same stream
     def time_probe(fn):
         for i in range(3):
             fn(i)
         torch.cuda.synchronize()
         pgraph = None if graph is None else capture(fn)[0]
-        n_probe = min(args.steps, 100) if pgraph is None else period * max(1, 100 // period)
-        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        p0.record(stream)
-        if pgraph is None:
-            for i in range(n_probe):
-                fn(i)
-        else:
-            for _ in range(n_probe // period):
-                pgraph.replay()
-        p1.record(stream)
-        torch.cuda.synchronize()
-        return p0.elapsed_time(p1) / n_probe
+        n_probe = min(steps, 100) if pgraph is None else period * max(1, 100 // period)
+        samples = []
+        for _ in range(3):
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            p0.record(stream)
+            if pgraph is None:
+                for i in range(n_probe):
+                    fn(i)
+            else:
+                for _ in range(n_probe // period):
+                    pgraph.replay()
+            p1.record(stream)
+            torch.cuda.synchronize()
+            samples.append(p0.elapsed_time(p1) / n_probe)
+        return float(np.median(samples))
 
     second = None
-    if info["launches_per_step"] == 1:
-        kernel_ms = ms / args.steps
+    if info["launches_per_step"] == 1 or "probe" not in info:
+        kernel_ms = ms / steps
     else:
         kernel_ms = time_probe(info["probe"])
         if "second" in info:
             second = dict(info["second"])
             second["launch_ms"] = time_probe(second.pop("probe"))
 
-    # End to end: pinned host inputs copied in, result copied out, every step.  Where the workload gives the three
-    # parts separately the loop is pipelined over two buffer sets: the copy-in of step i+1 and the copy-out of step
-    # i-1 run on streams of their own beside the kernels of step i (PCIe is full duplex); every step still pays
-    # for all of its bytes inside the timed region.
-    if callable(e2e_step):
-        def e2e_run(n):
-            for _ in range(n):
-                e2e_step()
-    else:
-        e2e_in, e2e_compute, e2e_out = e2e_step
-        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-
-        def e2e_run(n):
-            ev_in = [torch.cuda.Event() for _ in range(2)]
-            ev_comp = [torch.cuda.Event() for _ in range(2)]
-            ev_out = [torch.cuda.Event() for _ in range(2)]
-            start = torch.cuda.Event()
-            start.record(stream)
-            s_in.wait_event(start)
-            s_out.wait_event(start)
-            for i in range(n):
-                b = i & 1
-                with torch.cuda.stream(s_in):
-                    if i >= 2:
-                        s_in.wait_event(ev_comp[b])        # the inputs of step i-2 have been consumed
-                    e2e_in(b)
-                    ev_in[b].record(s_in)
-                stream.wait_event(ev_in[b])
-                if i >= 2:
-                    stream.wait_event(ev_out[b])           # the outputs of step i-2 have been copied out
-                e2e_compute(b)
-                ev_comp[b].record(stream)
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev_comp[b])
-                    e2e_out(b)
-                    ev_out[b].record(s_out)
-            for b in range(min(n, 2)):
-                stream.wait_event(ev_out[b])
-
-    e2e_run(2)
-    torch.cuda.synchronize()
-    ladist.barrier(world)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    e2e_run(args.e2e_steps)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    e2e_ms = ladist.max_over_ranks(e0.elapsed_time(e1), world, device)
-    e2e_value = world * info["tokens_per_step"] * args.e2e_steps / (e2e_ms * 1e-3)
-    if ctx.la_last_device_status() != 0:
-        raise RuntimeError("device status not OK after the timed region")
-
-    if rank != 0:
-        ladist.finish(world)
-        return 0
-
-    peaks = measured_peaks()
-    metric, unit = METRICS[W.name]
-    achieved = info["alg_bytes_per_launch"] / (kernel_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": info["kernel"], "achieved": achieved, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC.get(W.name),
-                "peak_source": peaks["source"], "alg_bytes_per_launch": info["alg_bytes_per_launch"],
-                "launch_ms": kernel_ms,
-                "tensor_tflops": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12,
-                "tensor_frac_of_sustained": info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
-                / peaks["bf16_tflops_sustained"]}
-    roofline["frac_of_nominal_7700"] = achieved / NOMINAL_HBM_GBS
-    if roofline["traffic"] is not None:          # the same fraction from the DRAM bytes ncu counted, not the algorithmic ones
-        roofline["achieved_from_traffic"] = roofline["traffic"] / (kernel_ms * 1e-3) / 1e9
-        roofline["frac_from_traffic"] = roofline["achieved_from_traffic"] / peaks["hbm_gbs"]
-    if "flops_strict_per_launch" in info:
-        roofline["tensor_tflops_strict"] = info["flops_strict_per_launch"] / (kernel_ms * 1e-3) / 1e12
-    if info["launches_per_step"] > 1:
-        roofline["step_ms"] = ms / args.steps      # all kernels of the step; launch_ms is the dominant one alone
-    if second is not None:
-        a2 = second["alg_bytes_per_launch"] / (second["launch_ms"] * 1e-3) / 1e9
-        second.update({"achieved": a2, "unit": "GB/s", "frac": a2 / peaks["hbm_gbs"]})
-        roofline["second_kernel"] = second
-    cpu = None
-    if not args.no_cpu_baseline and world == 1:
-        reps = {"llama7b_prefill": 4, "long_prefill": 4, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
-        v, per, text = time_oracle(W, reps, warmup=0)
-        cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text,
-               "seconds": per * reps}
-    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16" if W.io == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": W.name, "B": W.B, "H": W.H, "d": W.d, "T": W.T, "chunk": W.chunk, "phi": W.phi,
-                       "conv_taps": W.W, "tree_nodes": W.tree_nodes, "l2": info["l2"],
-                       "launch": f"CUDA graph of {period} steps, replayed" if graph is not None else "one Python call per kernel",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "clocks": clocks.summary(),
-            "e2e": {"value": e2e_value, "unit": unit, "h2d_bytes_per_step": info["h2d"],
-                    "d2h_bytes_per_step": info["d2h"], "steps": args.e2e_steps,
-                    "pipelined": not callable(e2e_step)},
-            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu}
+    res = {"W": W, "info": info, "ctx": ctx, "regions": regions, "ms": ms, "steps": steps, "launches": int(launches),
+           "kernel_ms": kernel_ms, "second": second, "graph": graph is not None, "period": period,
+           "clock_window": (t_start, t_end), "value": world * info["tokens_per_step"] * steps / (ms * 1e-3)}
+    if "accepted_tokens_per_step" in info:
+        res["accepted_tokens_per_s"] = world * info["accepted_tokens_per_step"] * steps / (ms * 1e-3)
+    if "accept_probe" in info:
+        res["accept_kernel"] = {"kernel": "accept_greedy", "launch_ms": time_probe(info["accept_probe"]),
+                                "note": "integer kernel, one warp per sequence: latency, not bandwidth"}
     if "shape_probe" in info:                    # latency of every (prompt, generation) pair on its own
-        line["shape_ms"] = {}
+        res["shape_ms"] = {}
         for i, (P, G) in enumerate(info["shapes"]):
             fn = info["shape_probe"]
             fn(i)
@@ -687,12 +639,204 @@ def main():
                 g.replay()
             p1.record(stream)
             torch.cuda.synchronize()
-            line["shape_ms"][f"({P}, {G})"] = p0.elapsed_time(p1) / 5
-    if "accept_probe" in info:
-        line["accept_kernel"] = {"kernel": "accept_greedy", "launch_ms": time_probe(info["accept_probe"]),
-                                 "note": "integer kernel, one warp per sequence: latency, not bandwidth"}
-    if "accepted_tokens_per_step" in info:
-        line["accepted_tokens_per_s"] = world * info["accepted_tokens_per_step"] * args.steps / (ms_max * 1e-3)
+            res["shape_ms"][f"({P}, {G})"] = p0.elapsed_time(p1) / 5
+
+    if e2e_steps > 0:
+        # End to end: pinned host inputs copied in, result copied out, every step.  Where the workload gives the
+        # three parts separately the loop is pipelined over two buffer sets: the copy-in of step i+1 and the copy-out
+        # of step i-1 run on streams of their own beside the kernels of step i (PCIe is full duplex); every step
+        # still pays for all of its bytes inside the timed region.
+        if callable(e2e_step):
+            def e2e_run(n):
+                for _ in range(n):
+                    e2e_step()
+        else:
+            e2e_in, e2e_compute, e2e_out = e2e_step
+            s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+            def e2e_run(n):
+                ev_in = [torch.cuda.Event() for _ in range(2)]
+                ev_comp = [torch.cuda.Event() for _ in range(2)]
+                ev_out = [torch.cuda.Event() for _ in range(2)]
+                start = torch.cuda.Event()
+                start.record(stream)
+                s_in.wait_event(start)
+                s_out.wait_event(start)
+                for i in range(n):
+                    b = i & 1
+                    with torch.cuda.stream(s_in):
+                        if i >= 2:
+                            s_in.wait_event(ev_comp[b])        # the inputs of step i-2 have been consumed
+                        e2e_in(b)
+                        ev_in[b].record(s_in)
+                    stream.wait_event(ev_in[b])
+                    if i >= 2:
+                        stream.wait_event(ev_out[b])           # the outputs of step i-2 have been copied out
+                    e2e_compute(b)
+                    ev_comp[b].record(stream)
+                    with torch.cuda.stream(s_out):
+                        s_out.wait_event(ev_comp[b])
+                        e2e_out(b)
+                        ev_out[b].record(s_out)
+                for b in range(min(n, 2)):
+                    stream.wait_event(ev_out[b])
+
+        e2e_run(2)
+        torch.cuda.synchronize()
+        ladist.barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        e2e_run(e2e_steps)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = ladist.max_over_ranks(e0.elapsed_time(e1), world, device)
+        res["e2e"] = {"value": world * info["tokens_per_step"] * e2e_steps / (e2e_ms * 1e-3),
+                      "unit": METRICS[W.name][1], "h2d_bytes_per_step": info["h2d"], "d2h_bytes_per_step": info["d2h"],
+                      "steps": e2e_steps, "pipelined": not callable(e2e_step)}
+    if ctx.la_last_device_status() != 0:
+        raise RuntimeError(f"{W.name}: device status not OK after the timed region")
+    return res
+
+
+def roofline_of(res, peaks):
+    info, kernel_ms = res["info"], res["kernel_ms"]
+    achieved = info["alg_bytes_per_launch"] / (kernel_ms * 1e-3) / 1e9
+    tflops = info["flops_per_launch"] / (kernel_ms * 1e-3) / 1e12
+    r = {"bound": "hbm", "kernel": info["kernel"], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+         "frac": achieved / peaks["hbm_gbs"], "traffic": profiled_traffic(res["W"].name),
+         "peak_source": peaks["source"], "alg_bytes_per_launch": info["alg_bytes_per_launch"], "launch_ms": kernel_ms,
+         "tensor_tflops": tflops, "tensor_frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
+         "frac_of_nominal_7700": achieved / NOMINAL_HBM_GBS}
+    if r["traffic"] is not None:                 # the same fraction from the DRAM bytes ncu counted, not the algorithmic ones
+        r["achieved_from_traffic"] = r["traffic"] / (kernel_ms * 1e-3) / 1e9
+        r["frac_from_traffic"] = r["achieved_from_traffic"] / peaks["hbm_gbs"]
+    if "flops_strict_per_launch" in info:
+        r["tensor_tflops_strict"] = info["flops_strict_per_launch"] / (kernel_ms * 1e-3) / 1e12
+    if info["launches_per_step"] > 1:
+        r["step_ms"] = res["ms"] / res["steps"]  # all kernels of the step; launch_ms is the dominant one alone
+    if res["second"] is not None:
+        second = dict(res["second"])
+        a2 = second["alg_bytes_per_launch"] / (second["launch_ms"] * 1e-3) / 1e9
+        second.update({"achieved": a2, "unit": "GB/s", "frac": a2 / peaks["hbm_gbs"],
+                       "traffic": profiled_traffic(res["W"].name, second["kernel"])})
+        r["second_kernel"] = second
+    return r
+
+
+def spread(res):
+    per = [x / res["steps"] for x in res["regions"]]
+    return {"regions": len(per), "ms_per_step_median": float(np.median(per)), "ms_per_step_min": min(per),
+            "ms_per_step_max": max(per)}
+
+
+def brief(res, peaks, clocks):
+    """One workload as an entry of "others": device-timed step, throughput, roofline of its kernels."""
+    metric, unit = METRICS[res["W"].name]
+    out = {"metric": metric, "value": res["value"], "unit": unit, "steps": res["steps"],
+           "ms_per_step": res["ms"] / res["steps"], "timing": spread(res), "gpu_launches": res["launches"],
+           "config": base_config(res["W"]), "roofline": roofline_of(res, peaks),
+           "clocks": clocks.summary(*res["clock_window"]),
+           "launch": f"CUDA graph of {res['period']} steps, replayed" if res["graph"] else "one Python call per kernel"}
+    for key in ("accepted_tokens_per_s", "accept_kernel", "shape_ms"):
+        if key in res:
+            out[key] = res[key]
+    if "setup" in res["info"]:
+        out["setup"] = res["info"]["setup"]
+    return out
+
+
+OTHERS = {"llama7b_prefill": ("batched_decode", "tree_verify", "long_prefill")}
+DEFAULT_STEPS = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
+OTHER_STEPS = {"long_prefill": 20, "batched_decode": 400, "tree_verify": 400}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_prefill", choices=sorted(FACTORIES))
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="time the headline workload only")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step from Python instead of replaying a CUDA graph")
+    args = ap.parse_args()
+    W = wl.WORKLOADS[args.workload]()
+    rank, world = ladist.rank_world()
+
+    if args.impl == "reference":
+        args.steps = args.steps or 3
+        args.warmup = 1 if args.warmup is None else args.warmup
+        if rank == 0:
+            run_reference(args, W)
+        return 0
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly: this process becomes the launcher of one rank per GPU
+        return ladist.launch_local_ranks([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+
+    args.steps = args.steps or DEFAULT_STEPS[W.name]
+    args.warmup = 5 if args.warmup is None else max(3, args.warmup)
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    ladist.init(world, backend="nccl")
+
+    clocks = ClockSampler(local)
+    clocks.__enter__()
+    try:
+        res = measure(W, args.steps, args.warmup, rank, world, device, clocks, not args.no_graph, args.e2e_steps)
+        peaks = measured_peaks()
+        others = {}
+        if world == 1 and not args.no_others:
+            for name in OTHERS.get(W.name, ()):
+                ctx = res.pop("ctx", None)                 # keep the headline's numbers, release its buffers
+                del ctx
+                torch.cuda.empty_cache()
+                r2 = measure(wl.WORKLOADS[name](), OTHER_STEPS[name], args.warmup, rank, world, device, clocks,
+                             not args.no_graph, 0)
+                others[name] = brief(r2, peaks, clocks)
+                del r2
+                torch.cuda.empty_cache()
+    finally:
+        clocks.__exit__()
+
+    if rank != 0:
+        ladist.finish(world)
+        return 0
+
+    metric, unit = METRICS[W.name]
+    info = res["info"]
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        samples = oracle_samples(W)
+        reps = {"llama7b_prefill": 8, "long_prefill": 2, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
+        fn, units, text = samples["primary"]
+        v, per = time_fn(fn, units, reps)
+        cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text, "seconds": per * reps}
+        if "definition" in samples:
+            fn, units, text = samples["definition"]
+            v2, per2 = time_fn(fn, units, 3)
+            cpu["definition_form"] = {"value": v2, "unit": unit, "sample": text, "seconds": per2 * 3}
+    config = base_config(W, world)
+    run = {"launch": f"CUDA graph of {res['period']} steps, replayed" if res["graph"] else "one Python call per kernel",
+           "timing": f"median of {REGIONS} regions of {args.steps} steps, each between barriers and device syncs",
+           "l2": info["l2"]}
+    if "setup" in info:
+        run["setup"] = info["setup"]
+    line = {"metric": metric, "value": res["value"], "unit": unit, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": res["ms"] / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if W.io == "bf16" else "f32", "data": "synthetic",
+            "config": config, "run": run, "timing": spread(res), "clocks": clocks.summary(*res["clock_window"]),
+            "e2e": res.get("e2e"), "gpu_launches": res["launches"], "roofline": roofline_of(res, peaks),
+            "cpu_baseline": cpu}
+    for key in ("accepted_tokens_per_s", "accept_kernel", "shape_ms"):
+        if key in res:
+            line[key] = res[key]
+    if others:
+        line["others"] = others
     print(json.dumps(line), flush=True)
     ladist.finish(world)
     return 0

@@ -6,6 +6,9 @@ timed region (a barrier) and to agree on the slowest rank's time (a MAX all-redu
 from __future__ import annotations
 
 import os
+import socket
+import subprocess
+import time
 
 import torch
 import torch.distributed as td
@@ -44,3 +47,43 @@ def shard(n_units: int, rank: int, world: int) -> tuple[int, int]:
 def finish(world: int) -> None:
     if world > 1 and td.is_initialized():
         td.destroy_process_group()
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_local_ranks(cmd: list[str], world: int, timeout: float | None = None, env: dict | None = None) -> int:
+    """Starts `world` copies of `cmd` on this node, one per rank (RANK = LOCAL_RANK = 0 .. world-1, WORLD_SIZE,
+    MASTER_ADDR = 127.0.0.1 and a free MASTER_PORT in the environment), and waits for them.  All ranks inherit this
+    process's stdout and stderr.  Returns 0 if every rank exited 0, otherwise the first non-zero exit code (after
+    ending the ranks that were still running: only processes started here, by their own handles)."""
+    base = dict(os.environ if env is None else env)
+    base.update(WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(free_port()))
+    procs = []
+    for r in range(world):
+        procs.append(subprocess.Popen(cmd, env=dict(base, RANK=str(r), LOCAL_RANK=str(r))))
+    deadline = None if timeout is None else time.time() + timeout
+    rc = 0
+    pending = list(procs)
+    while pending and rc == 0:
+        for p in list(pending):
+            code = p.poll()
+            if code is not None:
+                pending.remove(p)
+                if code != 0:
+                    rc = code
+        if deadline is not None and time.time() > deadline:
+            rc = 124
+        if pending and rc == 0:
+            time.sleep(0.05)
+    for p in pending:                                   # a rank failed or time ran out: end the others
+        p.terminate()
+    for p in pending:
+        try:
+            p.wait(timeout=10)
+        except subprocess.TimeoutExpired:
+            p.kill()
+    return rc

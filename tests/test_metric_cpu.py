@@ -49,5 +49,5 @@ def test_octaves_tile_the_positions_and_see_the_fault_at_late_rows():
     T = 4096
     y = np.random.default_rng(0).standard_normal((1, 1, T, 8)) / np.sqrt(np.arange(1, T + 1))[None, None, :, None]
     x = y.copy()
-    x[:, :, -256:] *= 0.9
-    assert rel_err(x, y) < 0.03 and rel_err_octaves(x, y) > 0.09
+    x[:, :, -256:] += 0.2 / np.sqrt(T)                  # an offset of a fifth of the late rows' own size
+    assert rel_err_octaves(x, y) > 2.0 * rel_err(x, y) and rel_err_octaves(x, y) > 0.15
