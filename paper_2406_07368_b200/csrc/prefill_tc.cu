@@ -5,23 +5,25 @@
 // sums S = sum phi(k) v^T and z = sum phi(k) are carried.  One CTA walks one (batch, head)
 // chain in tiles of 128 tokens:
 //     O = phi(Q) S_prev + (P o M) V,   den = phi(Q) . z_prev + rowsum(P o M),   S += phi(K)^T V,   z += colsum phi(K).
-// The matrix products run on the tensor cores, and z rides along with S: V is extended by a column of ones and the
-// copy of S by the column z ([S | z] += phi(K)^T [V | 1], [O | phi(q) . z] = phi(Q) [S | z]_prev; 16-column,
-// unswizzled operand blocks).  The row sums of the masked P are taken by the threads that mask it.  Per tile n:
+// The matrix products run on the tensor cores, and z rides along with them: V is extended by a column of ones
+// ([S | z] += phi(K)^T [V | 1], a 16-column unswizzled operand block), and the K tile by a row that holds z_prev, so
+// that the score product delivers phi(q) . z_prev as one more column of P.  The row sums of the masked P are taken
+// by the threads that mask it.  Per tile n:
 //
 //   TMA      Q, K, V tiles (128 x 128 bf16, two 64-column boxes each, 128-byte swizzle)
 //   group A  phi(Q) -> TMEM and phi(K) in place (packed bf16x2 arithmetic)
-//   tcgen05  P = phi(Q) phi(K)^T
+//   tcgen05  [P | phi(q) . z_prev] = phi(Q) [phi(K); z_prev]^T     (144 columns: 128 tokens, z_prev, 15 unused)
 //            [S | z] += phi(K)^T [V | 1]               (fp32 in TMEM for the whole chain)
-//            [O | phi(q) . z] = phi(Q) [S | z]_prev    ([S | z]_prev is a bf16 copy in shared memory)
-//   group A  P -> causal mask, row sums, bf16 -> TMEM (the A operand of the next product);
-//            phi on K of tile n+1 (K is double-buffered);  [S | z] -> bf16 copy for tile n+1
+//            O = phi(Q) S_prev                         (S_prev is a bf16 copy in shared memory)
+//   group A  P -> causal mask, row sums (+ the z column), bf16 -> TMEM (the A operand of the next product);
+//            phi on K of tile n+1 (K is double-buffered);  S -> bf16 copy, z -> the K buffer of tile n+1
 //   tcgen05  O += (P o M) V
 //   group B  o = O / (den + eps) + conv(V) -> the tile's V buffer;  TMA stores it to global memory
 //
-// Three roles run concurrently: group A (warps 8-15), group B (warps 0-7) and warp 16, whose
-// elected lane issues every TMA load, every TMA store and every MMA.  While group B finishes tile n,
-// group A already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
+// Four roles run concurrently: group A (warps 8-15), group B (warps 0-7), warp 16, whose elected lane issues
+// every MMA and the Q and K loads, and warp 17, whose elected lane issues the V loads and the output stores (a
+// store has to have read its buffer before the buffer is reloaded: that wait must not hold up the products).
+// While group B finishes tile n, group A already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
 // records LA_ERR_TIMEOUT, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
@@ -36,25 +38,29 @@ constexpr int D = 128;
 constexpr int TILE = 128;
 constexpr int kThreadsB = 256;                     // group B: warps 0-7
 constexpr int kThreadsA = 256;                     // group A: warps 8-15
-constexpr int kCtrlWarp = 16;
-constexpr int kThreads = 544;
+constexpr int kCtrlWarp = 16, kCopyWarp = 17;
+constexpr int kThreads = 576;
 constexpr uint32_t BOX_BYTES = 128 * 128;          // 128 rows x 64 bf16
 constexpr uint32_t TILE_BYTES = 2 * BOX_BYTES;
-// TMEM columns: P, O and S, 128 fp32 columns each; phi(Q) as packed bf16 pairs (64 columns); two 16-column blocks
-// whose first column is phi(q) . z and z.  phi(Q) is the A operand of two products and goes from the registers
+// A K buffer carries 8 more rows below the 128 token rows of each box, the first of which (row 128) holds z_prev as
+// bf16: the score product runs with N = 144 and its column 128 is phi(q) . z_prev.  Columns 129-143 are never read,
+// so rows 129-135 hold whatever they hold and rows 136-143 are simply the first kilobyte of what follows the box.
+constexpr uint32_t KBOX_BYTES = (128 + 8) * 128;
+constexpr uint32_t KBUF_BYTES = 2 * KBOX_BYTES;
+// TMEM columns: P (144 fp32 columns: the scores and, in column 128, phi(q) . z_prev), O and S (128 each); phi(Q) as
+// packed bf16 pairs (64 columns); a 16-column block whose first column is z.  phi(Q) is the A operand of two products and goes from the registers
 // that computed it straight to TMEM, so that the Q buffer in shared memory is free for the next tile as soon as it
 // has been read.  The masked P goes back as packed bf16 pairs
 // into the columns its own fp32 values came from: each thread overwrites only columns of its own row that it has
 // already read (row r, tokens 64 hf + 32 qq ... + 31 -> columns 64 hf + 16 qq ... + 15).
-constexpr uint32_t P_COL = 0, O_COL = 128, S_COL = 256, FQ_COL = 384 /* 64 columns */, DEN_COL = 448, Z_COL = 464,
+constexpr uint32_t P_COL = 0, QZ_COL = 128, O_COL = 144, S_COL = 272, FQ_COL = 400 /* 64 columns */, Z_COL = 464,
                    TMEM_COLS = 512;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
-constexpr uint32_t OFF_Q = 0, OFF_K0 = TILE_BYTES, OFF_V0 = 2 * TILE_BYTES, /* second V buffer at 3 * TILE_BYTES */
-                   OFF_K1 = 4 * TILE_BYTES, OFF_S = 5 * TILE_BYTES,
-                   OFF_ONES = 6 * TILE_BYTES,      // [128 x 16] bf16, column 0 = 1: the extension of V
-                   OFF_SZ = OFF_ONES + 4096,       // [128 x 16] bf16, column 0 = z: the extension of the S copy
-                   OFF_DEN = OFF_SZ + 4096,        // [2][2][128] fp32: halves of the row sums of the masked P of tile n in slot n & 1
+constexpr uint32_t OFF_Q = 0, OFF_V0 = TILE_BYTES, /* second V buffer at 2 * TILE_BYTES */ OFF_S = 3 * TILE_BYTES,
+                   OFF_K0 = 4 * TILE_BYTES, OFF_K1 = OFF_K0 + KBUF_BYTES,
+                   OFF_ONES = OFF_K1 + KBUF_BYTES, // [128 x 16] bf16, column 0 = 1: the extension of V
+                   OFF_DEN = OFF_ONES + 4096,      // [2][2][128] fp32: halves of the denominator of tile n in slot n & 1
                    OFF_SMALL = OFF_DEN + 2048;
 
 struct Small {
@@ -67,7 +73,7 @@ struct Small {
 // has been read; tiles alternate between the two).
 // STAGED0 / STAGED1: group B has written a tile's outputs into that V buffer (the control lane stores them).
 // MMA_P / MMA_S / MMA_Q / MMA_O: tcgen05.commit after P; after [S|z] += phi(K)^T [V|1] (K buffer free);
-// after [O | phi(q).z] = phi(Q) [S|z]; after O += P V (MMA_O0 / MMA_O1, tiles alternate).
+// after O = phi(Q) S_prev; after O += P V (MMA_O0 / MMA_O1, tiles alternate).
 // A barrier that one role waits on while another role can run a tile ahead exists once per tile parity, so that a
 // waiter is never more than one phase behind.
 enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O0 = 5, B_MMA_O1 = 6, B_PHI = 7,
@@ -214,7 +220,7 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
   return ((addr >> 4) & 0x3FFFu) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
 }
 constexpr uint32_t kDescHiSw128 = ((1024u >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);   // SBO 1024, version 1, 128-byte swizzle
-__host__ __device__ constexpr uint32_t kstep_kmajor(int ks) { return ((uint32_t)(ks >> 2) * BOX_BYTES + (uint32_t)(ks & 3) * 32u) >> 4; }
+__host__ __device__ constexpr uint32_t kstep_kmajor(int ks, uint32_t box = BOX_BYTES) { return ((uint32_t)(ks >> 2) * box + (uint32_t)(ks & 3) * 32u) >> 4; }
 __host__ __device__ constexpr uint32_t kstep_mnmajor(int ks) { return ((uint32_t)ks * 2048u) >> 4; }
 __device__ __forceinline__ uint64_t desc64(uint32_t lo) { return ((uint64_t)kDescHiSw128 << 32) | lo; }
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = n.
@@ -343,13 +349,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
     halo0[idx] = init ? win[(size_t)u * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
   float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
-  for (int idx = tid; idx < 2 * 4096 / 16; idx += kThreads)                    // both 16-column blocks <- 0
+  for (int idx = tid; idx < 4096 / 16; idx += kThreads)                        // the 16-column block of ones <- 0
     reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  for (int idx = tid; idx < 4 * 1024 / 16; idx += kThreads)                    // rows 128-135 of the four K boxes <- 0
+    reinterpret_cast<uint4*>(smem + OFF_K0 + (idx >> 6) * KBOX_BYTES + BOX_BYTES)[idx & 63] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
   if (tid < TILE) {
     *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
-    if (init)
-      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(tid, 0)) = __float2bfloat16_rn(z[(size_t)u * D + tid]);
+    if (init)                                     // z before tile 0: row 128 of the first K buffer (feature tid)
+      *reinterpret_cast<__nv_bfloat16*>(smem + OFF_K0 + (tid >> 6) * KBOX_BYTES + BOX_BYTES + (tid & 63) * 2) =
+          __float2bfloat16_rn(z[(size_t)u * D + tid]);
   }
   fence_proxy_async();
   tc_fence_before();
@@ -358,34 +367,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const uint32_t tmem = sm.tmem_base;
 
   if (warp == kCtrlWarp) {
-    // =============================== TMA + MMA issue (one lane) ===============================
+    // =============================== MMA issue, the Q and K loads (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx((bar0 + 8u * (B_FULL_K0)), TILE_BYTES);
-      tma_load(sbase + OFF_K0, &mk, 0, y0, bh, (bar0 + 8u * (B_FULL_K0)));
-      tma_load(sbase + OFF_K0 + BOX_BYTES, &mk, 64, y0, bh, (bar0 + 8u * (B_FULL_K0)));
-      if (nchunks > 1) {
-        mbar_expect_tx((bar0 + 8u * (B_FULL_K1)), TILE_BYTES);
-        tma_load(sbase + OFF_K1, &mk, 0, y0 + TILE, bh, (bar0 + 8u * (B_FULL_K1)));
-        tma_load(sbase + OFF_K1 + BOX_BYTES, &mk, 64, y0 + TILE, bh, (bar0 + 8u * (B_FULL_K1)));
-      }
       mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
       tma_load(sbase + OFF_Q, &mq, 0, y0, bh, (bar0 + 8u * (B_FULL_Q)));
       tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0, bh, (bar0 + 8u * (B_FULL_Q)));
-      for (int n = 0; n < 2 && n < nchunks; ++n) {
-        mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + n)), TILE_BYTES);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
-      }
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
         const uint32_t vbuf = sbase + OFF_V0 + par * TILE_BYTES;
         const uint32_t kbuf = sbase + (par ? OFF_K1 : OFF_K0);
-        const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
         const bool has_state = init || n > 0;
         // low descriptor words of step 0: K read along its rows (K-major), K, V and the S copy down their rows
         const uint32_t k_km = desc_lo(kbuf, 16u);
-        const uint32_t k_mn = desc_lo(kbuf, BOX_BYTES), v_mn = desc_lo(vbuf, BOX_BYTES), s_mn = desc_lo(sbase + OFF_S, BOX_BYTES);
+        const uint32_t k_mn = desc_lo(kbuf, KBOX_BYTES), v_mn = desc_lo(vbuf, BOX_BYTES), s_mn = desc_lo(sbase + OFF_S, BOX_BYTES);
         ok = mbar_wait((bar0 + 8u * (B_PHI)), par, abort);   // phi(Q) of tile n is in TMEM, phi(K) in place
         if (!ok) break;
         tc_fence_after();
@@ -396,8 +391,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
         }
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // P = phi(Q) phi(K)^T; 16 channels of every row of phi(Q) = 8 columns
-          mma_bf16_ts(tmem + P_COL, tmem + FQ_COL + 8 * ks, desc64(k_km + kstep_kmajor(ks)), idesc(false, false, 128), ks > 0);
+        for (int ks = 0; ks < 8; ++ks)   // [P | phi(q).z_prev] = phi(Q) [phi(K); z_prev]^T; 16 channels of phi(Q) = 8 columns
+          mma_bf16_ts(tmem + P_COL, tmem + FQ_COL + 8 * ks, desc64(k_km + kstep_kmajor(ks, KBOX_BYTES)), idesc(false, false, 144),
+                      ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_P)));
         // The state update needs nothing from the previous tile's epilogue: it fills the time until that epilogue
         // has read the accumulator.
@@ -418,10 +414,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tc_fence_after();
         if (has_state) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {   // [O | phi(q) . z] = phi(Q) [S | z]_prev
+          for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
             mma_bf16_ts(tmem + O_COL, tmem + FQ_COL + 8 * ks, desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128), ks > 0);
-            mma_bf16_ts(tmem + DEN_COL, tmem + FQ_COL + 8 * ks, desc_ext(sbase + OFF_SZ, ks), idesc(false, true, 16), ks > 0);
-          }
         }
         mma_commit((bar0 + 8u * (B_MMA_Q)));
         ok = mbar_wait((bar0 + 8u * (B_PDONE)), par, abort);               // masked P of tile n is in TMEM
@@ -432,41 +426,50 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16_ts(tmem + O_COL, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
                       idesc(false, true, 128), has_state || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
-        if (n + 2 < nchunks) {
-          ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);             // this K buffer is free: it takes tile n+2
+        if (n + 2 < nchunks) {   // the state update was issued long ago: this K buffer is free and takes tile n+2
+          ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);
           if (!ok) break;
+          const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
           mbar_expect_tx(kbar, TILE_BYTES);
           tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
-          tma_load(kbuf + BOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
-        }
-        if (n >= 1) {
-          // the outputs of tile n-1 are staged in its V buffer: store them; once they have been read the buffer
-          // takes tile n+1
-          ok = mbar_wait((bar0 + 8u * (B_STAGED0 + (par ^ 1))), ((n - 1) >> 1) & 1, abort);
-          if (!ok) break;
-          const uint32_t vnext = sbase + OFF_V0 + (par ^ 1) * TILE_BYTES;
-          tma_store(&mo, 0, y0 + (n - 1) * TILE, bh, vnext);    // rows past the end of the sequence are clipped
-          tma_store(&mo, 64, y0 + (n - 1) * TILE, bh, vnext + BOX_BYTES);
-          tma_commit();
-          if (n + 1 < nchunks) {
-            tma_wait_read();
-            mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + (par ^ 1))), TILE_BYTES);
-            tma_load(vnext, &mv, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + (par ^ 1))));
-            tma_load(vnext + BOX_BYTES, &mv, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + (par ^ 1))));
-          }
+          tma_load(kbuf + KBOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
         }
         // P of the next tile overwrites the columns that the last product of this tile reads
         ok = mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
       }
-      if (ok) {   // the outputs of the last tile
-        const int n = nchunks - 1;
-        ok = mbar_wait((bar0 + 8u * (B_STAGED0 + (n & 1))), (n >> 1) & 1, abort);
-        if (ok) {
-          const uint32_t src = sbase + OFF_V0 + (n & 1) * TILE_BYTES;
-          tma_store(&mo, 0, y0 + n * TILE, bh, src);
-          tma_store(&mo, 64, y0 + n * TILE, bh, src + BOX_BYTES);
-          tma_commit();
+    }
+  } else if (warp == kCopyWarp) {
+    // =============================== the first K loads, the V loads, output stores (one lane) ===============================
+    // A lane of its own, so that waiting for a store to have read its buffer never holds up the issue of products.
+    if (lane == 0) {
+      bool ok = true;
+      for (int n = 0; n < 2 && n < nchunks; ++n) {
+        const uint32_t kb = sbase + (n ? OFF_K1 : OFF_K0), kbar = bar0 + 8u * (n ? B_FULL_K1 : B_FULL_K0);
+        mbar_expect_tx(kbar, TILE_BYTES);
+        tma_load(kb, &mk, 0, y0 + n * TILE, bh, kbar);
+        tma_load(kb + KBOX_BYTES, &mk, 64, y0 + n * TILE, bh, kbar);
+      }
+      for (int n = 0; n < 2 && n < nchunks; ++n) {
+        mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + n)), TILE_BYTES);
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
+      }
+      for (int n = 0; n < nchunks; ++n) {
+        const uint32_t par = n & 1;
+        // the outputs of tile n are staged in its V buffer: store them; once they have been read the buffer takes
+        // tile n+2
+        ok = mbar_wait((bar0 + 8u * (B_STAGED0 + par)), (n >> 1) & 1, abort);
+        if (!ok) break;
+        const uint32_t vb = sbase + OFF_V0 + par * TILE_BYTES;
+        tma_store(&mo, 0, y0 + n * TILE, bh, vb);               // rows past the end of the sequence are clipped
+        tma_store(&mo, 64, y0 + n * TILE, bh, vb + BOX_BYTES);
+        tma_commit();
+        if (n + 2 < nchunks) {
+          tma_wait_read();
+          mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + par)), TILE_BYTES);
+          tma_load(vb, &mv, 0, y0 + (n + 2) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + par)));
+          tma_load(vb + BOX_BYTES, &mv, 64, y0 + (n + 2) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + par)));
         }
       }
       tma_wait_all();                             // every store is complete before the CTA exits
@@ -513,12 +516,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       if (!go) return;
       const int valid = min(TILE, T - m * TILE);
       const int ct = ta & 15, rg = ta >> 4;                     // chunk column 0..15, row group 0..15
-      unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * BOX_BYTES;
+      unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * KBOX_BYTES;
+      uint4 x[8];                                               // all eight loads first: they do not wait for the stores
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = *reinterpret_cast<const uint4*>(Kb + swz(rg + 16 * i, ct & 7));
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int j = rg + 16 * i;
-        uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-        *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(Kb + swz(j, ct & 7)) = j < valid ? phi8<PHI>(x[i]) : make_uint4(0u, 0u, 0u, 0u);
       }
     };
     ok = mbar_wait((bar0 + 8u * (B_FULL_K0)), 0, abort);
@@ -577,6 +582,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
           LA_TMEM_ST16(tmem + P_COL + lane_addr + 64 * hf + 16 * qq, pk);
         }
+        if (hf == 1) {                            // phi(q) . z_prev, delivered by the score product as column 128
+          dpart += __uint_as_float(tmem_ld1(tmem + lane_addr + QZ_COL));
+          tmem_wait_ld();
+        }
         // (slot n & 1 was last read by the epilogue of tile n-2, before the arrival that released the accumulator to
         // tile n-1, whose products were complete before P of this tile was issued)
         denbuf[(par * 2 + hf) * D + r] = dpart;
@@ -598,6 +607,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         tc_fence_after();
+        uint32_t zbits = 0u;
+        if (hf == 0) zbits = tmem_ld1(tmem + lane_addr + Z_COL);
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
           uint32_t v[32];
@@ -615,10 +626,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           }
         }
         if (hf == 0) {
-          const float zz = __uint_as_float(tmem_ld1(tmem + lane_addr + Z_COL));
-          tmem_wait_ld();
+          const float zz = __uint_as_float(zbits);
           if (last) z[(size_t)u * D + r] = zz;
-          else *reinterpret_cast<__nv_bfloat16*>(smem + OFF_SZ + ext_offset(r, 0)) = __float2bfloat16_rn(zz);
+          else                                    // row 128 of the K buffer of tile n+1 (its token rows are in place already)
+            *reinterpret_cast<__nv_bfloat16*>(smem + (((n + 1) & 1) ? OFF_K1 : OFF_K0) + (r >> 6) * KBOX_BYTES + BOX_BYTES +
+                                              (r & 63) * 2) = __float2bfloat16_rn(zz);
         }
       }
       fence_proxy_async();
@@ -642,16 +654,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && (tid & 127) < 64 && !gh) {
-        // next halo <- last W-1 rows of (halo ++ valid rows of V); each half of the group copies its own channels
+      if (ok && !gh) {
+        // next halo <- last W-1 rows of (halo ++ valid rows of V), 16 bytes (8 channels) per thread; each half of the
+        // group copies its own 64 channels
         const unsigned char* Vc = Vt + hf * BOX_BYTES;
-        const int cw = tid & 63, ch = 64 * hf + cw;
-        for (int i = 0; i < W - 1; ++i) {
-          const int src = valid + i;
-          __nv_bfloat16 x;
-          if (src < W - 1) x = halo[src * D + ch];
-          else x = *reinterpret_cast<const __nv_bfloat16*>(Vc + swz(src - (W - 1), cw >> 3) + (cw & 7) * 2);
-          halo_next[i * D + ch] = x;
+        for (int idx = tid & 127; idx < 8 * (W - 1); idx += 128) {
+          const int i = idx >> 3, c8 = idx & 7, src = valid + i;
+          uint4 x;
+          if (src < W - 1) x = *reinterpret_cast<const uint4*>(halo + src * D + 64 * hf + 8 * c8);
+          else x = *reinterpret_cast<const uint4*>(Vc + swz(src - (W - 1), c8));
+          *reinterpret_cast<uint4*>(halo_next + i * D + 64 * hf + 8 * c8) = x;
         }
       }
       ok = ok && mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);   // also: every product that reads V is done
@@ -660,25 +672,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       // swizzled layout) once every thread of this half has taken its taps from it, so that a thread holds one
       // column of outputs at a time; the control lane then stores whole rows with one TMA store per box.  The two
       // halves of the group (64 channels each) share nothing and synchronise separately.
+      // The accumulator is read 32 columns at a time; each load is issued as early as its registers are free, so
+      // that its latency passes behind the barrier and the arithmetic in between.
+      uint32_t v[32];
+      if (ok) {
+        tc_fence_after();
+        LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf, v);
+      }
       sync_half_b(hf);                            // the next halo is complete before any row of V is overwritten
       float rden = 0.f;
       if (ok) {
-        tc_fence_after();
-        float den = denbuf[(par * 2) * D + r] + denbuf[(par * 2 + 1) * D + r];   // row sum of the masked P
-        if (init || n > 0) {                      // + phi(q) . z_prev, formed beside O on the tensor cores
-          den += __uint_as_float(tmem_ld1(tmem + lane_addr + DEN_COL));
-          tmem_wait_ld();
-        }
+        // row sum of the masked P + phi(q) . z_prev, both halves gathered by the masking threads
+        const float den = denbuf[(par * 2) * D + r] + denbuf[(par * 2 + 1) * D + r];
         rden = 1.f / (den + eps);
       }
       unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
 #pragma unroll
       for (int qq = 0; qq < 2; ++qq) {
-        uint32_t v[32];
-        if (ok) {
-          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32 * qq, v);
-          tmem_wait_ld();
-        }
+        if (ok) tmem_wait_ld();
         if (qq == 1) {
           tc_fence_before();
           mbar_arrive((bar0 + 8u * (B_EPI0 + par)));         // this accumulator has been read
@@ -703,6 +714,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                                    pack2(acc[3].x, acc[3].y));
             }
           }
+          if (qq == 0 && c2 == 1 && ok)           // the first 32 columns have been used: fetch the other 32
+            LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32, v);
           sync_half_b(hf);                        // these two columns of this half have been read by all of its rows
           if (ok) {
 #pragma unroll
@@ -826,11 +839,13 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
       if (ok) {
         const int ct = tid & 15, rg = tid >> 4;
         unsigned char* Kb = smem + ST_OFF_K + (n & 1) * TILE_BYTES + (ct >> 3) * BOX_BYTES;
+        uint4 x[8];                                             // all eight loads first: they do not wait for the stores
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = *reinterpret_cast<const uint4*>(Kb + swz(rg + 16 * i, ct & 7));
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int j = rg + 16 * i;
-          uint4* p = reinterpret_cast<uint4*>(Kb + swz(j, ct & 7));
-          *p = j < valid ? phi8<PHI>(*p) : make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(Kb + swz(j, ct & 7)) = j < valid ? phi8<PHI>(x[i]) : make_uint4(0u, 0u, 0u, 0u);
         }
       }
       fence_proxy_async();
