@@ -24,6 +24,9 @@ Sec. 4.1/4.2):
 * Grouped processing (Sec. 4.1): the sequence is cut into non-overlapping
   groups, groups are processed in parallel inside, and only the group-level
   cumulative sums of phi(K)^T V are carried between groups ("chunked" below).
+* The three-branch block of Sec. 4.1 (`prefill_grouped_block`): between groups only the group-level sums
+  (no linear-attention term inside a group), inside a group causal softmax attention, plus the
+  convolution; alpha weighs the global term.
 * Speculative verification (Sec. 4.2 "Proposed Solution" and Sec. 5.3
   "Comparison with Direct Integration"): every node of a draft-token tree sees
   the committed prefix (one shared state) plus its own ancestors, and the
@@ -200,6 +203,61 @@ def prefill_chunked(q, k, v, w, kind: str, eps: float, chunk: int, state: State 
         o[:, :, lo:hi] = num / (den + eps)[..., None]
         S = S + np.matmul(np.swapaxes(fk, -1, -2), vc)
         z = z + fk.sum(axis=2)
+    o += causal_dwconv(v, w, st.win)
+    return o, State(S, z, _next_window(st.win, v), st.pos + T)
+
+
+# ---------------------------------------------------------------------------
+# The three-branch block of Sec. 4.1: grouped linear attention between groups, softmax
+# attention inside a group, masked depthwise convolution
+# ---------------------------------------------------------------------------
+
+def prefill_grouped_block(q, k, v, w, kind: str, eps: float, group: int, alpha: float, scale: float,
+                          state: State | None = None):
+    """The augmented block as Sec. 4.1 describes it (Fig. "la_aug", three branches), token by token.
+
+    The sequence is cut into non-overlapping groups of `group` tokens, counted from the first token of the
+    sequence.  For token i in group g:
+
+      middle branch  glob_i = phi(q_i)^T S_{<g} / (phi(q_i) . z_{<g} + eps): linear attention against the
+                     group-level cumulative sums of the groups before g only ("within each group we bypass local
+                     dependencies"); defined as 0 where that denominator is 0 (no earlier group and eps = 0);
+      left branch    loc_i = sum_{j in g, j <= i} softmax_j(scale q_i . k_j) v_j: causal softmax attention inside
+                     the group, on the raw q and k;
+      right branch   conv_i: the masked depthwise convolution of v;
+      o_i = alpha * glob_i + loc_i + conv_i   (alpha balances the global against the local term).
+
+    Readings where the paper is silent: the softmax scale is an argument (1/sqrt(d) is the usual choice), alpha
+    multiplies the global branch only, groups are aligned to the start of the sequence.  With a carried `state` the
+    tokens absorbed so far must end at a group boundary (state.pos a multiple of `group`); the returned state holds
+    S, z over all tokens, the convolution window and pos, as the other forms do.
+    Returns (o [B,H,T,d], new State).
+    """
+    q, k, v, w = _f64(q, k, v, w)
+    B, H, T, d = q.shape
+    W = w.shape[2]
+    st = empty_state(B, H, d, W) if state is None else state
+    if np.any(st.pos % group != 0):
+        raise ValueError("the carried state does not end at a group boundary")
+    fq, fk = phi(q, kind), phi(k, kind)
+    S, z = st.S.copy(), st.z.copy()
+    o = np.zeros_like(v)
+    for lo in range(0, T, group):
+        hi = min(lo + group, T)
+        for i in range(lo, hi):
+            # middle branch: the groups before this one
+            num = np.einsum("bha,bhac->bhc", fq[:, :, i], S)
+            den = np.einsum("bha,bha->bh", fq[:, :, i], z) + eps
+            glob = np.where(den[..., None] != 0.0, num / np.where(den != 0.0, den, 1.0)[..., None], 0.0)
+            # left branch: softmax over the tokens of this group up to and including i
+            logits = scale * np.einsum("bha,bhja->bhj", q[:, :, i], k[:, :, lo:i + 1])
+            e = np.exp(logits - logits.max(axis=-1, keepdims=True))
+            prob = e / e.sum(axis=-1, keepdims=True)
+            loc = np.einsum("bhj,bhjc->bhc", prob, v[:, :, lo:i + 1])
+            o[:, :, i] = alpha * glob + loc
+        # the group is complete: its sums join the group-level cumulative sums
+        S = S + np.matmul(np.swapaxes(fk[:, :, lo:hi], -1, -2), v[:, :, lo:hi])
+        z = z + fk[:, :, lo:hi].sum(axis=2)
     o += causal_dwconv(v, w, st.win)
     return o, State(S, z, _next_window(st.win, v), st.pos + T)
 
