@@ -126,6 +126,35 @@ la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const voi
                      const float* conv_w, int32_t init_state, la_state* st /*host struct*/, void* o,
                      void* stream);
 
+/* Prefill of the three-branch block: Sec. 4.1 "LA Augmentation for Autoregressive LLMs" as the paper describes it
+ * (Fig. "la_aug"), where la_prefill computes the exact masked linear attention inside a group instead.  The
+ * sequence is cut into non-overlapping groups of `group` tokens, counted from the first token of the sequence.
+ * For token i of group g:
+ *   middle branch   glob_i = phi(q_i)^T S_{<g} / (phi(q_i) . z_{<g} + eps): linear attention against the group-level
+ *                   cumulative sums of the groups before g only (inside a group the local dependencies are bypassed);
+ *                   0 where that denominator is 0 (no earlier group and eps = 0);
+ *   left branch     loc_i = sum over j in g, j <= i of softmax_j(softmax_scale * q_i . k_j) v_j: causal softmax
+ *                   attention inside the group, on the raw q and k;
+ *   right branch    the masked depthwise convolution of v, as in la_prefill;
+ *   o_i = alpha * glob_i + loc_i + conv_i     (alpha: the paper's hyper-parameter that balances global against local).
+ *
+ *   group          1 .. la_prefill_grouped_max_group(ctx) (what the kernel's shared memory holds: 128 for bf16 io
+ *                  with d = 128, 256 for bf16 with d = 64, 128 / 64 for fp32 with d = 64 / 128); larger groups
+ *                  return LA_ERR_UNSUPPORTED
+ *   softmax_scale  multiplies q . k before the softmax (1 / sqrt(d) is the usual choice)
+ *   init_state     1: continue from st, whose tokens must end at a group boundary (the library cannot see where
+ *                  earlier groups ended and does not check)
+ *   st             in-out as for la_prefill: on return S and z hold the sums over all tokens, the window the last
+ *                  W-1 values of v, pos the token count
+ *   other arguments as for la_prefill.
+ *
+ * This entry point runs on the CUDA cores in fp32 (a register-tiled kernel, one thread block per (batch, head)); it
+ * is several times slower per token than the tensor-core la_prefill. */
+la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
+                             const float* conv_w, int32_t group, float alpha, float softmax_scale, int32_t init_state,
+                             la_state* st /*host struct*/, void* o, void* stream);
+int32_t la_prefill_grouped_max_group(const la_ctx* ctx);
+
 /* Decode: one token per sequence.  The cumulative sum of Sec. 4.1 (query t meets
  * sum_{i<=t} K_i V_i) as a recurrence: S += phi(k) v^T, z += phi(k), then
  * o = phi(q)^T S / (phi(q).z + eps) + conv, with the convolution reading the carried

@@ -25,7 +25,7 @@ LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
            "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy", "la_selftest_wait_timeout",
-           "la_prefill_workspace_bytes"]
+           "la_prefill_workspace_bytes", "la_prefill_grouped", "la_prefill_grouped_max_group"]
 
 
 class LaError(RuntimeError):
@@ -58,6 +58,10 @@ def lib() -> C.CDLL:
         L.la_status_str.argtypes = [C.c_int]
         L.la_status_str.restype = C.c_char_p
         L.la_prefill.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, C.POINTER(la_state), vp, vp]
+        L.la_prefill_grouped.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, C.c_float, C.c_float, i32, C.POINTER(la_state),
+                                         vp, vp]
+        L.la_prefill_grouped_max_group.argtypes = [vp]
+        L.la_prefill_grouped_max_group.restype = i32
         L.la_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
@@ -74,7 +78,7 @@ def lib() -> C.CDLL:
         L.la_prefill_workspace_bytes.restype = C.c_uint64
         L.la_launch_count.restype = C.c_int64
         for name in EXPORTS:
-            if name not in ("la_status_str", "la_launch_count", "la_prefill_workspace_bytes"):
+            if name not in ("la_status_str", "la_launch_count", "la_prefill_workspace_bytes", "la_prefill_grouped_max_group"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -174,6 +178,22 @@ class Context:
             _ptr(conv_w, torch.float32, (self.H, self.d, self.W), "conv_w"), int(bool(init_state)), C.byref(cs),
             _ptr(out, self.dtype, shp, "o"), _stream(stream)))
         return out
+
+    def la_prefill_grouped(self, q, k, v, conv_w, state: State, group: int, alpha: float, softmax_scale: float,
+                           init_state: bool = False, out=None, stream=None):
+        B, H, T, d = q.shape
+        shp = (B, self.H, T, self.d)
+        out = torch.empty(shp, dtype=self.dtype, device=q.device) if out is None else out
+        self._check_state(state, B)
+        cs = state.c()
+        _check("la_prefill_grouped", lib().la_prefill_grouped(
+            self._h, B, T, _ptr(q, self.dtype, shp, "q"), _ptr(k, self.dtype, shp, "k"), _ptr(v, self.dtype, shp, "v"),
+            _ptr(conv_w, torch.float32, (self.H, self.d, self.W), "conv_w"), int(group), float(alpha),
+            float(softmax_scale), int(bool(init_state)), C.byref(cs), _ptr(out, self.dtype, shp, "o"), _stream(stream)))
+        return out
+
+    def la_prefill_grouped_max_group(self) -> int:
+        return int(lib().la_prefill_grouped_max_group(self._h))
 
     def la_decode_step(self, q, k, v, conv_w, state: State, out=None, stream=None):
         B = q.shape[0]

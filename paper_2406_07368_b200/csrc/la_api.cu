@@ -126,6 +126,21 @@ la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const voi
                                                                                                    : LA_ERR_CUDA;
 }
 
+la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
+                             const float* conv_w, int32_t group, float alpha, float softmax_scale, int32_t init_state,
+                             la_state* st, void* o, void* stream) {
+  if (!ctx || B < 1 || T < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o)) return LA_ERR_INVALID_ARG;
+  if (!state_ok(ctx, st) || (init_state != 0 && init_state != 1) || group < 1) return LA_ERR_INVALID_ARG;
+  if (!std::isfinite(alpha) || !std::isfinite(softmax_scale)) return LA_ERR_INVALID_ARG;
+  if (group > la::prefill_grouped_max_group(ctx->cfg)) return LA_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return cuda_status(la::launch_prefill_grouped(ctx, B, T, q, k, v, conv_w, group, alpha, softmax_scale, init_state, *st, o,
+                                                static_cast<cudaStream_t>(stream)));
+}
+
+int32_t la_prefill_grouped_max_group(const la_ctx* ctx) { return ctx ? la::prefill_grouped_max_group(ctx->cfg) : 0; }
+
 la_status la_decode_step(la_ctx* ctx, int32_t B, const void* q, const void* k, const void* v, const float* conv_w,
                          la_state* st, void* o, void* stream) {
   if (!ctx || B < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o)) return LA_ERR_INVALID_ARG;

@@ -143,6 +143,11 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
 cudaError_t launch_accept(la_ctx* ctx, int B, int N, const int32_t* parent, const int32_t* draft, const int32_t* pred_root,
                           const int32_t* pred, int32_t* accept_node, int32_t* accept_len, int32_t* next_token,
                           cudaStream_t s);
+// The three-branch block (group-exclusive linear attention, softmax inside a group, convolution) on the CUDA cores.
+cudaError_t launch_prefill_grouped(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
+                                   int group, float alpha, float scale, int init_state, const la_state& st, void* o,
+                                   cudaStream_t s);
+int prefill_grouped_max_group(const la_config& c);   // largest group size the kernel's shared memory holds
 // Workspace la_prefill can use for a launch of B sequences of T tokens (0: none needed).
 size_t prefill_workspace_bytes(const la_ctx* ctx, int B, int T);
 }  // namespace la
