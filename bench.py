@@ -77,8 +77,10 @@ def measured_peaks():
     if os.path.exists(path):
         p = json.load(open(path))
         return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
-                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
 
 
 class ClockSampler:
@@ -403,10 +405,52 @@ def promptgen_workload(W: wl.Workload, rank: int, device):
     return step, e2e_step, info
 
 
-FACTORIES = {"llama7b_prefill": prefill_workload, "long_prefill": prefill_workload,
+def grouped_workload(W: wl.Workload, rank: int, device):
+    """The three-branch block (la_prefill_grouped) on the prefill shape: fp32 arithmetic on the CUDA cores."""
+    from paper_2406_07368_b200 import binding
+    io = W.io
+    q, k, v = W.prefill_inputs()
+    if rank:
+        q, k, v = wl.qkv(W.seed + 1000 * rank, q.shape, W.scale, io)
+    w = dev(W.weights(), "f32", device)
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, io, chunk=W.chunk)
+    per_set = 4 * q.size * 2
+    nsets = max(2, -(-2 * L2_BYTES // per_set) + 1)
+    base = [dev(x, io, device) for x in (q, k, v)]
+    sets = [[x.roll(i, dims=0).contiguous() if i else x for x in base] for i in range(nsets)]
+    outs = [torch.empty_like(base[0]) for _ in range(nsets)]
+    st = ctx.new_state(W.B)
+    alpha, sscale = W.extra["alpha"], W.extra["softmax_scale"]
+    counter = [0]
+
+    def step():
+        i = counter[0] % nsets
+        counter[0] += 1
+        ctx.la_prefill_grouped(sets[i][0], sets[i][1], sets[i][2], w, st, W.chunk, alpha, sscale, out=outs[i])
+
+    pinned = [torch.from_numpy(x).to(binding.TORCH_DTYPE[io]).pin_memory() for x in (q, k, v)]
+    o_host = torch.empty(q.shape, dtype=binding.TORCH_DTYPE[io]).pin_memory()
+
+    def e2e_step():                                  # host inputs in, one call, host outputs back
+        for dst, src in zip(sets[0], pinned):
+            dst.copy_(src, non_blocking=True)
+        ctx.la_prefill_grouped(sets[0][0], sets[0][1], sets[0][2], w, st, W.chunk, alpha, sscale, out=outs[0])
+        o_host.copy_(outs[0], non_blocking=True)
+
+    units = W.B * W.H * W.T
+    flops = units * (4 * W.d * W.d + 2 * W.d * (W.chunk + 1) + 2 * W.d * W.W)   # readout + state update, scores + PV, taps
+    info = {"ctx": ctx, "tokens_per_step": W.B * W.T, "alg_bytes_per_launch": units * 4 * W.d * 2, "launches_per_step": 1,
+            "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill_grouped (fp32 CUDA cores)",
+            "flops_per_launch": flops, "bound": "alu", "period": nsets,
+            "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
+    return step, e2e_step, info
+
+
+FACTORIES = {"llama7b_prefill": prefill_workload, "grouped_block": grouped_workload, "long_prefill": prefill_workload,
              "batched_decode": decode_workload, "tree_verify": verify_workload, "prompt_gen": promptgen_workload}
 METRICS = {"llama7b_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "long_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
+           "grouped_block": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "batched_decode": ("decode_tokens_per_s_per_layer", "tokens/s"),
            "tree_verify": ("verify_nodes_per_s_per_layer", "nodes/s"),
            "prompt_gen": ("prompt_and_generation_tokens_per_s_per_layer", "tokens/s")}
@@ -427,6 +471,12 @@ def oracle_samples(W: wl.Workload):
                             f"grouped form (groups of {W.chunk}), 1 of {W.B} sequences, all {W.H} heads, all {T} tokens"),
                 "definition": (lambda: orc.prefill_quadratic(q[:, :, :Tq], k[:, :, :Tq], v[:, :, :Tq], w, W.phi, W.eps), Tq,
                                f"quadratic definition, 1 of {W.B} sequences, all {W.H} heads, first {Tq} of {W.T} tokens")}
+    if W.name == "grouped_block":
+        q, k, v = W.prefill_inputs(B=1, H=4)
+        w = W.weights()[:4]
+        return {"primary": (lambda: orc.prefill_grouped_block(q, k, v, w, W.phi, W.eps, W.chunk, W.extra["alpha"],
+                                                              W.extra["softmax_scale"]), W.T * 4 / W.H,
+                            f"token-by-token form, 1 of {W.B} sequences, 4 of {W.H} heads, all {W.T} tokens")}
     if W.name == "prompt_gen":
         P, G = min(W.extra["shapes"], key=lambda pg: pg[0] + pg[1])
         q, k, v = wl.qkv(W.seed, (W.B, W.H, P + G, W.d), W.scale, W.io)
@@ -486,7 +536,7 @@ def time_fn(fn, units, repeats: int, warmup: int = 0):
 
 def l2_note(W: wl.Workload) -> str:
     """How the GPU arm keeps the 126 MB L2 from serving a step's inputs (a property of the workload's sizes)."""
-    if W.name in ("llama7b_prefill", "long_prefill"):
+    if W.name in ("llama7b_prefill", "long_prefill", "grouped_block"):
         per_set = 4 * W.B * W.H * W.T * W.d * 2
         nsets = max(2, -(-2 * L2_BYTES // per_set) + 1) if per_set < 4 * L2_BYTES else 1
         return f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"
@@ -707,6 +757,12 @@ def roofline_of(res, peaks):
          "peak_source": peaks["source"], "alg_bytes_per_launch": info["alg_bytes_per_launch"], "launch_ms": kernel_ms,
          "tensor_tflops": tflops, "tensor_frac_of_sustained": tflops / peaks["bf16_tflops_sustained"],
          "frac_of_nominal_7700": achieved / NOMINAL_HBM_GBS}
+    if info.get("bound") == "alu":
+        # fp32 multiply-adds on the CUDA cores: 148 SMs x 128 lanes x 2 flop at the maximum SM clock
+        peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        r.update({"bound": "alu", "achieved": tflops, "peak": peak, "unit": "TFLOP/s", "frac": tflops / peak,
+                  "peak_source": "derived: 148 SMs x 128 fp32 lanes x 2 flop x max SM clock",
+                  "hbm_gbs_algorithmic": achieved, "hbm_frac_algorithmic": achieved / peaks["hbm_gbs"]})
     if r["traffic"] is not None:                 # the same fraction from the DRAM bytes ncu counted, not the algorithmic ones
         r["achieved_from_traffic"] = r["traffic"] / (kernel_ms * 1e-3) / 1e9
         r["frac_from_traffic"] = r["achieved_from_traffic"] / peaks["hbm_gbs"]
@@ -745,9 +801,9 @@ def brief(res, peaks, clocks):
     return out
 
 
-OTHERS = {"llama7b_prefill": ("batched_decode", "tree_verify", "long_prefill")}
-DEFAULT_STEPS = {"llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
-OTHER_STEPS = {"long_prefill": 20, "batched_decode": 400, "tree_verify": 400}
+OTHERS = {"llama7b_prefill": ("batched_decode", "tree_verify", "long_prefill", "grouped_block")}
+DEFAULT_STEPS = {"grouped_block": 10, "llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
+OTHER_STEPS = {"long_prefill": 20, "batched_decode": 400, "tree_verify": 400, "grouped_block": 6}
 
 
 def main():
@@ -812,7 +868,7 @@ def main():
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         samples = oracle_samples(W)
-        reps = {"llama7b_prefill": 8, "long_prefill": 2, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
+        reps = {"grouped_block": 1, "llama7b_prefill": 8, "long_prefill": 2, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
         fn, units, text = samples["primary"]
         v, per = time_fn(fn, units, reps)
         cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text, "seconds": per * reps}

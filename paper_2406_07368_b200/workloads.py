@@ -254,4 +254,12 @@ def prompt_gen() -> Workload:
                     extra={"shapes": [(340, 160), (60, 20), (7000, 200), (1700, 400)]})
 
 
-WORKLOADS = {w().name: w for w in (tiny_fp32, llama7b_prefill, batched_decode, tree_verify, long_prefill, prompt_gen)}
+def grouped_block() -> Workload:
+    """The three-branch block on the LLaMA-2-7B-shaped prefill: B=4, H=32, d=128, T=2048 bf16, groups of 64 (the
+    paper's group size for LLaMA), softmax scale 1/sqrt(d), alpha 1, elu+1, 3 taps; inputs N(0,1)/sqrt(d)."""
+    return Workload("grouped_block", "bf16", 4, 32, 128, 2048, 3, 64, "elu1", 0.0, 6, 128 ** -0.5,
+                    extra={"alpha": 1.0, "softmax_scale": 128 ** -0.5})
+
+
+WORKLOADS = {w().name: w for w in (tiny_fp32, llama7b_prefill, batched_decode, tree_verify, long_prefill, prompt_gen,
+                                   grouped_block)}
