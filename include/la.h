@@ -155,6 +155,25 @@ la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, c
                              la_state* st /*host struct*/, void* o, void* stream);
 int32_t la_prefill_grouped_max_group(const la_ctx* ctx);
 
+/* A prefill cut along the sequence, for several GPUs that each hold one stretch of a long sequence.  Sec. 4.1:
+ * between groups only the cumulative sums of phi(k) v^T and of phi(k) are carried, so a stretch needs from all the
+ * tokens before it just those sums and the last W-1 values of v.
+ *
+ * la_segment_state computes the sums of one stretch on their own: dS[a][c] = sum_j phi(k_j)[a] v_j[c],
+ * dz[a] = sum_j phi(k_j)[a] over the T tokens given (K and V are read, Q is not needed).
+ *   k, v   [B, H, T, d] io type;  dS [B, H, d, d] fp32 out;  dz [B, H, d] fp32 out
+ *
+ * la_state_prefix adds up parts: S_out = S_base + sum of the first `count` of the `nparts` parts in dS_parts
+ * ([nparts, B, H, d, d], e.g. the all-gathered dS of all ranks, with count = this rank's index), likewise z.
+ * S_base / z_base may both be NULL (an empty starting state).  la_prefill(init_state = 1) then continues from
+ * (S_out, z_out, the last W-1 values of v before the stretch, the number of tokens before it).  S_out may not
+ * overlap the parts. */
+la_status la_segment_state(la_ctx* ctx, int32_t B, int32_t T, const void* k, const void* v, float* dS, float* dz,
+                           void* stream);
+la_status la_state_prefix(la_ctx* ctx, int32_t B, int32_t nparts, int32_t count, const float* dS_parts,
+                          const float* dz_parts, const float* S_base, const float* z_base, float* S_out, float* z_out,
+                          void* stream);
+
 /* Decode: one token per sequence.  The cumulative sum of Sec. 4.1 (query t meets
  * sum_{i<=t} K_i V_i) as a recurrence: S += phi(k) v^T, z += phi(k), then
  * o = phi(q)^T S / (phi(q).z + eps) + conv, with the convolution reading the carried

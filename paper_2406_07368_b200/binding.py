@@ -25,7 +25,8 @@ LA_MAX_TAPS, LA_MAX_NODES, LA_NOALLOC_MAX_SEQ = 32, 64, 1024
 EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_step", "la_verify_tree",
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
            "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy", "la_selftest_wait_timeout",
-           "la_prefill_workspace_bytes", "la_prefill_grouped", "la_prefill_grouped_max_group"]
+           "la_prefill_workspace_bytes", "la_prefill_grouped", "la_prefill_grouped_max_group",
+           "la_segment_state", "la_state_prefix"]
 
 
 class LaError(RuntimeError):
@@ -62,6 +63,8 @@ def lib() -> C.CDLL:
                                          vp, vp]
         L.la_prefill_grouped_max_group.argtypes = [vp]
         L.la_prefill_grouped_max_group.restype = i32
+        L.la_segment_state.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+        L.la_state_prefix.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.la_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
@@ -194,6 +197,30 @@ class Context:
 
     def la_prefill_grouped_max_group(self) -> int:
         return int(lib().la_prefill_grouped_max_group(self._h))
+
+    def la_segment_state(self, k, v, dS=None, dz=None, stream=None):
+        """Sums of one stretch of the sequence: (dS [B,H,d,d], dz [B,H,d]) fp32."""
+        B, H, T, d = k.shape
+        shp = (B, self.H, T, self.d)
+        dS = torch.empty(B, self.H, self.d, self.d, dtype=torch.float32, device=k.device) if dS is None else dS
+        dz = torch.empty(B, self.H, self.d, dtype=torch.float32, device=k.device) if dz is None else dz
+        _check("la_segment_state", lib().la_segment_state(
+            self._h, B, T, _ptr(k, self.dtype, shp, "k"), _ptr(v, self.dtype, shp, "v"),
+            _ptr(dS, torch.float32, (B, self.H, self.d, self.d), "dS"), _ptr(dz, torch.float32, (B, self.H, self.d), "dz"),
+            _stream(stream)))
+        return dS, dz
+
+    def la_state_prefix(self, dS_parts, dz_parts, count: int, S_base=None, z_base=None, stream=None):
+        """S_base + the first `count` parts of dS_parts [nparts,B,H,d,d] (likewise z): returns (S, z)."""
+        nparts, B = dS_parts.shape[0], dS_parts.shape[1]
+        S = torch.empty(dS_parts.shape[1:], dtype=torch.float32, device=dS_parts.device)
+        z = torch.empty(dz_parts.shape[1:], dtype=torch.float32, device=dz_parts.device)
+        _check("la_state_prefix", lib().la_state_prefix(
+            self._h, B, nparts, int(count), _ptr(dS_parts, torch.float32, (nparts, B, self.H, self.d, self.d), "dS_parts"),
+            _ptr(dz_parts, torch.float32, (nparts, B, self.H, self.d), "dz_parts"),
+            _ptr(S_base, torch.float32, (B, self.H, self.d, self.d), "S_base"),
+            _ptr(z_base, torch.float32, (B, self.H, self.d), "z_base"), S.data_ptr(), z.data_ptr(), _stream(stream)))
+        return S, z
 
     def la_decode_step(self, q, k, v, conv_w, state: State, out=None, stream=None):
         B = q.shape[0]

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libla_b200.so")
-SOURCES = ["la_api.cu", "decode.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_grouped.cu", "verify.cu", "verify_tc.cu", "commit.cu", "accept.cu", "selftest.cu"]
+SOURCES = ["la_api.cu", "decode.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_grouped.cu", "seqpar.cu", "verify.cu", "verify_tc.cu", "commit.cu", "accept.cu", "selftest.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -141,6 +141,28 @@ la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, c
 
 int32_t la_prefill_grouped_max_group(const la_ctx* ctx) { return ctx ? la::prefill_grouped_max_group(ctx->cfg) : 0; }
 
+la_status la_segment_state(la_ctx* ctx, int32_t B, int32_t T, const void* k, const void* v, float* dS, float* dz,
+                           void* stream) {
+  if (!ctx || B < 1 || T < 1 || !good(k) || !good(v) || !good(dS) || !good(dz)) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return cuda_status(la::launch_segment_state(ctx, B, T, k, v, dS, dz, static_cast<cudaStream_t>(stream)));
+}
+
+la_status la_state_prefix(la_ctx* ctx, int32_t B, int32_t nparts, int32_t count, const float* dS_parts,
+                          const float* dz_parts, const float* S_base, const float* z_base, float* S_out, float* z_out,
+                          void* stream) {
+  if (!ctx || B < 1 || nparts < 1 || count < 0 || count > nparts || !good(dS_parts) || !good(dz_parts) || !good(S_out) ||
+      !good(z_out) || (S_base == nullptr) != (z_base == nullptr) || !aligned16(S_base) || !aligned16(z_base))
+    return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  const size_t nz = (size_t)B * ctx->cfg.H * ctx->cfg.d, nS = nz * ctx->cfg.d;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (la::launch_state_prefix(ctx, dS_parts, S_base, S_out, nS, count, s) != cudaSuccess) return LA_ERR_CUDA;
+  return cuda_status(la::launch_state_prefix(ctx, dz_parts, z_base, z_out, nz, count, s));
+}
+
 la_status la_decode_step(la_ctx* ctx, int32_t B, const void* q, const void* k, const void* v, const float* conv_w,
                          la_state* st, void* o, void* stream) {
   if (!ctx || B < 1 || !good(q) || !good(k) || !good(v) || !good(conv_w) || !good(o)) return LA_ERR_INVALID_ARG;

@@ -148,6 +148,12 @@ cudaError_t launch_prefill_grouped(la_ctx* ctx, int B, int T, const void* q, con
                                    int group, float alpha, float scale, int init_state, const la_state& st, void* o,
                                    cudaStream_t s);
 int prefill_grouped_max_group(const la_config& c);   // largest group size the kernel's shared memory holds
+// Sums of one segment of the sequence (dS = sum phi(k) v^T, dz = sum phi(k)), and sums of such parts.
+cudaError_t launch_segment_state(la_ctx* ctx, int B, int T, const void* k, const void* v, float* dS, float* dz, cudaStream_t s);
+cudaError_t launch_segment_state_tc(la_ctx* ctx, int B, int T, const void* k, const void* v, float* dS, float* dz,
+                                    cudaStream_t s, bool* handled);
+cudaError_t launch_state_prefix(la_ctx* ctx, const float* parts, const float* base, float* out, size_t n, int count,
+                                cudaStream_t s);
 // Workspace la_prefill can use for a launch of B sequences of T tokens (0: none needed).
 size_t prefill_workspace_bytes(const la_ctx* ctx, int B, int T);
 }  // namespace la

@@ -1076,4 +1076,23 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   return e;
 }
 
+// The sums of one segment on the tensor cores (bf16 io, d = 128): the kernel of the sequence split with one segment
+// per (batch, head) chain.
+cudaError_t launch_segment_state_tc(la_ctx* ctx, int B, int T, const void* k, const void* v, float* dS, float* dz,
+                                    cudaStream_t s, bool* handled) {
+  const la_config& c = ctx->cfg;
+  *handled = false;
+  if (c.io_dtype != LA_BF16 || c.d != tc::D) return cudaSuccess;
+  const int BH = B * c.H;
+  CUtensorMap mk, mv;
+  if (!tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T)) return cudaErrorNotSupported;
+  auto skern = c.phi == LA_PHI_ELU1 ? tc::segment_state_kernel<LA_PHI_ELU1> : tc::segment_state_kernel<LA_PHI_RELU>;
+  cudaError_t e = cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kStateSmem);
+  if (e != cudaSuccess) return e;
+  skern<<<dim3(BH), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, dS, dz, ctx->d_status, T, 1, T);
+  ctx->launches += 1;
+  *handled = true;
+  return cudaGetLastError();
+}
+
 }  // namespace la
