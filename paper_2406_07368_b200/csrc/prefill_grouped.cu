@@ -16,7 +16,7 @@
 namespace la {
 namespace grp {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 512;
 
 template <typename T> struct Vec4;           // four consecutive elements of the io type
 template <> struct Vec4<float> {
@@ -36,13 +36,13 @@ template <> struct Vec4<__nv_bfloat16> {
   }
 };
 
-// Rows of a query block: the 256 threads form D/4 column groups (four channels each) times 1024/D row groups.
+// Rows of a query block: the 512 threads form D/4 column groups (four channels each) times 2048/D row groups.
 template <typename T, int D> struct Shape {
   static constexpr int kColGroups = D / 4;
   static constexpr int kRowGroups = kThreads / kColGroups;
   static constexpr int QB = (sizeof(T) == 4 && D == 128) ? 16 : 32;     // rows per query block
   static constexpr int RT = QB / kRowGroups;                            // rows per thread
-  static constexpr int SB = D / 16;                                     // edge of a thread's block of S
+  static constexpr int SBA = D / 32, SBC = D / 16;                      // a thread's block of S: SBA rows x SBC columns
   static constexpr int kMaxGroup = (32768 / (D * (int)sizeof(T))) < 256 ? (32768 / (D * (int)sizeof(T))) : 256;
 };
 
@@ -50,9 +50,9 @@ template <typename T, int D> __host__ __device__ inline size_t smem_bytes(int C,
   using Sh = Shape<T, D>;
   size_t b = 0;
   b += (size_t)2 * C * D * sizeof(T);                       // k, phi(k)
-  b += (size_t)(C + W - 1) * D * sizeof(T);                 // W-1 rows before the group, then v
+  b += (size_t)(C + W - 1 + 3) * D * sizeof(T);             // W-1 rows before the group, v, three rows of zeros
   b += (size_t)2 * Sh::QB * D * sizeof(T);                  // q, phi(q) of a block
-  b += (size_t)Sh::QB * (C + 1) * sizeof(float);            // scores of a block, then their row sums
+  b += (size_t)Sh::QB * (((C + 3) & ~3) + 1) * sizeof(float);   // scores of a block (rows padded to four floats), then their row sums
   b += (size_t)D * D * sizeof(float) + D * sizeof(float);   // S, z before the group
   b += (size_t)W * D * sizeof(float);                       // taps
   b += (size_t)Sh::QB * sizeof(float);                      // phi(q) . z
@@ -66,15 +66,16 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
                        int64_t* __restrict__ pos, T* __restrict__ o, int H, int Tlen, int W, int C, float eps,
                        float alpha, float scale, int init) {
   using Sh = Shape<T, D>;
-  constexpr int QB = Sh::QB, RT = Sh::RT, SB = Sh::SB, CG = Sh::kColGroups;
+  constexpr int QB = Sh::QB, RT = Sh::RT, SBA = Sh::SBA, SBC = Sh::SBC, CG = Sh::kColGroups;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   T* ks = reinterpret_cast<T*>(smem_raw);                    // [C][D]
   T* fks = ks + (size_t)C * D;                               // [C][D]   phi(k)
-  T* vs = fks + (size_t)C * D;                               // [W-1 + C][D]
-  T* qs = vs + (size_t)(C + W - 1) * D;                      // [QB][D]
+  T* vs = fks + (size_t)C * D;                               // [W-1 + C + 3][D]: the product with P reads four rows at a time
+  T* qs = vs + (size_t)(C + W - 1 + 3) * D;                  // [QB][D]
   T* fqs = qs + (size_t)QB * D;                              // [QB][D]  phi(q)
-  float* P = reinterpret_cast<float*>(fqs + (size_t)QB * D); // [QB][C]
-  float* rowsum = P + (size_t)QB * C;                        // [QB]
+  const int CP = (C + 3) & ~3;                               // row pitch of P
+  float* P = reinterpret_cast<float*>(fqs + (size_t)QB * D); // [QB][CP]
+  float* rowsum = P + (size_t)QB * CP;                       // [QB]
   float* Ss = rowsum + QB;                                   // [D][D]
   float* zs = Ss + (size_t)D * D;                            // [D]
   float* ws = zs + D;                                        // [W][D]
@@ -83,15 +84,15 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
   const int bh = blockIdx.x, h = bh % H, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t base = (size_t)bh * Tlen * D;
   const int tx = tid % CG, ty = tid / CG;                    // output tile of a block: rows ty*RT.., channels tx*4..
-  const int sa = (tid / 16) * SB, sc = (tid % 16) * SB;      // this thread's block of S
+  const int sa = (tid / 16) * SBA, sc = (tid % 16) * SBC;    // this thread's block of S
 
   // ---- set-up: state, taps, the rows before the sequence ----
-  float sreg[SB][SB];
+  float sreg[SBA][SBC];
   float zreg = 0.f;                                          // z[tid] for tid < D
 #pragma unroll
-  for (int a = 0; a < SB; ++a)
+  for (int a = 0; a < SBA; ++a)
 #pragma unroll
-    for (int c = 0; c < SB; ++c) sreg[a][c] = init ? S[(size_t)bh * D * D + (size_t)(sa + a) * D + sc + c] : 0.f;
+    for (int c = 0; c < SBC; ++c) sreg[a][c] = init ? S[(size_t)bh * D * D + (size_t)(sa + a) * D + sc + c] : 0.f;
   if (tid < D) zreg = init ? z[(size_t)bh * D + tid] : 0.f;
   for (int idx = tid; idx < W * D; idx += kThreads) ws[idx] = w[((size_t)h * D + idx % D) * W + idx / D];
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
@@ -111,10 +112,13 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
       *reinterpret_cast<Vec4<T>*>(vs + (size_t)(W - 1) * D + 4 * idx) =
           *reinterpret_cast<const Vec4<T>*>(v + base + (size_t)g0 * D + 4 * idx);
     }
+    // three rows of zeros behind the group's last value: the product with P reads four rows at a time
+    for (int idx = tid; idx < 3 * D; idx += kThreads) vs[(size_t)(W - 1 + Cg) * D + idx] = from_f32<T>(0.f);
 #pragma unroll
-    for (int a = 0; a < SB; ++a)
+    for (int a = 0; a < SBA; ++a)
 #pragma unroll
-      for (int c = 0; c < SB; ++c) Ss[(sa + a) * D + sc + c] = sreg[a][c];
+      for (int c = 0; c < SBC; c += 4)
+        *reinterpret_cast<float4*>(Ss + (sa + a) * D + sc + c) = make_float4(sreg[a][c], sreg[a][c + 1], sreg[a][c + 2], sreg[a][c + 3]);
     if (tid < D) zs[tid] = zreg;
 
     for (int r0 = 0; r0 < Cg; r0 += QB) {                    // query blocks of the group
@@ -150,7 +154,7 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
           }
         }
 #pragma unroll
-        for (int i = 0; i < RT; ++i) P[(size_t)(ty * RT + i) * C + j] = acc[i] * scale;
+        for (int i = 0; i < RT; ++i) P[(size_t)(ty * RT + i) * CP + j] = acc[i] * scale;
       }
       // phi(q) . z for the rows of the block (one warp per row, rows warp, warp + 8, ...)
       for (int r = warp; r < QB; r += kThreads / 32) {
@@ -165,13 +169,13 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
       // ---- causal softmax along each row (one warp per row); the row keeps exp(s - max), its sum goes aside ----
       for (int r = warp; r < nr; r += kThreads / 32) {
         const int last = r0 + r;                             // the row's own column
-        float* row = P + (size_t)r * C;
+        float* row = P + (size_t)r * CP;
         float m = -INFINITY;
         for (int j = lane; j <= last; j += 32) m = fmaxf(m, row[j]);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
         float sum = 0.f;
-        for (int j = lane; j < jmax; j += 32) {
+        for (int j = lane; j < ((jmax + 3) & ~3); j += 32) {     // (up to the padded end: the product reads four at a time)
           const float e = j <= last ? expf(row[j] - m) : 0.f;
           row[j] = e;
           sum += e;
@@ -189,28 +193,44 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
 #pragma unroll
         for (int c = 0; c < 4; ++c) loc[i][c] = glo[i][c] = 0.f;
       const int jhi = min(jmax, r0 + ty * RT + RT);          // columns this thread's rows can see
-      for (int j = 0; j < jhi; ++j) {                        // loc += P V
-        const float4 vv = reinterpret_cast<const Vec4<T>*>(vs + (size_t)(W - 1 + j) * D + 4 * tx)->f();
+      // loc += P V, four columns of P per step (the rows of P are padded to a multiple of four floats and columns
+      // past a row's own hold zeros, so the last step may run past jhi)
+      for (int j = 0; j < jhi; j += 4) {
+        float4 vv[4], pp[RT];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) vv[jj] = reinterpret_cast<const Vec4<T>*>(vs + (size_t)(W - 1 + j + jj) * D + 4 * tx)->f();
+#pragma unroll
+        for (int i = 0; i < RT; ++i) pp[i] = *reinterpret_cast<const float4*>(P + (size_t)(ty * RT + i) * CP + j);
 #pragma unroll
         for (int i = 0; i < RT; ++i) {
-          const float p = P[(size_t)(ty * RT + i) * C + j];
-          loc[i][0] = fmaf(p, vv.x, loc[i][0]);
-          loc[i][1] = fmaf(p, vv.y, loc[i][1]);
-          loc[i][2] = fmaf(p, vv.z, loc[i][2]);
-          loc[i][3] = fmaf(p, vv.w, loc[i][3]);
+          const float pj[4] = {pp[i].x, pp[i].y, pp[i].z, pp[i].w};
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj) {
+            loc[i][0] = fmaf(pj[jj], vv[jj].x, loc[i][0]);
+            loc[i][1] = fmaf(pj[jj], vv[jj].y, loc[i][1]);
+            loc[i][2] = fmaf(pj[jj], vv[jj].z, loc[i][2]);
+            loc[i][3] = fmaf(pj[jj], vv[jj].w, loc[i][3]);
+          }
         }
       }
       if (have_state) {                                      // glo = phi(Q) S_{<g}
-#pragma unroll 4
-        for (int a = 0; a < D; ++a) {
-          const float4 s4 = *reinterpret_cast<const float4*>(Ss + (size_t)a * D + 4 * tx);
+#pragma unroll 2
+        for (int a = 0; a < D; a += 4) {                     // four features per step
+          float4 s4[4], ff[RT];
+#pragma unroll
+          for (int aa = 0; aa < 4; ++aa) s4[aa] = *reinterpret_cast<const float4*>(Ss + (size_t)(a + aa) * D + 4 * tx);
+#pragma unroll
+          for (int i = 0; i < RT; ++i) ff[i] = reinterpret_cast<const Vec4<T>*>(fqs + (size_t)(ty * RT + i) * D + a)->f();
 #pragma unroll
           for (int i = 0; i < RT; ++i) {
-            const float f = to_f32(fqs[(size_t)(ty * RT + i) * D + a]);
-            glo[i][0] = fmaf(f, s4.x, glo[i][0]);
-            glo[i][1] = fmaf(f, s4.y, glo[i][1]);
-            glo[i][2] = fmaf(f, s4.z, glo[i][2]);
-            glo[i][3] = fmaf(f, s4.w, glo[i][3]);
+            const float fa[4] = {ff[i].x, ff[i].y, ff[i].z, ff[i].w};
+#pragma unroll
+            for (int aa = 0; aa < 4; ++aa) {
+              glo[i][0] = fmaf(fa[aa], s4[aa].x, glo[i][0]);
+              glo[i][1] = fmaf(fa[aa], s4[aa].y, glo[i][1]);
+              glo[i][2] = fmaf(fa[aa], s4[aa].z, glo[i][2]);
+              glo[i][3] = fmaf(fa[aa], s4[aa].w, glo[i][3]);
+            }
           }
         }
       }
@@ -239,18 +259,23 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
 
     // ---- the group is complete: S += phi(K)^T V, z += column sums of phi(K) ----
     for (int j = 0; j < Cg; ++j) {
-      float fa[SB], vc[SB];
+      float fa[SBA], vc[SBC];
+      if (SBA == 4) {
+        const float4 x = reinterpret_cast<const Vec4<T>*>(fks + (size_t)j * D + sa)->f();
+        fa[0] = x.x; fa[1] = x.y; fa[SBA - 2] = x.z; fa[SBA - 1] = x.w;
+      } else {
 #pragma unroll
-      for (int a = 0; a < SB; a += 4) {
-        const float4 x = reinterpret_cast<const Vec4<T>*>(fks + (size_t)j * D + sa + a)->f();
-        fa[a] = x.x; fa[a + 1] = x.y; fa[a + 2] = x.z; fa[a + 3] = x.w;
-        const float4 y = reinterpret_cast<const Vec4<T>*>(vs + (size_t)(W - 1 + j) * D + sc + a)->f();
-        vc[a] = y.x; vc[a + 1] = y.y; vc[a + 2] = y.z; vc[a + 3] = y.w;
+        for (int a = 0; a < SBA; ++a) fa[a] = to_f32(fks[(size_t)j * D + sa + a]);
       }
 #pragma unroll
-      for (int a = 0; a < SB; ++a)
+      for (int c = 0; c < SBC; c += 4) {
+        const float4 y = reinterpret_cast<const Vec4<T>*>(vs + (size_t)(W - 1 + j) * D + sc + c)->f();
+        vc[c] = y.x; vc[c + 1] = y.y; vc[c + 2] = y.z; vc[c + 3] = y.w;
+      }
 #pragma unroll
-        for (int c = 0; c < SB; ++c) sreg[a][c] = fmaf(fa[a], vc[c], sreg[a][c]);
+      for (int a = 0; a < SBA; ++a)
+#pragma unroll
+        for (int c = 0; c < SBC; ++c) sreg[a][c] = fmaf(fa[a], vc[c], sreg[a][c]);
     }
     if (tid < D)
       for (int j = 0; j < Cg; ++j) zreg += to_f32(fks[(size_t)j * D + tid]);
@@ -264,9 +289,9 @@ prefill_grouped_kernel(const T* __restrict__ q, const T* __restrict__ k, const T
 
   // ---- the state after all tokens ----
 #pragma unroll
-  for (int a = 0; a < SB; ++a)
+  for (int a = 0; a < SBA; ++a)
 #pragma unroll
-    for (int c = 0; c < SB; ++c) S[(size_t)bh * D * D + (size_t)(sa + a) * D + sc + c] = sreg[a][c];
+    for (int c = 0; c < SBC; ++c) S[(size_t)bh * D * D + (size_t)(sa + a) * D + sc + c] = sreg[a][c];
   if (tid < D) z[(size_t)bh * D + tid] = zreg;
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads) win[(size_t)bh * (W - 1) * D + idx] = vs[idx];
   if (h == 0 && tid == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + Tlen;
