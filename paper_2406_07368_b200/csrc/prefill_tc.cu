@@ -297,7 +297,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                   const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
                   __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, const __nv_bfloat16* __restrict__ vg,
                   int* status, int H, int Ttot, int W, float eps, int init, int nseg,
-                  int seg_len) {
+                  int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -484,6 +484,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     unsigned char* Qb = smem + OFF_Q + hf * BOX_BYTES;
     unsigned char* Sb = smem + OFF_S + hf * BOX_BYTES;
     float* Sg = S + (size_t)u * D * D + (size_t)r * D + 64 * hf;
+    // Where the state after this unit goes: its own slot, or -- for the last segment of a chain that was cut -- the
+    // caller's state (the pre-pass does not visit last segments: nobody starts from their sums).
+    const bool to_caller = nseg > 1 && (u % nseg) == nseg - 1;
+    float* Sout = to_caller ? S_fin + (size_t)bh * D * D + (size_t)r * D + 64 * hf : Sg;
+    float* zout = to_caller ? z_fin + (size_t)bh * D : z + (size_t)u * D;
     bool ok = true;
 
     if (init) {   // S -> TMEM (fp32) and bf16 copy in shared memory (z was copied during set-up)
@@ -617,7 +622,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           if (last) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<float4*>(Sg + 32 * qq + e) =
+              *reinterpret_cast<float4*>(Sout + 32 * qq + e) =
                   make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
                               __uint_as_float(v[e + 3]));
           } else {
@@ -627,7 +632,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         }
         if (hf == 0) {
           const float zz = __uint_as_float(zbits);
-          if (last) z[(size_t)u * D + r] = zz;
+          if (last) zout[r] = zz;
           else                                    // row 128 of the K buffer of tile n+1 (its token rows are in place already)
             *reinterpret_cast<__nv_bfloat16*>(smem + (((n + 1) & 1) ? OFF_K1 : OFF_K0) + (r >> 6) * KBOX_BYTES + BOX_BYTES +
                                               (r & 63) * 2) = __float2bfloat16_rn(zz);
@@ -767,7 +772,7 @@ template <int PHI>
 __global__ void __launch_bounds__(kStateThreads, 1)
 segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
                      float* __restrict__ S_out, float* __restrict__ z_out, int* status, int Ttot, int nseg,
-                     int seg_len) {
+                     int seg_len, int nrun) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -775,8 +780,10 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ST_OFF_SMALL + 128);
   volatile int* abort = reinterpret_cast<int*>(smem + ST_OFF_SMALL + 132);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int u = blockIdx.x, bh = u / nseg;
-  const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
+  // The launch visits the first nrun of a chain's nseg segments (all of them, or all but the last, whose sums no
+  // other segment starts from); results go to slot bh * nseg + segment.
+  const int bh = blockIdx.x / nrun, sg = blockIdx.x % nrun, u = bh * nseg + sg;
+  const int y0 = sg * seg_len, T = min(seg_len, Ttot - y0);
   const int nchunks = (T + TILE - 1) / TILE;
   const uint32_t bar0 = smem_u32(&bars[0]);       // barrier i lives at bar0 + 8 i
 
@@ -891,7 +898,9 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
 }
 
 // Exclusive prefix over the segments of one chain, in place: on return S_seg[bh][s] / z_seg[bh][s] hold the state
-// segment s starts from, win_seg its incoming window, and S / z / win / pos of the caller the final state.
+// segment s starts from and win_seg its incoming window; win / pos of the caller get their final values here, S / z
+// of the caller are written by the last segment's block of the main pass (the sums of last segments are not
+// computed beforehand, so their slots are not read).
 // grid = (BH, d*d / 1024), 256 threads, four consecutive elements of S per thread.
 __global__ void __launch_bounds__(256)
 prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat16* __restrict__ win_seg,
@@ -905,15 +914,14 @@ prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat1
     float4 d[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (sg0 + j < nseg) d[j] = *reinterpret_cast<const float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4);
+      if (sg0 + j < nseg - 1) d[j] = *reinterpret_cast<const float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4);
 #pragma unroll
     for (int j = 0; j < 16; ++j)
       if (sg0 + j < nseg) {
         *reinterpret_cast<float4*>(S_seg + ((size_t)bh * nseg + sg0 + j) * D * D + e4) = run;
-        run.x += d[j].x; run.y += d[j].y; run.z += d[j].z; run.w += d[j].w;
+        if (sg0 + j < nseg - 1) { run.x += d[j].x; run.y += d[j].y; run.z += d[j].z; run.w += d[j].w; }
       }
   }
-  *reinterpret_cast<float4*>(S + (size_t)bh * D * D + e4) = run;
   if (blockIdx.y == 0 && threadIdx.x < D) {
     const int c = threadIdx.x;
     float rz = init ? z[(size_t)bh * D + c] : 0.f;
@@ -921,15 +929,14 @@ prefix_kernel(float* __restrict__ S_seg, float* __restrict__ z_seg, __nv_bfloat1
       float d[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        if (sg0 + j < nseg) d[j] = z_seg[((size_t)bh * nseg + sg0 + j) * D + c];
+        if (sg0 + j < nseg - 1) d[j] = z_seg[((size_t)bh * nseg + sg0 + j) * D + c];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
         if (sg0 + j < nseg) {
           z_seg[((size_t)bh * nseg + sg0 + j) * D + c] = rz;
-          rz += d[j];
+          if (sg0 + j < nseg - 1) rz += d[j];
         }
     }
-    z[(size_t)bh * D + c] = rz;
     if (c == 0 && bh % H == 0) pos[bh / H] = (init ? pos[bh / H] : 0) + Ttot;
   }
   // Incoming windows: the W-1 values of v before each segment; before the first one the caller's window or zeros.
@@ -985,10 +992,10 @@ template <int PHI>
 static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
                             __nv_bfloat16* win, int64_t* pos, const void* vg, int* status, int nseg, int seg_len,
-                            cudaStream_t s) {
+                            float* S_fin, float* z_fin, cudaStream_t s) {
   const size_t smem = tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               const __nv_bfloat16*, int*, int, int, int, float, int, int, int);
+               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*);
   switch (c.conv_taps) {     // unrolled tap loops for the common small widths
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
@@ -1000,7 +1007,7 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, (const __nv_bfloat16*)vg, status, c.H, T,
-                                                     c.conv_taps, c.eps, init, nseg, seg_len);
+                                                     c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin);
   return cudaGetLastError();
 }
 
@@ -1051,9 +1058,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   cudaError_t e;
   if (nseg == 1) {
     e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
-                                    ctx->d_status, 1, T, s)
+                                    ctx->d_status, 1, T, nullptr, nullptr, s)
             : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
-                                    ctx->d_status, 1, T, s);
+                                    ctx->d_status, 1, T, nullptr, nullptr, s);
     ctx->launches += 1;
     *handled = true;
     return e;
@@ -1066,14 +1073,15 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   auto skern = elu ? tc::segment_state_kernel<LA_PHI_ELU1> : tc::segment_state_kernel<LA_PHI_RELU>;
   e = cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kStateSmem);
   if (e != cudaSuccess) return e;
-  skern<<<dim3(units), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, S_seg, z_seg, ctx->d_status, T, nseg, seg_len);
+  skern<<<dim3(BH * (nseg - 1)), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, S_seg, z_seg, ctx->d_status, T, nseg,
+                                                                               seg_len, nseg - 1);
   tc::prefix_kernel<<<dim3(BH, tc::D * tc::D / 1024), dim3(256), 0, s>>>(S_seg, z_seg, win_seg, (const __nv_bfloat16*)v, st.S,
                                                                           st.z, (__nv_bfloat16*)st.win, st.pos, c.H, T,
                                                                           c.conv_taps, nseg, seg_len, init);
   e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
-                                  seg_len, s)
+                                  seg_len, st.S, st.z, s)
           : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
-                                  seg_len, s);
+                                  seg_len, st.S, st.z, s);
   ctx->launches += 3;
   *handled = true;
   return e;
@@ -1092,7 +1100,7 @@ cudaError_t launch_segment_state_tc(la_ctx* ctx, int B, int T, const void* k, co
   auto skern = c.phi == LA_PHI_ELU1 ? tc::segment_state_kernel<LA_PHI_ELU1> : tc::segment_state_kernel<LA_PHI_RELU>;
   cudaError_t e = cudaFuncSetAttribute(skern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc::kStateSmem);
   if (e != cudaSuccess) return e;
-  skern<<<dim3(BH), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, dS, dz, ctx->d_status, T, 1, T);
+  skern<<<dim3(BH), dim3(tc::kStateThreads), tc::kStateSmem, s>>>(mk, mv, dS, dz, ctx->d_status, T, 1, T, 1);
   ctx->launches += 1;
   *handled = true;
   return cudaGetLastError();
