@@ -107,3 +107,54 @@ def test_a_wait_that_nobody_ends_runs_out_and_reports_it():
     x = torch.randn(1, 2, 130, 128, device="cuda").bfloat16() * 0.1
     o = ctx.la_prefill(x, x, x, torch.ones(2, 128, 3, device="cuda"), st)
     assert ctx.la_last_device_status() == binding.LA_OK and torch.isfinite(o.float()).all()
+
+
+@pytest.mark.parametrize("io,d,T,W,C", [("bf16", 128, 333, 5, 64), ("f32", 64, 200, 32, 37), ("bf16", 64, 300, 3, 256)])
+def test_guards_survive_the_three_branch_block_and_the_segment_sums(io, d, T, W, C):
+    B, H = 2, 3
+    dt = binding.TORCH_DTYPE[io]
+    q, k, v = (dev(x, io) for x in wl.qkv(T + W + C, (B, H, T, d), 0.5, io))
+    w = dev(wl.conv_weights(2, H, d, W), "f32")
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    ar = Arena(64 << 20)
+    st = binding.State(ar.take((B, H, d, d), torch.float32, 0.0), ar.take((B, H, d), torch.float32, 0.0),
+                       ar.take((B, H, W - 1, d), dt, 0.0), ar.take((B,), torch.int64, 0))
+    o = ar.take((B, H, T, d), dt)
+    ctx.la_prefill_grouped(q, k, v, w, st, C, 0.7, d ** -0.5, out=o)
+    dS, dz = ar.take((B, H, d, d), torch.float32), ar.take((B, H, d), torch.float32)
+    ctx.la_segment_state(k, v, dS=dS, dz=dz)
+    parts_S, parts_z = torch.stack([dS, dS, dS]), torch.stack([dz, dz, dz])
+    S2, z2 = ctx.la_state_prefix(parts_S, parts_z, 2, st.S, st.z)
+    torch.cuda.synchronize()
+    assert ctx.la_last_device_status() == binding.LA_OK
+    ar.check()
+    assert torch.isfinite(o.float()).all() and torch.isfinite(dS).all() and torch.isfinite(S2).all()
+    assert torch.allclose(S2, st.S + 2 * dS, rtol=1e-5, atol=1e-5) and torch.allclose(z2, st.z + 2 * dz, rtol=1e-5, atol=1e-5)
+    assert st.pos.tolist() == [T] * B
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other():
+    """Calls of two contexts issued on two streams, interleaved, give the bits of the same calls issued alone."""
+    io, B, H, d, T, W = "bf16", 2, 4, 128, 700, 3
+    q, k, v = (dev(x, io) for x in wl.qkv(77, (B, H, T, d), d ** -0.5, io))
+    w = dev(wl.conv_weights(3, H, d, W), "f32")
+    ca, cb = binding.Context(H, d, W, "elu1", 0.0, io), binding.Context(H, d, W, "relu", 1e-6, io)
+    ref = []
+    for c in (ca, cb):
+        st = c.new_state(B)
+        ref.append((c.la_prefill(q, k, v, w, st), st))
+    torch.cuda.synchronize()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    outs = []
+    for _ in range(3):
+        got = []
+        for c, s in ((ca, sa), (cb, sb)):
+            st = c.new_state(B)
+            with torch.cuda.stream(s):
+                got.append((c.la_prefill(q, k, v, w, st, stream=s), st))
+        outs.append(got)
+    torch.cuda.synchronize()
+    for got in outs:
+        for (o, st), (ro, rst) in zip(got, ref):
+            assert torch.equal(o, ro) and torch.equal(st.S, rst.S) and torch.equal(st.z, rst.z)
+    assert ca.la_last_device_status() == binding.LA_OK and cb.la_last_device_status() == binding.LA_OK
