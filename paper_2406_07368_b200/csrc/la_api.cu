@@ -135,8 +135,15 @@ la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, c
   if (group > la::prefill_grouped_max_group(ctx->cfg)) return LA_ERR_UNSUPPORTED;
   DeviceGuard g(ctx->device);
   if (!g.ok) return LA_ERR_CUDA;
-  return cuda_status(la::launch_prefill_grouped(ctx, B, T, q, k, v, conv_w, group, alpha, softmax_scale, init_state, *st, o,
-                                                static_cast<cudaStream_t>(stream)));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (ctx->prefill_kernel == 0) {
+    bool handled = false;
+    const cudaError_t e = la::launch_prefill_grouped_tc(ctx, B, T, q, k, v, conv_w, group, alpha, softmax_scale, init_state,
+                                                        *st, o, s, &handled);
+    if (e != cudaSuccess) return cuda_status(e);
+    if (handled) return LA_OK;
+  }
+  return cuda_status(la::launch_prefill_grouped(ctx, B, T, q, k, v, conv_w, group, alpha, softmax_scale, init_state, *st, o, s));
 }
 
 int32_t la_prefill_grouped_max_group(const la_ctx* ctx) { return ctx ? la::prefill_grouped_max_group(ctx->cfg) : 0; }

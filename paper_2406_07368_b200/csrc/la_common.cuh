@@ -147,6 +147,9 @@ cudaError_t launch_accept(la_ctx* ctx, int B, int N, const int32_t* parent, cons
 cudaError_t launch_prefill_grouped(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
                                    int group, float alpha, float scale, int init_state, const la_state& st, void* o,
                                    cudaStream_t s);
+cudaError_t launch_prefill_grouped_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
+                                      int group, float alpha, float scale, int init_state, const la_state& st, void* o,
+                                      cudaStream_t s, bool* handled);
 int prefill_grouped_max_group(const la_config& c);   // largest group size the kernel's shared memory holds
 // Sums of one segment of the sequence (dS = sum phi(k) v^T, dz = sum phi(k)), and sums of such parts.
 cudaError_t launch_segment_state(la_ctx* ctx, int B, int T, const void* k, const void* v, float* dS, float* dz, cudaStream_t s);

@@ -89,6 +89,11 @@ __host__ __device__ inline bool global_halo(int W) { return smem_bytes2(W) > 227
 __host__ __device__ inline uint32_t smem_bytes(int W) {
   return global_halo(W) ? off_halo(W) + (uint32_t)(W - 1) * D * 2 + 1024 : smem_bytes2(W);
 }
+// The three-branch mode keeps 4 KB more behind the halo rows: z before the tile as fp32 [128], the halves of
+// phi(q) . z [2][128], and each half-row's running maximum and sum of the softmax [2][128] x 2.
+constexpr uint32_t kGrpScratch = 4096;
+__host__ __device__ inline uint32_t off_grp(int W) { return (smem_bytes(W) - 1024 + 15u) & ~15u; }
+__host__ __device__ inline uint32_t smem_bytes_grp(int W) { return off_grp(W) + kGrpScratch + 1024; }
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -106,6 +111,12 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void sync_group_b() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
+__device__ __forceinline__ void sync_group_a() { asm volatile("bar.sync 5, 256;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void sync_half_b(int hf) {
   if (hf) asm volatile("bar.sync 4, 128;" ::: "memory");
   else asm volatile("bar.sync 3, 128;" ::: "memory");
@@ -290,14 +301,18 @@ __device__ __forceinline__ uint4 pack8(const uint32_t* v) {
                     pack2(__uint_as_float(v[4]), __uint_as_float(v[5])), pack2(__uint_as_float(v[6]), __uint_as_float(v[7])));
 }
 
-template <int PHI, int WT>
+// GRP: the three-branch block of Sec. 4.1 with the group equal to the 128-token tile: the score product runs on the raw
+// q and k and its rows go through a causal softmax (left branch); the products with the state of the earlier tiles are
+// the group-exclusive linear attention (middle branch: there is no intra-tile linear term); both land in one
+// accumulator, the probabilities pre-scaled by (phi(q).z_prev + eps) / alpha so that one row factor finishes both.
+template <int PHI, int WT, bool GRP = false>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                   const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
                   const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
                   __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, const __nv_bfloat16* __restrict__ vg,
                   int* status, int H, int Ttot, int W, float eps, int init, int nseg,
-                  int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin) {
+                  int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin, float alpha, float sm_scale) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -308,6 +323,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const int halo_elems = (W > 1 ? W - 1 : 1) * D;
   const bool gh = global_halo(W);
   volatile int* abort = &sm.abort;
+  // three-branch mode only: z before the tile (fp32), the halves of phi(q) . z, the halves of the softmax statistics
+  float* zs = reinterpret_cast<float*>(smem + off_grp(W));                     // [128]
+  float* dgh = zs + D;                                                         // [2][128]
+  float2* mlh = reinterpret_cast<float2*>(dgh + 2 * D);                        // [2][128] (max, sum)
+  const bool use_glob = GRP && alpha != 0.f;     // alpha = 0: the global branch is switched off altogether
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // A launch covers BH chains cut into nseg segments of seg_len tokens (nseg = 1: whole chains).  Unit u owns
@@ -356,7 +376,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   __syncthreads();
   if (tid < TILE) {
     *reinterpret_cast<__nv_bfloat16*>(smem + OFF_ONES + ext_offset(tid, 0)) = __float2bfloat16_rn(1.f);
-    if (init)                                     // z before tile 0: row 128 of the first K buffer (feature tid)
+    if (GRP) zs[tid] = init ? z[(size_t)u * D + tid] : 0.f;
+    else if (init)                                // z before tile 0: row 128 of the first K buffer (feature tid)
       *reinterpret_cast<__nv_bfloat16*>(smem + OFF_K0 + (tid >> 6) * KBOX_BYTES + BOX_BYTES + (tid & 63) * 2) =
           __float2bfloat16_rn(z[(size_t)u * D + tid]);
   }
@@ -381,6 +402,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         // low descriptor words of step 0: K read along its rows (K-major), K, V and the S copy down their rows
         const uint32_t k_km = desc_lo(kbuf, 16u);
         const uint32_t k_mn = desc_lo(kbuf, KBOX_BYTES), v_mn = desc_lo(vbuf, BOX_BYTES), s_mn = desc_lo(sbase + OFF_S, BOX_BYTES);
+        if (GRP) {
+          // scores of the raw q and k, both operands from shared memory as TMA delivered them; group A applies phi
+          // only once this product is complete
+          ok = mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort) &&
+               mbar_wait((bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0)), (n >> 1) & 1, abort);
+          if (!ok) break;
+          const uint32_t q_km = desc_lo(sbase + OFF_Q, 16u);
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            mma_bf16(tmem + P_COL, desc64(q_km + kstep_kmajor(ks)), desc64(k_km + kstep_kmajor(ks, KBOX_BYTES)),
+                     idesc(false, false, 128), ks > 0);
+          mma_commit((bar0 + 8u * (B_MMA_P)));
+        }
         ok = mbar_wait((bar0 + 8u * (B_PHI)), par, abort);   // phi(Q) of tile n is in TMEM, phi(K) in place
         if (!ok) break;
         tc_fence_after();
@@ -390,11 +424,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
           tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
         }
+        if (!GRP) {
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)   // [P | phi(q).z_prev] = phi(Q) [phi(K); z_prev]^T; 16 channels of phi(Q) = 8 columns
-          mma_bf16_ts(tmem + P_COL, tmem + FQ_COL + 8 * ks, desc64(k_km + kstep_kmajor(ks, KBOX_BYTES)), idesc(false, false, 144),
-                      ks > 0);
-        mma_commit((bar0 + 8u * (B_MMA_P)));
+          for (int ks = 0; ks < 8; ++ks)   // [P | phi(q).z_prev] = phi(Q) [phi(K); z_prev]^T; 16 channels of phi(Q) = 8 columns
+            mma_bf16_ts(tmem + P_COL, tmem + FQ_COL + 8 * ks, desc64(k_km + kstep_kmajor(ks, KBOX_BYTES)),
+                        idesc(false, false, 144), ks > 0);
+          mma_commit((bar0 + 8u * (B_MMA_P)));
+        }
         // The state update needs nothing from the previous tile's epilogue: it fills the time until that epilogue
         // has read the accumulator.
         ok = mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
@@ -412,7 +448,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         if (ok && n >= 1) ok = mbar_wait((bar0 + 8u * (B_EPI0 + (par ^ 1))), ((n - 1) >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after();
-        if (has_state) {
+        if (has_state && (!GRP || use_glob)) {
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)     // O = phi(Q) S_prev
             mma_bf16_ts(tmem + O_COL, tmem + FQ_COL + 8 * ks, desc64(s_mn + kstep_mnmajor(ks)), idesc(false, true, 128), ks > 0);
@@ -424,7 +460,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)       // O += (P o M) V; 16 tokens of every row of P = 8 columns
           mma_bf16_ts(tmem + O_COL, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
-                      idesc(false, true, 128), has_state || ks > 0);
+                      idesc(false, true, 128), (has_state && (!GRP || use_glob)) || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
         if (n + 2 < nchunks) {   // the state update was issued long ago: this K buffer is free and takes tile n+2
           ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);
@@ -531,9 +567,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         *reinterpret_cast<uint4*>(Kb + swz(j, ct & 7)) = j < valid ? phi8<PHI>(x[i]) : make_uint4(0u, 0u, 0u, 0u);
       }
     };
-    ok = mbar_wait((bar0 + 8u * (B_FULL_K0)), 0, abort);
-    ok = __all_sync(0xffffffffu, ok);
-    phi_k(0, ok);
+    if (!GRP) {
+      ok = mbar_wait((bar0 + 8u * (B_FULL_K0)), 0, abort);
+      ok = __all_sync(0xffffffffu, ok);
+      phi_k(0, ok);
+    }
 
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
@@ -541,7 +579,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 
       // ---- phi on Q in place (phi on K of this tile was done one iteration earlier) ----
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort);
+      if (GRP)   // the score product runs on the raw q and k: phi may touch K only once it is complete
+        ok = ok && mbar_wait((bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0)), (n >> 1) & 1, abort) &&
+             mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
+      if (GRP) sync_group_a();                    // z of the previous snapshot (written by other threads) is in place
       // phi(q) of row r, this thread's 64 channels: 32 packed pairs = 32 TMEM columns of lane r.  (The products of
       // tile n-1 that read these columns are complete: the snapshot at the end of the previous iteration waited for them.)
       uint32_t fq[32];
@@ -552,17 +594,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           fq[4 * cc] = f.x; fq[4 * cc + 1] = f.y; fq[4 * cc + 2] = f.z; fq[4 * cc + 3] = f.w;
         }
         LA_TMEM_ST32(tmem + lane_addr + FQ_COL + 32 * hf, fq);
+        if (GRP) {                                // this half of phi(q) . z_prev, z in fp32
+          float dg = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float4 z4 = *reinterpret_cast<const float4*>(zs + 64 * hf + 2 * e);
+            dg = fmaf(lo_f(fq[e]), z4.x, fmaf(hi_f(fq[e]), z4.y, fmaf(lo_f(fq[e + 1]), z4.z, fmaf(hi_f(fq[e + 1]), z4.w, dg))));
+          }
+          dgh[hf * D + r] = dg;
+        }
         tmem_wait_st();
       }
+      if (GRP) phi_k(n, ok);                      // phi on K of this tile, in place, now that the scores are complete
       fence_proxy_async();                        // (phi(K) of this tile, written one iteration earlier)
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PHI)));
       float dpart = 0.f;                          // this half of the row sum of the masked P
 
       // ---- P: causal mask, packed bf16 -> TMEM ----
-      ok = ok && mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
+      if (!GRP) ok = ok && mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
+      if (!GRP && ok) {
         tc_fence_after();
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
@@ -596,11 +648,78 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         denbuf[(par * 2 + hf) * D + r] = dpart;
         tmem_wait_st();
       }
+      if (GRP) {
+        // ---- P: causal softmax along the rows.  A row's 128 columns belong to two threads (halves): each takes the
+        // running maximum and sum of its half, the halves meet through shared memory, and a second pass writes
+        // exp(s - max) / sum back as bf16 -- times (phi(q) . z_prev + eps) / alpha where the global branch is alive, so
+        // that the epilogue's one row factor alpha / (phi(q) . z_prev + eps) finishes both branches.
+        const float c2 = sm_scale * 1.4426950408889634f;       // scores -> exponents of two
+        float m_run = -INFINITY, l_run = 0.f;
+        if (ok) {
+          tc_fence_after();
+#pragma unroll
+          for (int qq = 0; qq < 2; ++qq) {
+            const int col0 = 64 * hf + 32 * qq;
+            if (col0 <= 32 * (wa & 3) + 31) {                   // warp-uniform: some row of this warp reaches col0
+              uint32_t v[32];
+              LA_TMEM_LD32(tmem + P_COL + lane_addr + col0, v);
+              tmem_wait_ld();
+              float bm = -INFINITY;
+#pragma unroll
+              for (int e = 0; e < 32; ++e)
+                if (col0 + e <= r) bm = fmaxf(bm, __uint_as_float(v[e]) * c2);
+              if (bm > -INFINITY) {
+                const float mn = fmaxf(m_run, bm);
+                float acc = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                  if (col0 + e <= r) acc += ex2(__uint_as_float(v[e]) * c2 - mn);
+                l_run = l_run * ex2(m_run - mn) + acc;
+                m_run = mn;
+              }
+            }
+          }
+        }
+        mlh[hf * D + r] = make_float2(m_run, l_run);
+        sync_group_a();
+        const float2 oth = mlh[(hf ^ 1) * D + r];
+        const float m = fmaxf(m_run, oth.x);                    // finite: the row's own column lies in one of the halves
+        const float l = l_run * ex2(m_run - m) + oth.y * ex2(oth.x - m);
+        const float den = dgh[r] + dgh[D + r] + eps;
+        const bool has_g = use_glob && (init || n > 0) && den != 0.f;
+        const float rs = has_g ? den / alpha : 1.f;
+        const float f = rs / l;
+        if (ok) {
+#pragma unroll
+          for (int qq = 0; qq < 2; ++qq) {
+            const int col0 = 64 * hf + 32 * qq;
+            uint32_t pk[16];
+            if (col0 <= 32 * (wa & 3) + 31) {
+              uint32_t v[32];
+              LA_TMEM_LD32(tmem + P_COL + lane_addr + col0, v);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 16; ++e) {
+                const float p0 = col0 + 2 * e <= r ? ex2(__uint_as_float(v[2 * e]) * c2 - m) * f : 0.f;
+                const float p1 = col0 + 2 * e + 1 <= r ? ex2(__uint_as_float(v[2 * e + 1]) * c2 - m) * f : 0.f;
+                pk[e] = pack2(p0, p1);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) pk[e] = 0u;
+            }
+            LA_TMEM_ST16(tmem + P_COL + lane_addr + 64 * hf + 16 * qq, pk);
+          }
+          // the epilogue's row factor is 1 / (the two halves + its eps): the factor here, nothing else
+          denbuf[(par * 2 + hf) * D + r] = hf == 0 ? rs : 0.f;
+          tmem_wait_st();
+        }
+      }
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PDONE)));
 
       // ---- phi on K of the next tile while the tensor cores work on this one ----
-      if (!last) {
+      if (!GRP && !last) {
         ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
         ok = __all_sync(0xffffffffu, ok);
         phi_k(n + 1, ok);
@@ -633,6 +752,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         if (hf == 0) {
           const float zz = __uint_as_float(zbits);
           if (last) zout[r] = zz;
+          else if (GRP) zs[r] = zz;               // fp32, for phi(q) . z of the next tile
           else                                    // row 128 of the K buffer of tile n+1 (its token rows are in place already)
             *reinterpret_cast<__nv_bfloat16*>(smem + (((n + 1) & 1) ? OFF_K1 : OFF_K0) + (r >> 6) * KBOX_BYTES + BOX_BYTES +
                                               (r & 63) * 2) = __float2bfloat16_rn(zz);
@@ -689,7 +809,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       if (ok) {
         // row sum of the masked P + phi(q) . z_prev, both halves gathered by the masking threads
         const float den = denbuf[(par * 2) * D + r] + denbuf[(par * 2 + 1) * D + r];
-        rden = 1.f / (den + eps);
+        rden = 1.f / (den + (GRP ? 0.f : eps));   // (three-branch mode: the masking threads left the finished factor)
       }
       unsigned char* Ob = smem + OFF_V0 + par * TILE_BYTES + hf * BOX_BYTES;
 #pragma unroll
@@ -992,10 +1112,14 @@ template <int PHI>
 static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
                             __nv_bfloat16* win, int64_t* pos, const void* vg, int* status, int nseg, int seg_len,
-                            float* S_fin, float* z_fin, cudaStream_t s) {
-  const size_t smem = tc::smem_bytes(c.conv_taps);
+                            float* S_fin, float* z_fin, cudaStream_t s, bool grouped = false, float alpha = 1.f,
+                            float sm_scale = 1.f) {
+  const size_t smem = grouped ? tc::smem_bytes_grp(c.conv_taps) : tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*);
+               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*, float, float);
+  if (grouped) {
+    kern = c.conv_taps == 3 ? tc::prefill_tc_kernel<PHI, 3, true> : tc::prefill_tc_kernel<PHI, 0, true>;
+  } else
   switch (c.conv_taps) {     // unrolled tap loops for the common small widths
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
@@ -1007,7 +1131,7 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, (const __nv_bfloat16*)vg, status, c.H, T,
-                                                     c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin);
+                                                     c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin, alpha, sm_scale);
   return cudaGetLastError();
 }
 
@@ -1083,6 +1207,30 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
           : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
                                   seg_len, st.S, st.z, s);
   ctx->launches += 3;
+  *handled = true;
+  return e;
+}
+
+// The three-branch block on the tensor cores: bf16 io, d = 128, groups of exactly one 128-token tile, and few enough
+// taps for the 4 KB of extra shared memory.  Sets *handled to false otherwise (the CUDA-core kernel takes those).
+cudaError_t launch_prefill_grouped_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
+                                      int group, float alpha, float scale, int init, const la_state& st, void* o,
+                                      cudaStream_t s, bool* handled) {
+  const la_config& c = ctx->cfg;
+  *handled = false;
+  if (c.io_dtype != LA_BF16 || c.d != tc::D || group != tc::TILE) return cudaSuccess;
+  if (tc::smem_bytes_grp(c.conv_taps) > 227u * 1024u) return cudaSuccess;
+  const int BH = B * c.H;
+  CUtensorMap mq, mk, mv, mo;
+  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
+      !tc::make_map(&mo, o, BH, T))
+    return cudaErrorNotSupported;
+  cudaError_t e = c.phi == LA_PHI_ELU1
+                      ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale)
+                      : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale);
+  ctx->launches += 1;
   *handled = true;
   return e;
 }

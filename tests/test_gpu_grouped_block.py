@@ -121,3 +121,50 @@ def test_grouped_block_rejects_groups_beyond_what_the_kernel_holds():
         ctx.la_prefill_grouped(x, x, x, w, ctx.new_state(1), 0, 1.0, 0.1)
     assert e.value.code == binding.LA_ERR_INVALID_ARG
     assert ctx.la_launch_count() == 0
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+@pytest.mark.parametrize("phi,eps,W,T,alpha,v_mean,zero_w", [
+    ("elu1", 0.0, 3, 700, 1.0, 0.0, False), ("elu1", 0.0, 3, 700, 0.5, 1.0, True), ("relu", 1e-6, 5, 333, 0.7, 1.0, False),
+    ("elu1", 0.0, 3, 128, 1.0, 0.0, False), ("elu1", 0.0, 3, 129, 1.0, 1.0, False), ("elu1", 0.0, 3, 1, 1.0, 0.0, False),
+    ("relu", 0.0, 1, 400, 2.0, 1.0, False), ("elu1", 0.0, 16, 300, 1.0, 0.0, False), ("elu1", 0.0, 3, 2048, 1.0, 1.0, True),
+    ("elu1", 0.0, 3, 500, 0.0, 1.0, False)])
+def test_grouped_block_with_groups_of_one_tile_on_both_kernels(kernel, phi, eps, W, T, alpha, v_mean, zero_w):
+    """Groups of 128 tokens with bf16 and d = 128: the tensor-core kernel (0) and the CUDA-core kernel (1)."""
+    io, B, H, d, C = "bf16", 2, 3, 128, 128
+    q, k, v = wl.qkv(5000 + T + W, (B, H, T, d), 0.5, io, v_mean=v_mean)
+    w = wl.conv_weights(T + W, H, d, W)
+    if zero_w:
+        w = np.zeros_like(w)
+    ctx = binding.Context(H, d, W, phi, eps, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    o = ctx.la_prefill_grouped(dev(q, io), dev(k, io), dev(v, io), dev(w, "f32"), st, C, alpha, d ** -0.5)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want, wst = orc.prefill_grouped_block(q, k, v, w, phi, eps, C, alpha, d ** -0.5)
+    assert rel_err(host(o), want) < TOL[io]
+    if T > 2 * C:
+        assert rel_err(host(o)[:, :, C:], want[:, :, C:]) < TOL[io]
+        assert rel_err(host(o)[:, :, -C:], want[:, :, -C:]) < TOL[io]
+    check_state(st, wst, io)
+
+
+@pytest.mark.parametrize("kernel", [0, 1])
+def test_grouped_block_of_one_tile_continues_and_hands_over_to_decode(kernel):
+    io, B, H, d, C, W, T, cut = "bf16", 1, 2, 128, 128, 4, 900, 384
+    q, k, v = wl.qkv(5100, (B, H, T, d), 0.5, io, v_mean=0.5)
+    w = wl.conv_weights(5100, H, d, W)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    ctx.la_set_prefill_kernel(kernel)
+    st = ctx.new_state(B)
+    sl = lambda x, a, b: dev(x[:, :, a:b], io)
+    o1 = ctx.la_prefill_grouped(sl(q, 0, cut), sl(k, 0, cut), sl(v, 0, cut), dev(w, "f32"), st, C, 0.8, 0.1)
+    o2 = ctx.la_prefill_grouped(sl(q, cut, T), sl(k, cut, T), sl(v, cut, T), dev(w, "f32"), st, C, 0.8, 0.1, init_state=True)
+    want, wst = orc.prefill_grouped_block(q, k, v, w, "elu1", 0.0, C, 0.8, 0.1)
+    assert rel_err(host(torch.cat([o1, o2], dim=2)), want) < TOL[io]
+    assert rel_err(host(o2), want[:, :, cut:]) < TOL[io]
+    check_state(st, wst, io)
+    qs, ks, vs = wl.qkv(5101, (B, H, d), 0.5, io)
+    od = ctx.la_decode_step(dev(qs, io), dev(ks, io), dev(vs, io), dev(w, "f32"), st)
+    wd, _ = orc.decode_step(qs, ks, vs, w, "elu1", 0.0, wst)
+    assert rel_err(host(od), wd) < TOL[io]
