@@ -406,7 +406,8 @@ def promptgen_workload(W: wl.Workload, rank: int, device):
 
 
 def grouped_workload(W: wl.Workload, rank: int, device):
-    """The three-branch block (la_prefill_grouped) on the prefill shape: fp32 arithmetic on the CUDA cores."""
+    """The three-branch block (la_prefill_grouped) on the prefill shape.  bf16 with d = 128 and groups of 64 or 128
+    tokens run on the tensor cores (a group of 64 takes one half-filled 128-row tile); other shapes on the CUDA cores."""
     from paper_2406_07368_b200 import binding
     io = W.io
     q, k, v = W.prefill_inputs()
@@ -440,8 +441,9 @@ def grouped_workload(W: wl.Workload, rank: int, device):
     units = W.B * W.H * W.T
     flops = units * (4 * W.d * W.d + 2 * W.d * (W.chunk + 1) + 2 * W.d * W.W)   # readout + state update, scores + PV, taps
     info = {"ctx": ctx, "tokens_per_step": W.B * W.T, "alg_bytes_per_launch": units * 4 * W.d * 2, "launches_per_step": 1,
-            "h2d": 3 * q.size * 2, "d2h": q.size * 2, "kernel": "prefill_grouped (fp32 CUDA cores)",
-            "flops_per_launch": flops, "bound": "alu", "period": nsets,
+            "h2d": 3 * q.size * 2, "d2h": q.size * 2,
+            "kernel": "prefill_tc in three-branch mode (groups of 64: one half-filled tile per group)",
+            "flops_per_launch": flops, "period": nsets,
             "l2": f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"}
     return step, e2e_step, info
 

@@ -312,7 +312,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                   const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
                   __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, const __nv_bfloat16* __restrict__ vg,
                   int* status, int H, int Ttot, int W, float eps, int init, int nseg,
-                  int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin, float alpha, float sm_scale) {
+                  int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin, float alpha, float sm_scale,
+                  int tstep) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
@@ -334,7 +335,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   // tokens [y0, y0 + T) of chain bh; state, window and z of a unit are addressed by u.
   const int u = blockIdx.x, bh = u / nseg, h = bh % H;
   const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
-  const int nchunks = (T + TILE - 1) / TILE;
+  // tstep: tokens per tile, 128 except for three-branch groups of 64, which take one half-filled tile each (the TMA
+  // boxes are then 64 rows high; rows 64-127 of the operands hold zeros or values that the causal mask discards).
+  const int nchunks = (T + tstep - 1) / tstep;
+  const uint32_t tile_tx = (uint32_t)tstep * 256u;            // bytes a tile's two boxes bring
   const uint32_t bar0 = smem_u32(&sm.bars[0]);    // barrier i lives at bar0 + 8 i
 
   // ---- set-up ----
@@ -371,6 +375,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
   for (int idx = tid; idx < 4096 / 16; idx += kThreads)                        // the 16-column block of ones <- 0
     reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
+  if (GRP && tstep < TILE)                                                     // half-filled tiles: rows 64-127 of V <- 0
+    for (int idx = tid; idx < 4 * 8192 / 16; idx += kThreads)
+      reinterpret_cast<uint4*>(smem + OFF_V0 + (idx >> 9) * BOX_BYTES + 8192)[idx & 511] = make_uint4(0u, 0u, 0u, 0u);
   for (int idx = tid; idx < 4 * 1024 / 16; idx += kThreads)                    // rows 128-135 of the four K boxes <- 0
     reinterpret_cast<uint4*>(smem + OFF_K0 + (idx >> 6) * KBOX_BYTES + BOX_BYTES)[idx & 63] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
@@ -391,7 +398,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     // =============================== MMA issue, the Q and K loads (one lane) ===============================
     if (lane == 0) {
       bool ok = true;
-      mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
+      mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), tile_tx);
       tma_load(sbase + OFF_Q, &mq, 0, y0, bh, (bar0 + 8u * (B_FULL_Q)));
       tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0, bh, (bar0 + 8u * (B_FULL_Q)));
       for (int n = 0; n < nchunks; ++n) {
@@ -420,9 +427,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tc_fence_after();
         // The Q buffer has been read by then (phi(Q) lives in TMEM): its reload, which sets the pace, goes out first.
         if (n + 1 < nchunks) {
-          mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), TILE_BYTES);
-          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
-          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * TILE, bh, (bar0 + 8u * (B_FULL_Q)));
+          mbar_expect_tx((bar0 + 8u * (B_FULL_Q)), tile_tx);
+          tma_load(sbase + OFF_Q, &mq, 0, y0 + (n + 1) * tstep, bh, (bar0 + 8u * (B_FULL_Q)));
+          tma_load(sbase + OFF_Q + BOX_BYTES, &mq, 64, y0 + (n + 1) * tstep, bh, (bar0 + 8u * (B_FULL_Q)));
         }
         if (!GRP) {
 #pragma unroll
@@ -466,9 +473,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);
           if (!ok) break;
           const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
-          mbar_expect_tx(kbar, TILE_BYTES);
-          tma_load(kbuf, &mk, 0, y0 + (n + 2) * TILE, bh, kbar);
-          tma_load(kbuf + KBOX_BYTES, &mk, 64, y0 + (n + 2) * TILE, bh, kbar);
+          mbar_expect_tx(kbar, tile_tx);
+          tma_load(kbuf, &mk, 0, y0 + (n + 2) * tstep, bh, kbar);
+          tma_load(kbuf + KBOX_BYTES, &mk, 64, y0 + (n + 2) * tstep, bh, kbar);
         }
         // P of the next tile overwrites the columns that the last product of this tile reads
         ok = mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);
@@ -482,14 +489,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       bool ok = true;
       for (int n = 0; n < 2 && n < nchunks; ++n) {
         const uint32_t kb = sbase + (n ? OFF_K1 : OFF_K0), kbar = bar0 + 8u * (n ? B_FULL_K1 : B_FULL_K0);
-        mbar_expect_tx(kbar, TILE_BYTES);
-        tma_load(kb, &mk, 0, y0 + n * TILE, bh, kbar);
-        tma_load(kb + KBOX_BYTES, &mk, 64, y0 + n * TILE, bh, kbar);
+        mbar_expect_tx(kbar, tile_tx);
+        tma_load(kb, &mk, 0, y0 + n * tstep, bh, kbar);
+        tma_load(kb + KBOX_BYTES, &mk, 64, y0 + n * tstep, bh, kbar);
       }
       for (int n = 0; n < 2 && n < nchunks; ++n) {
-        mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + n)), TILE_BYTES);
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
-        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * TILE, bh, (bar0 + 8u * (B_FULL_V0 + n)));
+        mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + n)), tile_tx);
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES, &mv, 0, y0 + n * tstep, bh, (bar0 + 8u * (B_FULL_V0 + n)));
+        tma_load(sbase + OFF_V0 + n * TILE_BYTES + BOX_BYTES, &mv, 64, y0 + n * tstep, bh, (bar0 + 8u * (B_FULL_V0 + n)));
       }
       for (int n = 0; n < nchunks; ++n) {
         const uint32_t par = n & 1;
@@ -498,14 +505,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         ok = mbar_wait((bar0 + 8u * (B_STAGED0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
         const uint32_t vb = sbase + OFF_V0 + par * TILE_BYTES;
-        tma_store(&mo, 0, y0 + n * TILE, bh, vb);               // rows past the end of the sequence are clipped
-        tma_store(&mo, 64, y0 + n * TILE, bh, vb + BOX_BYTES);
+        tma_store(&mo, 0, y0 + n * tstep, bh, vb);               // rows past the end of the sequence are clipped
+        tma_store(&mo, 64, y0 + n * tstep, bh, vb + BOX_BYTES);
         tma_commit();
         if (n + 2 < nchunks) {
           tma_wait_read();
-          mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + par)), TILE_BYTES);
-          tma_load(vb, &mv, 0, y0 + (n + 2) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + par)));
-          tma_load(vb + BOX_BYTES, &mv, 64, y0 + (n + 2) * TILE, bh, (bar0 + 8u * (B_FULL_V0 + par)));
+          mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + par)), tile_tx);
+          tma_load(vb, &mv, 0, y0 + (n + 2) * tstep, bh, (bar0 + 8u * (B_FULL_V0 + par)));
+          tma_load(vb + BOX_BYTES, &mv, 64, y0 + (n + 2) * tstep, bh, (bar0 + 8u * (B_FULL_V0 + par)));
         }
       }
       tma_wait_all();                             // every store is complete before the CTA exits
@@ -555,7 +562,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     // phi on the K tile of tile m, in place; rows at or beyond the end of the sequence become zero
     auto phi_k = [&](int m, bool go) {
       if (!go) return;
-      const int valid = min(TILE, T - m * TILE);
+      const int valid = min(tstep, T - m * tstep);
       const int ct = ta & 15, rg = ta >> 4;                     // chunk column 0..15, row group 0..15
       unsigned char* Kb = smem + ((m & 1) ? OFF_K1 : OFF_K0) + (ct >> 3) * KBOX_BYTES;
       uint4 x[8];                                               // all eight loads first: they do not wait for the stores
@@ -770,12 +777,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     bool ok = true;
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
-      const int valid = min(TILE, T - n * TILE);
+      const int valid = min(tstep, T - n * tstep);
       const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
       // rows before this tile, addressed so that row -1 is the last of W-1 rows
       const __nv_bfloat16* halo = !gh      ? halo0 + par * halo_elems
                                   : n == 0 ? halo0
-                                           : vg + ((size_t)bh * Ttot + y0 + (size_t)n * TILE - (W - 1)) * D;
+                                           : vg + ((size_t)bh * Ttot + y0 + (size_t)n * tstep - (W - 1)) * D;
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -828,7 +835,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
             const int cc = 4 * qq + c;                          // chunk inside this half's box
             const int ch0 = 64 * hf + 8 * cc;                   // first channel of the chunk
             outp[j] = make_uint4(0u, 0u, 0u, 0u);
-            if (ok) {
+            if (ok && r < valid) {                              // rows past the tile's tokens stage zeros
               float2 acc[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e)
@@ -1094,12 +1101,12 @@ static EncodeTiledFn encode_fn() {
 
 // [BH, T, 128] bf16 viewed as a 3-D tensor; boxes of 64 columns x 128 rows x 1, 128-byte swizzle.
 // Rows past T read as zeros and are clipped on store.
-static bool make_map(CUtensorMap* m, const void* base, int BH, int T) {
+static bool make_map(CUtensorMap* m, const void* base, int BH, int T, int box_rows = TILE) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)T, (cuuint64_t)BH};
   cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)T * D * 2};
-  cuuint32_t box[3] = {64, (cuuint32_t)TILE, 1};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
   cuuint32_t es[3] = {1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1113,10 +1120,10 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
                             const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
                             __nv_bfloat16* win, int64_t* pos, const void* vg, int* status, int nseg, int seg_len,
                             float* S_fin, float* z_fin, cudaStream_t s, bool grouped = false, float alpha = 1.f,
-                            float sm_scale = 1.f) {
+                            float sm_scale = 1.f, int tstep = tc::TILE) {
   const size_t smem = grouped ? tc::smem_bytes_grp(c.conv_taps) : tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*, float, float);
+               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*, float, float, int);
   if (grouped) {
     kern = c.conv_taps == 3 ? tc::prefill_tc_kernel<PHI, 3, true> : tc::prefill_tc_kernel<PHI, 0, true>;
   } else
@@ -1131,7 +1138,7 @@ static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensor
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, (const __nv_bfloat16*)vg, status, c.H, T,
-                                                     c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin, alpha, sm_scale);
+                                                     c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin, alpha, sm_scale, tstep);
   return cudaGetLastError();
 }
 
@@ -1211,25 +1218,25 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   return e;
 }
 
-// The three-branch block on the tensor cores: bf16 io, d = 128, groups of exactly one 128-token tile, and few enough
-// taps for the 4 KB of extra shared memory.  Sets *handled to false otherwise (the CUDA-core kernel takes those).
+// The three-branch block on the tensor cores: bf16 io, d = 128, groups of one 128-token tile or of 64 tokens (one
+// half-filled tile per group), and few enough taps for the 4 KB of extra shared memory.  Sets *handled to false otherwise (the CUDA-core kernel takes those).
 cudaError_t launch_prefill_grouped_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
                                       int group, float alpha, float scale, int init, const la_state& st, void* o,
                                       cudaStream_t s, bool* handled) {
   const la_config& c = ctx->cfg;
   *handled = false;
-  if (c.io_dtype != LA_BF16 || c.d != tc::D || group != tc::TILE) return cudaSuccess;
+  if (c.io_dtype != LA_BF16 || c.d != tc::D || (group != tc::TILE && group != tc::TILE / 2)) return cudaSuccess;
   if (tc::smem_bytes_grp(c.conv_taps) > 227u * 1024u) return cudaSuccess;
   const int BH = B * c.H;
   CUtensorMap mq, mk, mv, mo;
-  if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
-      !tc::make_map(&mo, o, BH, T))
+  if (!tc::make_map(&mq, q, BH, T, group) || !tc::make_map(&mk, k, BH, T, group) || !tc::make_map(&mv, v, BH, T, group) ||
+      !tc::make_map(&mo, o, BH, T, group))
     return cudaErrorNotSupported;
   cudaError_t e = c.phi == LA_PHI_ELU1
                       ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
-                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale)
+                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale, group)
                       : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
-                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale);
+                                              ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale, group);
   ctx->launches += 1;
   *handled = true;
   return e;

@@ -129,9 +129,11 @@ def test_grouped_block_rejects_groups_beyond_what_the_kernel_holds():
     ("elu1", 0.0, 3, 128, 1.0, 0.0, False), ("elu1", 0.0, 3, 129, 1.0, 1.0, False), ("elu1", 0.0, 3, 1, 1.0, 0.0, False),
     ("relu", 0.0, 1, 400, 2.0, 1.0, False), ("elu1", 0.0, 16, 300, 1.0, 0.0, False), ("elu1", 0.0, 3, 2048, 1.0, 1.0, True),
     ("elu1", 0.0, 3, 500, 0.0, 1.0, False)])
-def test_grouped_block_with_groups_of_one_tile_on_both_kernels(kernel, phi, eps, W, T, alpha, v_mean, zero_w):
-    """Groups of 128 tokens with bf16 and d = 128: the tensor-core kernel (0) and the CUDA-core kernel (1)."""
-    io, B, H, d, C = "bf16", 2, 3, 128, 128
+@pytest.mark.parametrize("C", [128, 64])
+def test_grouped_block_with_groups_of_one_tile_on_both_kernels(C, kernel, phi, eps, W, T, alpha, v_mean, zero_w):
+    """Groups of 128 or 64 tokens with bf16 and d = 128: the tensor-core kernel (0; a group of 64 takes a half-filled
+    tile) and the CUDA-core kernel (1)."""
+    io, B, H, d = "bf16", 2, 3, 128
     q, k, v = wl.qkv(5000 + T + W, (B, H, T, d), 0.5, io, v_mean=v_mean)
     w = wl.conv_weights(T + W, H, d, W)
     if zero_w:
