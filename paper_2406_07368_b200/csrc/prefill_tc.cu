@@ -335,8 +335,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   // tokens [y0, y0 + T) of chain bh; state, window and z of a unit are addressed by u.
   const int u = blockIdx.x, bh = u / nseg, h = bh % H;
   const int y0 = (u % nseg) * seg_len, T = min(seg_len, Ttot - y0);
-  // tstep: tokens per tile, 128 except for three-branch groups of 64, which take one half-filled tile each (the TMA
-  // boxes are then 64 rows high; rows 64-127 of the operands hold zeros or values that the causal mask discards).
+  // tstep: tokens per tile, 128 except for three-branch groups shorter than that, which take one partly filled tile
+  // each (the TMA boxes are then tstep rows high; the rows below hold zeros or values that the causal mask discards).
   const int nchunks = (T + tstep - 1) / tstep;
   const uint32_t tile_tx = (uint32_t)tstep * 256u;            // bytes a tile's two boxes bring
   const uint32_t bar0 = smem_u32(&sm.bars[0]);    // barrier i lives at bar0 + 8 i
@@ -375,9 +375,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
   for (int idx = tid; idx < 4096 / 16; idx += kThreads)                        // the 16-column block of ones <- 0
     reinterpret_cast<uint4*>(smem + OFF_ONES)[idx] = make_uint4(0u, 0u, 0u, 0u);
-  if (GRP && tstep < TILE)                                                     // half-filled tiles: rows 64-127 of V <- 0
-    for (int idx = tid; idx < 4 * 8192 / 16; idx += kThreads)
-      reinterpret_cast<uint4*>(smem + OFF_V0 + (idx >> 9) * BOX_BYTES + 8192)[idx & 511] = make_uint4(0u, 0u, 0u, 0u);
+  if (GRP && tstep < TILE) {                                                   // partly filled tiles: rows tstep-127 of V <- 0
+    const int per_box = (TILE - tstep) * 8;                                    // 16-byte pieces per box
+    for (int idx = tid; idx < 4 * per_box; idx += kThreads)
+      reinterpret_cast<uint4*>(smem + OFF_V0 + (idx / per_box) * BOX_BYTES + tstep * 128)[idx % per_box] = make_uint4(0u, 0u, 0u, 0u);
+  }
   for (int idx = tid; idx < 4 * 1024 / 16; idx += kThreads)                    // rows 128-135 of the four K boxes <- 0
     reinterpret_cast<uint4*>(smem + OFF_K0 + (idx >> 6) * KBOX_BYTES + BOX_BYTES)[idx & 63] = make_uint4(0u, 0u, 0u, 0u);
   __syncthreads();
@@ -1218,14 +1220,15 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   return e;
 }
 
-// The three-branch block on the tensor cores: bf16 io, d = 128, groups of one 128-token tile or of 64 tokens (one
-// half-filled tile per group), and few enough taps for the 4 KB of extra shared memory.  Sets *handled to false otherwise (the CUDA-core kernel takes those).
+// The three-branch block on the tensor cores: bf16 io, d = 128, groups of 32 to 128 tokens (one tile per group, partly
+// filled below 128: a group of 64 runs the tensor cores half empty and still beats the CUDA-core kernel seven times;
+// below 32 that kernel takes over), and few enough taps for the 4 KB of extra shared memory.  Sets *handled to false otherwise (the CUDA-core kernel takes those).
 cudaError_t launch_prefill_grouped_tc(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
                                       int group, float alpha, float scale, int init, const la_state& st, void* o,
                                       cudaStream_t s, bool* handled) {
   const la_config& c = ctx->cfg;
   *handled = false;
-  if (c.io_dtype != LA_BF16 || c.d != tc::D || (group != tc::TILE && group != tc::TILE / 2)) return cudaSuccess;
+  if (c.io_dtype != LA_BF16 || c.d != tc::D || group < 32 || group > tc::TILE) return cudaSuccess;
   if (tc::smem_bytes_grp(c.conv_taps) > 227u * 1024u) return cudaSuccess;
   const int BH = B * c.H;
   CUtensorMap mq, mk, mv, mo;

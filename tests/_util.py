@@ -46,4 +46,20 @@ def rel_err_octaves(x, y, axis: int = 2) -> float:
     return worst
 
 
+def rel_err_group_octaves(x, y, group: int, axis: int = 2) -> float:
+    """rel_err per octave of the position WITHIN a group of `group` tokens (all groups together), the largest.
+
+    The local branch of the three-branch block is a softmax mean over the tokens of the group so far, so with zero
+    taps and zero-mean values the output's scale follows the position in the group the way rel_err_octaves
+    describes for the position in a fresh sequence.
+    """
+    x, y = np.asarray(x), np.asarray(y)
+    t = np.arange(y.shape[axis]) % group
+    worst = 0.0
+    for lo, hi in position_octaves(group):
+        pick = np.nonzero((t >= lo) & (t < hi))[0]
+        worst = max(worst, rel_err(np.take(x, pick, axis=axis), np.take(y, pick, axis=axis)))
+    return worst
+
+
 TOL = {"f32": 1e-4, "bf16": 2e-2}

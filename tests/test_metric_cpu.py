@@ -51,3 +51,19 @@ def test_octaves_tile_the_positions_and_see_the_fault_at_late_rows():
     x = y.copy()
     x[:, :, -256:] += 0.2 / np.sqrt(T)                  # an offset of a fifth of the late rows' own size
     assert rel_err_octaves(x, y) > 2.0 * rel_err(x, y) and rel_err_octaves(x, y) > 0.15
+
+
+def test_group_octaves_pick_the_position_within_the_group():
+    from tests._util import rel_err_group_octaves
+    T, C = 50, 16
+    y = np.ones((1, 1, T, 4))
+    x = y.copy()
+    assert rel_err_group_octaves(x, y, C) == 0.0
+    x[0, 0, 35] *= 1.25                                  # position 3 of the third group
+    assert abs(rel_err_group_octaves(x, y, C) - 0.25) < 1e-12
+    # a decaying signal within each group: a fault at the group's late rows hides behind the tensor's RMS
+    t = np.arange(T) % C
+    y = (1.0 / (1.0 + t) ** 2)[None, None, :, None] * np.ones((1, 1, T, 4))
+    x = y.copy()
+    x[:, :, t >= 8] += 0.2 * y[:, :, t >= 8]
+    assert rel_err(x, y) < 0.02 < 0.15 < rel_err_group_octaves(x, y, C)
