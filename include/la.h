@@ -117,7 +117,9 @@ const char* la_status_str(la_status s);
  *   st          in-out; on return holds S, z, the window and pos after the T tokens
  *   o           [B, H, T, d] io type
  *
- * Kernels: bf16 io with d = 128 runs grouped on the tensor cores (128-token tiles).  fp32 io, and
+ * Kernels: bf16 io with d = 128 runs grouped on the tensor cores (128-token tiles); with more than
+ * 5 taps its tap sum is formed in fp32, added to the attention term after that term has been
+ * rounded to bf16, and the sum rounded to bf16 (with fewer taps both terms meet in fp32).  fp32 io, and
  * d = 64 in either type, take a CUDA-core kernel that walks the tokens in order -- the cumulative
  * sum taken literally, every product an fp32 multiply-add, which is what the fp32 tolerance
  * needs; it is correct for any T but far slower per token.
@@ -148,8 +150,10 @@ la_status la_prefill(la_ctx* ctx, int32_t B, int32_t T, const void* q, const voi
  *                  W-1 values of v, pos the token count
  *   other arguments as for la_prefill.
  *
- * This entry point runs on the CUDA cores in fp32 (a register-tiled kernel, one thread block per (batch, head)); it
- * is several times slower per token than the tensor-core la_prefill. */
+ * Kernels: bf16 io with d = 128 and groups of 32 to 128 tokens run on the tensor cores, one 128-row tile per group
+ * (a shorter group leaves the rest of its tile empty; the probabilities of the softmax are rounded to bf16 there
+ * before they multiply v).  Everything else runs on the CUDA cores in fp32 (a register-tiled kernel, one thread
+ * block per (batch, head)), several times slower per token. */
 la_status la_prefill_grouped(la_ctx* ctx, int32_t B, int32_t T, const void* q, const void* k, const void* v,
                              const float* conv_w, int32_t group, float alpha, float softmax_scale, int32_t init_state,
                              la_state* st /*host struct*/, void* o, void* stream);

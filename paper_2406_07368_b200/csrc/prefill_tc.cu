@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "la_common.cuh"
 
@@ -82,18 +83,24 @@ enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
-// Two halo buffers (the rows of v before a tile, for the convolution) while they fit; for the longest tap windows
-// one buffer for the first tile only, and later tiles take those rows from v in global memory.
-__host__ __device__ inline uint32_t smem_bytes2(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
-__host__ __device__ inline bool global_halo(int W) { return smem_bytes2(W) > 227u * 1024u; }
-__host__ __device__ inline uint32_t smem_bytes(int W) {
-  return global_halo(W) ? off_halo(W) + (uint32_t)(W - 1) * D * 2 + 1024 : smem_bytes2(W);
-}
+// Two halo buffers (the rows of v before a tile, for the convolution): tile n reads one and fills the other.
+__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
 // The three-branch mode keeps 4 KB more behind the halo rows: z before the tile as fp32 [128], the halves of
 // phi(q) . z [2][128], and each half-row's running maximum and sum of the softmax [2][128] x 2.
 constexpr uint32_t kGrpScratch = 4096;
-__host__ __device__ inline uint32_t off_grp(int W) { return (smem_bytes(W) - 1024 + 15u) & ~15u; }
-__host__ __device__ inline uint32_t smem_bytes_grp(int W) { return off_grp(W) + kGrpScratch + 1024; }
+// The epilogue for longer tap windows ("long" below) keeps the taps padded with zeros to whole groups of 8 and ONE
+// halo buffer, updated in place, of as many rows as the padded taps reach back (the rows before the window stay 0).
+__host__ __device__ inline uint32_t long_taps(int W) { return ((uint32_t)W + 7u) & ~7u; }
+__host__ __device__ inline uint32_t off_halo_long(int W) { return off_w() + long_taps(W) * D * 4; }
+__host__ __device__ inline uint32_t smem_bytes_long(int W) { return off_halo_long(W) + (long_taps(W) - 1) * D * 2 + 1024; }
+__host__ __device__ inline uint32_t off_grp(int W, bool lng = false) {
+  return ((lng ? smem_bytes_long(W) : smem_bytes(W)) - 1024 + 15u) & ~15u;
+}
+__host__ __device__ inline uint32_t smem_bytes_grp(int W, bool lng = false) { return off_grp(W, lng) + kGrpScratch + 1024; }
+// Which windows take the long epilogue: above 5 taps it is the faster of the two (measured on 128 chains of 2048
+// tokens: 6 taps 126 us either way, 8 taps 132 against 154 us, 16 taps 126 against 254, 32 taps 162 against 686).
+// The three-branch mode compiles the short epilogue for 3 taps only.
+inline bool long_epilogue(int W, bool grouped = false) { return grouped ? W != 3 : W > 5; }
 
 // ---- PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -296,6 +303,89 @@ __device__ __forceinline__ void conv8(float2* acc, int W, int r, int cc, int ch0
   }
 }
 
+// Long-window epilogue: one thread owns a pair of channels and 32 consecutive rows of the tile, in four blocks of 8.
+// conv_block adds one group of 8 taps to the 8 sums of block BLK: the 15 rows of v that those taps reach are each
+// read once, as one packed pair, and feed up to 8 of the sums.  Where the rows come from is fixed at compile time:
+//   ALL_V  the V buffer: pg[k] = the thread's column at (its first row - 8 g), for rows = k mod 8 (the swizzle)
+//   ALL_H  the halo column: hq = its row 8 (BLK - g) - 7
+//   MIXED  (g = BLK, first 32 rows of the tile) rows -7 ... -1 from the halo (hq = its row -7), rows 0 ... 7 from V
+// so that every load is one instruction with an immediate offset.
+template <int I, int N, typename F>
+__device__ __forceinline__ void static_for(F&& f) {           // f(integral_constant<int, I>) ... for I, I + 1, ..., N - 1
+  if constexpr (I < N) {
+    f(std::integral_constant<int, I>{});
+    static_for<I + 1, N>(f);
+  }
+}
+enum { ALL_V = 0, MIXED = 1, ALL_H = 2 };
+// (Shared-memory addresses as 32-bit numbers and explicit ld.shared / st.shared: one register per address.)
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ float2 lds_f2(uint32_t a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+  return v;
+}
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+template <int BLK, int KIND>
+__device__ __forceinline__ void conv_block(float2 (&acc)[8], uint32_t wtap, const uint32_t (&pg)[8], uint32_t hq) {
+  float2 wg[8];
+  static_for<0, 8>([&](auto tc_) {
+    constexpr int t = decltype(tc_)::value;
+    wg[t] = lds_f2(wtap + t * (D * 4));
+  });
+  static_for<0, 15>([&](auto ic) {
+    constexpr int i = decltype(ic)::value;
+    uint32_t u;
+    if constexpr (KIND == ALL_V) {
+      constexpr int rel = 8 * BLK - 7 + i;        // row, from the thread's first row, before the 8 g rows of the group
+      u = lds32(pg[rel & 7] + rel * 128);
+    } else if constexpr (KIND == ALL_H || i < 7) {
+      u = lds32(hq + i * (D * 2));
+    } else {
+      u = lds32(pg[i - 7] + (i - 7) * 128);
+    }
+    const float2 x = bf2(u);
+    static_for<0, 8>([&](auto tc_) {
+      constexpr int tau = decltype(tc_)::value;   // tap (within the group) that links input row i to sum jj
+      constexpr int jj = i - 7 + tau;
+      if constexpr (jj >= 0 && jj < 8) acc[jj] = __ffma2_rn(wg[tau], x, acc[jj]);
+    });
+  });
+}
+// All tap groups of block BLK (rows 8 BLK ... 8 BLK + 7 of the thread), then the sums are added to the attention
+// term that waits in the output tile.  FIRST: the thread owns the first 32 rows of the tile (rows before them
+// come from the halo, hend = the halo column just past its last row).
+template <int BLK, bool FIRST>
+__device__ __forceinline__ void conv_rows(uint32_t wcol, const uint32_t (&pv)[8], uint32_t sthr, int cc, uint32_t hend, int ngroups) {
+  float2 acc[8];
+#pragma unroll
+  for (int jj = 0; jj < 8; ++jj) acc[jj] = make_float2(0.f, 0.f);
+#pragma unroll 1
+  for (int g = 0; g < ngroups; ++g) {
+    const uint32_t wtap = wcol + g * (8 * D * 4);
+    if (!FIRST || g < BLK) {
+      uint32_t pg[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) pg[k] = pv[k] - g * 1024;
+      conv_block<BLK, ALL_V>(acc, wtap, pg, 0u);
+    } else if (g == BLK) {
+      conv_block<BLK, MIXED>(acc, wtap, pv, hend - 7 * (D * 2));
+    } else {
+      conv_block<BLK, ALL_H>(acc, wtap, pv, hend + (8 * (BLK - g) - 7) * (D * 2));
+    }
+  }
+#pragma unroll
+  for (int jj = 0; jj < 8; ++jj) {
+    const uint32_t at = sthr + (8 * BLK + jj) * 128 + ((cc ^ jj) << 4);
+    const float2 la = bf2(lds32(at));
+    sts32(at, pack2(acc[jj].x + la.x, acc[jj].y + la.y));
+  }
+}
+
 __device__ __forceinline__ uint4 pack8(const uint32_t* v) {
   return make_uint4(pack2(__uint_as_float(v[0]), __uint_as_float(v[1])), pack2(__uint_as_float(v[2]), __uint_as_float(v[3])),
                     pack2(__uint_as_float(v[4]), __uint_as_float(v[5])), pack2(__uint_as_float(v[6]), __uint_as_float(v[7])));
@@ -310,7 +400,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                   const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
                   const float* __restrict__ w, float* __restrict__ S, float* __restrict__ z,
-                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos, const __nv_bfloat16* __restrict__ vg,
+                  __nv_bfloat16* __restrict__ win, int64_t* __restrict__ pos,
                   int* status, int H, int Ttot, int W, float eps, int init, int nseg,
                   int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin, float alpha, float sm_scale,
                   int tstep) {
@@ -318,14 +408,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   Small& sm = *reinterpret_cast<Small*>(smem + OFF_SMALL);
-  float* wsm = reinterpret_cast<float*>(smem + off_w());                       // [W][128]
-  // two halo buffers [W-1][128], oldest row first: tile n reads buffer n&1 and writes buffer (n+1)&1
-  __nv_bfloat16* halo0 = reinterpret_cast<__nv_bfloat16*>(smem + off_halo(W));
+  constexpr bool LONG = WT < 0;                  // the epilogue for longer tap windows
+  float* wsm = reinterpret_cast<float*>(smem + off_w());                       // [W][128] ([W up to a multiple of 8][128] if LONG)
+  // two halo buffers [W-1][128], oldest row first: tile n reads buffer n&1 and writes buffer (n+1)&1 (LONG: one buffer)
+  __nv_bfloat16* halo0 = reinterpret_cast<__nv_bfloat16*>(smem + (LONG ? off_halo_long(W) : off_halo(W)));
   const int halo_elems = (W > 1 ? W - 1 : 1) * D;
-  const bool gh = global_halo(W);
   volatile int* abort = &sm.abort;
   // three-branch mode only: z before the tile (fp32), the halves of phi(q) . z, the halves of the softmax statistics
-  float* zs = reinterpret_cast<float*>(smem + off_grp(W));                     // [128]
+  float* zs = reinterpret_cast<float*>(smem + off_grp(W, LONG));               // [128]
   float* dgh = zs + D;                                                         // [2][128]
   float2* mlh = reinterpret_cast<float2*>(dgh + 2 * D);                        // [2][128] (max, sum)
   const bool use_glob = GRP && alpha != 0.f;     // alpha = 0: the global branch is switched off altogether
@@ -369,7 +459,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  for (int idx = tid; idx < W * D; idx += kThreads) wsm[idx] = w[((size_t)h * D + (idx % D)) * W + idx / D];
+  for (int idx = tid; idx < (LONG ? (int)long_taps(W) : W) * D; idx += kThreads)
+    wsm[idx] = idx < W * D ? w[((size_t)h * D + (idx % D)) * W + idx / D] : 0.f;
+  if (LONG) {                                    // [long_taps - 1][128]: zeros, then the W-1 rows of the window
+    const int lead = ((int)long_taps(W) - W) * D;
+    for (int idx = tid; idx < ((int)long_taps(W) - 1) * D; idx += kThreads)
+      halo0[idx] = init && idx >= lead ? win[(size_t)u * (W - 1) * D + idx - lead] : __float2bfloat16_rn(0.f);
+  } else
   for (int idx = tid; idx < (W - 1) * D; idx += kThreads)
     halo0[idx] = init ? win[(size_t)u * (W - 1) * D + idx] : __float2bfloat16_rn(0.f);
   float* denbuf = reinterpret_cast<float*>(smem + OFF_DEN);
@@ -471,7 +567,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16_ts(tmem + O_COL, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
                       idesc(false, true, 128), (has_state && (!GRP || use_glob)) || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
-        if (n + 2 < nchunks) {   // the state update was issued long ago: this K buffer is free and takes tile n+2
+        if (!LONG && n + 2 < nchunks) {   // the state update was issued long ago: this K buffer is free and takes tile n+2
           ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);
           if (!ok) break;
           const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
@@ -507,6 +603,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         ok = mbar_wait((bar0 + 8u * (B_STAGED0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
         const uint32_t vb = sbase + OFF_V0 + par * TILE_BYTES;
+        if (LONG) {
+          // the outputs wait in the token rows of this tile's K buffer; every tap has been taken from its V buffer
+          const uint32_t kb = sbase + (par ? OFF_K1 : OFF_K0), kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
+          tma_store(&mo, 0, y0 + n * tstep, bh, kb);
+          tma_store(&mo, 64, y0 + n * tstep, bh, kb + KBOX_BYTES);
+          tma_commit();
+          if (n + 2 < nchunks) {
+            mbar_expect_tx((bar0 + 8u * (B_FULL_V0 + par)), tile_tx);
+            tma_load(vb, &mv, 0, y0 + (n + 2) * tstep, bh, (bar0 + 8u * (B_FULL_V0 + par)));
+            tma_load(vb + BOX_BYTES, &mv, 64, y0 + (n + 2) * tstep, bh, (bar0 + 8u * (B_FULL_V0 + par)));
+            tma_wait_read();
+            mbar_expect_tx(kbar, tile_tx);
+            tma_load(kb, &mk, 0, y0 + (n + 2) * tstep, bh, kbar);
+            tma_load(kb + KBOX_BYTES, &mk, 64, y0 + (n + 2) * tstep, bh, kbar);
+          }
+          continue;
+        }
         tma_store(&mo, 0, y0 + n * tstep, bh, vb);               // rows past the end of the sequence are clipped
         tma_store(&mo, 64, y0 + n * tstep, bh, vb + BOX_BYTES);
         tma_commit();
@@ -777,18 +890,100 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     const int hf = warp >> 2;                     // column half
     const uint32_t lane_addr = (uint32_t)(32 * (warp & 3)) << 16;
     bool ok = true;
+    if constexpr (LONG) {
+      // Two phases per tile.  (1) Row by row, as the accumulator's lanes dictate: the attention term O / den goes,
+      // rounded to bf16, into the token rows of this tile's K buffer, which every product has finished with (its
+      // reload for tile n + 2 waits, in this mode, until the outputs have left).  (2) Channel pair by channel pair:
+      // thread (cp, jq) owns channels 2 cp, 2 cp + 1 and rows 32 jq ... 32 jq + 31, forms the tap sums of 16 rows at a
+      // time in registers (every row of v it needs is read once per group of 8 taps, and the taps of a group sit in
+      // registers), adds the attention term and writes the output over it.  The shared-memory traffic of a tile no
+      // longer grows with rows x taps x 16 bytes, and the V buffer is never written.
+      const int cp = tid & 63, jq = tid >> 6;
+      const int cc = (cp & 31) >> 2;                                         // 16-byte piece of the pair in its box row
+      const uint32_t colv = (uint32_t)(cp >> 5) * BOX_BYTES + (uint32_t)(cp & 3) * 4u + (uint32_t)jq * 4096u;
+      const uint32_t colk = (uint32_t)(cp >> 5) * KBOX_BYTES + (uint32_t)(cp & 3) * 4u + (uint32_t)jq * 4096u;
+      const int lead = (int)long_taps(W) - W;                                // rows of zeros at the head of the halo
+      const uint32_t hcol = sbase + off_halo_long(W) + 4u * cp;
+      const uint32_t hend = hcol + (long_taps(W) - 1) * (D * 2);
+      const uint32_t wcol = sbase + off_w() + 8u * cp;
+      const int ngroups = (W + 7) >> 3;
+      for (int n = 0; n < nchunks; ++n) {
+        const uint32_t par = n & 1;
+        const int valid = min(tstep, T - n * tstep);
+        const uint32_t vthr = sbase + OFF_V0 + par * TILE_BYTES + colv;       // this thread's column at its first row
+        unsigned char* stage = smem + (par ? OFF_K1 : OFF_K0);
+        ok = ok && mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);   // also: every product that reads K or V is done
+        ok = __all_sync(0xffffffffu, ok);
+        uint32_t v[32];
+        float rden = 0.f;
+        if (ok) {
+          tc_fence_after();
+          LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf, v);
+          const float den = denbuf[(par * 2) * D + r] + denbuf[(par * 2 + 1) * D + r];
+          rden = 1.f / (den + (GRP ? 0.f : eps));
+        }
+        unsigned char* Lb = stage + hf * KBOX_BYTES;
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          if (ok) {
+            tmem_wait_ld();
+            uint4 la[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              la[c] = make_uint4(pack2(__uint_as_float(v[8 * c]) * rden, __uint_as_float(v[8 * c + 1]) * rden),
+                                 pack2(__uint_as_float(v[8 * c + 2]) * rden, __uint_as_float(v[8 * c + 3]) * rden),
+                                 pack2(__uint_as_float(v[8 * c + 4]) * rden, __uint_as_float(v[8 * c + 5]) * rden),
+                                 pack2(__uint_as_float(v[8 * c + 6]) * rden, __uint_as_float(v[8 * c + 7]) * rden));
+            if (qq == 0) LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf + 32, v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint4*>(Lb + swz(r, 4 * qq + c)) = la[c];
+          }
+        }
+        tc_fence_before();
+        mbar_arrive((bar0 + 8u * (B_EPI0 + par)));           // this accumulator has been read
+        ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        sync_group_b();                                      // the attention term of every row is in place
+        if (ok) {
+          uint32_t pv[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) pv[k] = vthr + ((cc ^ k) << 4);
+          const uint32_t sthr = sbase + (par ? OFF_K1 : OFF_K0) + colk;
+          const int mine = valid - 32 * jq;                  // rows of this thread that hold tokens
+          if (jq == 0) {
+            if (mine > 0) conv_rows<0, true>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 8) conv_rows<1, true>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 16) conv_rows<2, true>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 24) conv_rows<3, true>(wcol, pv, sthr, cc, hend, ngroups);
+            // The rows before the next tile: the last W-1 of (halo ++ valid rows of v), in place.  This thread is the
+            // only one that reads or writes this column of the halo (the rows of the other threads start at 32, and
+            // no window reaches back further than 31 rows).
+            for (int i = 0; i < W - 1; ++i) {
+              const int src = valid - (W - 1) + i;
+              const uint32_t x = src >= 0 ? lds32(vthr + src * 128 + ((cc ^ (src & 7)) << 4)) : lds32(hend + src * (D * 2));
+              sts32(hcol + (lead + i) * (D * 2), x);
+            }
+          } else {
+            if (mine > 0) conv_rows<0, false>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 8) conv_rows<1, false>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 16) conv_rows<2, false>(wcol, pv, sthr, cc, hend, ngroups);
+            if (mine > 24) conv_rows<3, false>(wcol, pv, sthr, cc, hend, ngroups);
+          }
+        }
+        fence_proxy_async();
+        mbar_arrive((bar0 + 8u * (B_STAGED0 + par)));
+      }
+    } else
     for (int n = 0; n < nchunks; ++n) {
       const uint32_t par = n & 1;
       const int valid = min(tstep, T - n * tstep);
       const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
       // rows before this tile, addressed so that row -1 is the last of W-1 rows
-      const __nv_bfloat16* halo = !gh      ? halo0 + par * halo_elems
-                                  : n == 0 ? halo0
-                                           : vg + ((size_t)bh * Ttot + y0 + (size_t)n * tstep - (W - 1)) * D;
+      const __nv_bfloat16* halo = halo0 + par * halo_elems;
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok && !gh) {
+      if (ok) {
         // next halo <- last W-1 rows of (halo ++ valid rows of V), 16 bytes (8 channels) per thread; each half of the
         // group copies its own 64 channels
         const unsigned char* Vc = Vt + hf * BOX_BYTES;
@@ -863,12 +1058,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     sync_group_b();                               // both halves of the last halo are complete
     if (ok && tid < D) {
       // the window to carry on: the last W-1 values of (incoming window ++ this unit's v)
-      const __nv_bfloat16* halo = halo0 + (nchunks & 1) * halo_elems;
-      for (int i = 0; i < W - 1; ++i) {
-        const int t = T - (W - 1) + i;
-        win[((size_t)u * (W - 1) + i) * D + tid] =
-            !gh ? halo[i * D + tid] : t >= 0 ? vg[((size_t)bh * Ttot + y0 + t) * D + tid] : halo0[(t + W - 1) * D + tid];
-      }
+      const __nv_bfloat16* halo = halo0 + (LONG ? ((int)long_taps(W) - W) * D : (nchunks & 1) * halo_elems);
+      for (int i = 0; i < W - 1; ++i) win[((size_t)u * (W - 1) + i) * D + tid] = halo[i * D + tid];
       if (tid == 0 && h == 0 && nseg == 1) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
   }
@@ -1120,26 +1311,27 @@ static bool make_map(CUtensorMap* m, const void* base, int BH, int T, int box_ro
 template <int PHI>
 static cudaError_t launch_w(const la_config& c, int units, int T, const CUtensorMap& mq, const CUtensorMap& mk,
                             const CUtensorMap& mv, const CUtensorMap& mo, const float* w, int init, float* S, float* z,
-                            __nv_bfloat16* win, int64_t* pos, const void* vg, int* status, int nseg, int seg_len,
+                            __nv_bfloat16* win, int64_t* pos, int* status, int nseg, int seg_len,
                             float* S_fin, float* z_fin, cudaStream_t s, bool grouped = false, float alpha = 1.f,
                             float sm_scale = 1.f, int tstep = tc::TILE) {
-  const size_t smem = grouped ? tc::smem_bytes_grp(c.conv_taps) : tc::smem_bytes(c.conv_taps);
+  const bool lng = tc::long_epilogue(c.conv_taps, grouped);
+  const size_t smem = grouped ? tc::smem_bytes_grp(c.conv_taps, lng) : lng ? tc::smem_bytes_long(c.conv_taps) : tc::smem_bytes(c.conv_taps);
   void (*kern)(CUtensorMap, CUtensorMap, CUtensorMap, CUtensorMap, const float*, float*, float*, __nv_bfloat16*, int64_t*,
-               const __nv_bfloat16*, int*, int, int, int, float, int, int, int, float*, float*, float, float, int);
+               int*, int, int, int, float, int, int, int, float*, float*, float, float, int);
   if (grouped) {
-    kern = c.conv_taps == 3 ? tc::prefill_tc_kernel<PHI, 3, true> : tc::prefill_tc_kernel<PHI, 0, true>;
+    kern = lng ? tc::prefill_tc_kernel<PHI, -1, true> : tc::prefill_tc_kernel<PHI, 3, true>;
   } else
-  switch (c.conv_taps) {     // unrolled tap loops for the common small widths
+  switch (c.conv_taps) {     // short windows: the tap loop unrolled; the others: the long epilogue
     case 1: kern = tc::prefill_tc_kernel<PHI, 1>; break;
     case 2: kern = tc::prefill_tc_kernel<PHI, 2>; break;
     case 3: kern = tc::prefill_tc_kernel<PHI, 3>; break;
     case 4: kern = tc::prefill_tc_kernel<PHI, 4>; break;
     case 5: kern = tc::prefill_tc_kernel<PHI, 5>; break;
-    default: kern = tc::prefill_tc_kernel<PHI, 0>; break;
+    default: kern = tc::prefill_tc_kernel<PHI, -1>; break;
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, (const __nv_bfloat16*)vg, status, c.H, T,
+  kern<<<dim3(units), dim3(tc::kThreads), smem, s>>>(mq, mk, mv, mo, w, S, z, win, pos, status, c.H, T,
                                                      c.conv_taps, c.eps, init, nseg, seg_len, S_fin, z_fin, alpha, sm_scale, tstep);
   return cudaGetLastError();
 }
@@ -1178,7 +1370,8 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   const la_config& c = ctx->cfg;
   *handled = false;
   if (c.io_dtype != LA_BF16 || c.d != tc::D) return cudaSuccess;
-  if (tc::smem_bytes(c.conv_taps) > 227u * 1024u) return cudaSuccess;   // (does not happen up to LA_MAX_TAPS)
+  if ((tc::long_epilogue(c.conv_taps) ? tc::smem_bytes_long(c.conv_taps) : tc::smem_bytes(c.conv_taps)) > 227u * 1024u)
+    return cudaSuccess;                                                  // (does not happen up to LA_MAX_TAPS)
   const int BH = B * c.H;
   CUtensorMap mq, mk, mv, mo;
   if (!tc::make_map(&mq, q, BH, T) || !tc::make_map(&mk, k, BH, T) || !tc::make_map(&mv, v, BH, T) ||
@@ -1190,9 +1383,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   const bool elu = c.phi == LA_PHI_ELU1;
   cudaError_t e;
   if (nseg == 1) {
-    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+    e = elu ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                     ctx->d_status, 1, T, nullptr, nullptr, s)
-            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+            : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                     ctx->d_status, 1, T, nullptr, nullptr, s);
     ctx->launches += 1;
     *handled = true;
@@ -1211,9 +1404,9 @@ cudaError_t launch_prefill_tc(la_ctx* ctx, int B, int T, const void* q, const vo
   tc::prefix_kernel<<<dim3(BH, tc::D * tc::D / 1024), dim3(256), 0, s>>>(S_seg, z_seg, win_seg, (const __nv_bfloat16*)v, st.S,
                                                                           st.z, (__nv_bfloat16*)st.win, st.pos, c.H, T,
                                                                           c.conv_taps, nseg, seg_len, init);
-  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
+  e = elu ? launch_w<LA_PHI_ELU1>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
                                   seg_len, st.S, st.z, s)
-          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, v, ctx->d_status, nseg,
+          : launch_w<LA_PHI_RELU>(c, units, T, mq, mk, mv, mo, w, 1, S_seg, z_seg, win_seg, st.pos, ctx->d_status, nseg,
                                   seg_len, st.S, st.z, s);
   ctx->launches += 3;
   *handled = true;
@@ -1229,16 +1422,16 @@ cudaError_t launch_prefill_grouped_tc(la_ctx* ctx, int B, int T, const void* q, 
   const la_config& c = ctx->cfg;
   *handled = false;
   if (c.io_dtype != LA_BF16 || c.d != tc::D || group < 32 || group > tc::TILE) return cudaSuccess;
-  if (tc::smem_bytes_grp(c.conv_taps) > 227u * 1024u) return cudaSuccess;
+  if (tc::smem_bytes_grp(c.conv_taps, tc::long_epilogue(c.conv_taps, true)) > 227u * 1024u) return cudaSuccess;
   const int BH = B * c.H;
   CUtensorMap mq, mk, mv, mo;
   if (!tc::make_map(&mq, q, BH, T, group) || !tc::make_map(&mk, k, BH, T, group) || !tc::make_map(&mv, v, BH, T, group) ||
       !tc::make_map(&mo, o, BH, T, group))
     return cudaErrorNotSupported;
   cudaError_t e = c.phi == LA_PHI_ELU1
-                      ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+                      ? launch_w<LA_PHI_ELU1>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                               ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale, group)
-                      : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos, v,
+                      : launch_w<LA_PHI_RELU>(c, BH, T, mq, mk, mv, mo, w, init, st.S, st.z, (__nv_bfloat16*)st.win, st.pos,
                                               ctx->d_status, 1, T, nullptr, nullptr, s, true, alpha, scale, group);
   ctx->launches += 1;
   *handled = true;

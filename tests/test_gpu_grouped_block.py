@@ -126,6 +126,27 @@ def test_grouped_block_rejects_groups_beyond_what_the_kernel_holds():
     assert ctx.la_launch_count() == 0
 
 
+@pytest.mark.parametrize("W", [1, 8, 20])
+@pytest.mark.parametrize("C", [128, 48])
+def test_grouped_block_on_tensor_cores_with_other_tap_windows(C, W):
+    """Every window but 3 taps takes the long epilogue in the three-branch mode of the tensor-core kernel; a second
+    call continues from the state and the window of the first."""
+    io, d, B, H, T, alpha = "bf16", 128, 2, 2, 3 * 128 + 50, 0.6
+    q, k, v = wl.qkv(3300 + C + W, (B, H, T, d), 0.5, io, v_mean=0.5)
+    w = wl.conv_weights(3300 + W, H, d, W)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io)
+    st = ctx.new_state(B)
+    cut = 2 * C
+    sl = lambda x, a, b: dev(x[:, :, a:b], io)
+    o1 = ctx.la_prefill_grouped(sl(q, 0, cut), sl(k, 0, cut), sl(v, 0, cut), dev(w, "f32"), st, C, alpha, d ** -0.5)
+    o2 = ctx.la_prefill_grouped(sl(q, cut, T), sl(k, cut, T), sl(v, cut, T), dev(w, "f32"), st, C, alpha, d ** -0.5,
+                                init_state=True)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    want, wst = orc.prefill_grouped_block(q, k, v, w, "elu1", 0.0, C, alpha, d ** -0.5)
+    assert rel_err(host(torch.cat([o1, o2], dim=2)), want) < TOL[io]
+    check_state(st, wst, io)
+
+
 @pytest.mark.parametrize("kernel", [0, 1])
 @pytest.mark.parametrize("phi,eps,W,T,alpha,v_mean,zero_w", [
     ("elu1", 0.0, 3, 700, 1.0, 0.0, False), ("elu1", 0.0, 3, 700, 0.5, 1.0, True), ("relu", 1e-6, 5, 333, 0.7, 1.0, False),

@@ -104,11 +104,13 @@ def test_prefill_more_chains_than_sms():
     assert st.pos.tolist() == [T] * B
 
 
-@pytest.mark.parametrize("T1,T2,T3", [(20, 300, 9), (140, 17, 130)])
-def test_prefill_continuation_with_the_longest_tap_window(T1, T2, T3):
-    """32 taps: the window carried between calls is longer than some of the pieces, and tiles after the first take
-    the rows before them from v in global memory."""
-    io, B, H, d, W = "bf16", 2, 2, 128, 32
+@pytest.mark.parametrize("W", [32, 9, 6])
+@pytest.mark.parametrize("T1,T2,T3", [(20, 300, 9), (140, 17, 130), (3, 1, 260)])
+def test_prefill_continuation_with_long_tap_windows(T1, T2, T3, W):
+    """Windows that take the long epilogue (taps in groups of 8, one halo updated in place): the window carried
+    between calls is longer than some of the pieces, 32 taps reach back across a whole 32-row block, and 9 and 6
+    taps leave most of a group of 8 as zero padding."""
+    io, B, H, d = "bf16", 2, 2, 128
     T = T1 + T2 + T3
     q, k, v, w = make(io, B, H, d, T, W, seed=15, scale=0.5)
     ctx = binding.Context(H, d, W, "elu1", 0.0, io)
