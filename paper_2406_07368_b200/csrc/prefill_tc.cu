@@ -405,7 +405,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
                   int seg_len, float* __restrict__ S_fin, float* __restrict__ z_fin, float alpha, float sm_scale,
                   int tstep) {
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  // (an offset into the array rather than an integer cast: the compiler then knows that these are shared-memory
+  // addresses: 32-bit arithmetic, ld.shared / st.shared)
+  unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   Small& sm = *reinterpret_cast<Small*>(smem + OFF_SMALL);
   constexpr bool LONG = WT < 0;                  // the epilogue for longer tap windows
@@ -1094,7 +1096,9 @@ segment_state_kernel(const __grid_constant__ CUtensorMap mk, const __grid_consta
                      float* __restrict__ S_out, float* __restrict__ z_out, int* status, int Ttot, int nseg,
                      int seg_len, int nrun) {
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  // (an offset into the array rather than an integer cast: the compiler then knows that these are shared-memory
+  // addresses: 32-bit arithmetic, ld.shared / st.shared)
+  unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + ST_OFF_SMALL);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + ST_OFF_SMALL + 128);

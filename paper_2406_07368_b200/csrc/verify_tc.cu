@@ -14,8 +14,8 @@
 //                                                                    that tap j of the causal convolution reads)
 // and the CUDA cores are left with phi, the tree walk, the mask, the denominators and
 //     o[n][c] = acc[c][n] / (phi(q_n) . z + sum_m Pm[n][m] + eps) + sum_j w[j][c] G_j[c][n].
-// Taps beyond the fourth (W > 4) are added by the CUDA cores in the epilogue, from the same shared-memory copy of V
-// and a table of the rows they read.  Nothing of the state is written.  CTAs are persistent: group X prepares
+// Taps beyond the fourth (W > 4) are summed by the CUDA cores, from the same shared-memory copy of V and a table of
+// the places they read, while the tensor cores work on the unit's products.  Nothing of the state is written.  CTAs are persistent: group X prepares
 // unit t + 1 while group Y finishes unit t, and one thread feeds TMA and the tensor cores.
 #include <cuda.h>
 
@@ -48,7 +48,8 @@ struct alignas(16) Tab {
   float den_part[2][NMAX];                         // masked row sums of P, one per column half
   float rden[NMAX];                                // 1 / (denominator + eps)
   int par[NMAX];                                   // the parent array (private to the tree warp)
-  unsigned char ext[2][kExtTaps][NMAX];            // row of the V copy that tap 4 + j of node n reads (W > 4 only)
+  unsigned short ext[2][kExtTaps][NMAX];           // where in a box of the V copy tap 4 + j of node n reads its row
+                                                   // (row * 128 + ((row & 7) << 4); W > 4 only)
 };
 struct alignas(16) Ctl {
   unsigned long long bars[12];
@@ -57,7 +58,9 @@ struct alignas(16) Ctl {
 };
 // XDONE comes as a pair indexed by the unit parity (phase t >> 1); every other barrier completes once per unit
 // (phase t), and the protocol lets none complete again before the waiters of its previous phase have passed.
-enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_SCONV, B_P, B_PS, B_SG, B_PMDONE, B_O, B_EPI, kNumBars };
+// XT (more than four taps only): group Y has taken the values of the later taps from the V copy and its tables.
+enum { B_FULL_S = 0, B_FULL_V, B_XDONE0, B_XDONE1, B_SCONV, B_P, B_PS, B_SG, B_PMDONE, B_O, B_EPI, B_XT, kNumBars };
+static_assert(kNumBars <= 12, "Ctl::bars");
 constexpr uint32_t OFF_S = 0;                               // S as it lies in memory (fp32, rows = features)
 constexpr uint32_t OFF_SB = OFF_S + S_BYTES;                // S as bf16: two boxes of 64 channels, rows = features
 constexpr uint32_t OFF_QB = OFF_SB + 2 * SB_BOX;            // phi(Q) as bf16: two boxes of 64 features
@@ -68,9 +71,15 @@ constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // row 64 j + n, col
 constexpr uint32_t OFF_PM = OFF_SELW + Q_BOX;               // masked scores, bf16
 constexpr uint32_t OFF_TAB = OFF_PM + Q_BOX;
 constexpr uint32_t OFF_CTL = OFF_TAB + (uint32_t)sizeof(Tab);
-constexpr uint32_t kSmemBytes = OFF_CTL + (uint32_t)sizeof(Ctl) + 1024;
+// Taps 4 .. W-1 of this unit's head, fp32 [128 channels][wext_pitch]: the pitch is odd, so that 32 channels read one
+// tap, and 32 consecutive elements of the head's [128][W] block are written, without bank conflicts.
+constexpr uint32_t OFF_WEXT = (OFF_CTL + (uint32_t)sizeof(Ctl) + 15u) & ~15u;
+__host__ __device__ constexpr uint32_t wext_pitch(int W) { return (uint32_t)(W - kMaxTaps) | 1u; }
+__host__ __device__ constexpr uint32_t smem_bytes(int W) { return OFF_WEXT + (W > kMaxTaps ? wext_pitch(W) * D * 4 : 0u) + 1024; }
+constexpr uint32_t kSmemBytes = smem_bytes(LA_MAX_TAPS);
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 static_assert(offsetof(Tab, rden) % 16 == 0, "rden is read four at a time");
+static_assert(offsetof(Tab, ext) % 16 == 0, "the offsets of 8 nodes are read at a time");
 static_assert(OFF_V % 1024 == 0 && V_BOX % 1024 == 0 && OFF_TAB % 16 == 0, "swizzled regions are 1024-byte aligned");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -171,7 +180,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
                  const __nv_bfloat16* __restrict__ win, __nv_bfloat16* __restrict__ o, int* status, int H, int N, int W,
                  float eps, int units) {
   extern __shared__ unsigned char smem_dyn[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  // (an offset into the array rather than an integer cast: the compiler then knows that these are shared-memory
+  // addresses: 32-bit arithmetic, ld.shared / st.shared)
+  unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   Tab& tab = *reinterpret_cast<Tab*>(smem + OFF_TAB);
   Ctl& ctl = *reinterpret_cast<Ctl*>(smem + OFF_CTL);
@@ -195,6 +206,7 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
     mbar_init(bar[B_PMDONE], kThreadsY);
     mbar_init(bar[B_O], 1);
     mbar_init(bar[B_EPI], kThreadsY);
+    mbar_init(bar[B_XT], kThreadsY);
     ctl.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -291,8 +303,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         }
         mma_commit(bar[B_O]);
         if (!mbar_wait(bar[B_O], par, abort)) break;       // V has been read by the tensor cores
-        // with more than four taps the epilogue of this unit reads V too
-        if (EXT && !mbar_wait(bar[B_EPI], par, abort)) break;
+        // with more than four taps group Y reads V too
+        if (EXT && !mbar_wait(bar[B_XT], par, abort)) break;
         if (t + 1 < nloc) load_v(t + 1);
       }
     }
@@ -315,6 +327,13 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         wv[i] = (!EXT && idx < 64 * (W - 1)) ? *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx)
                                                       : 0u;
       }
+      // more than four taps: the window is up to 31 rows, 16 bytes per lane and load, 8 loads in flight at a time
+      const uint4* wsrc = reinterpret_cast<const uint4*>(win + (size_t)u * (W - 1) * D);
+      const int wtotal = EXT ? (W - 1) * 16 : 0;
+      uint4 wq[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (EXT && lane + 32 * i < wtotal) wq[i] = wsrc[lane + 32 * i];
       __syncwarp();
       // ---- each lane follows the parents of its two nodes (integer work) ----
       unsigned long long mask[2] = {0ull, 0ull};
@@ -338,13 +357,34 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         }
       }
       const bool bad_any = __any_sync(0xffffffffu, !good);
+      if (EXT) {
+        // Where the taps beyond the fourth read: a second walk.  (This parity's table was last read two units ago,
+        // and the wait for that lies an iteration back.)
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int n = lane + 32 * s2;
+          if (n >= N)                                        // read like the others, never stored: any row will do
+            for (int kk = kMaxTaps; kk < W; ++kk) tab.ext[par][kk - kMaxTaps][n] = 0;
+          if (n < N && !bad_any) {
+            int m = n, kk = 0;
+            for (; m >= 0 && kk < W; ++kk) {
+              if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned short)(m * 128 + ((m & 7) << 4));
+              m = tab.par[m];
+            }
+            for (; kk < W; ++kk)                             // behind the chain: window rows, newest first
+              if (kk >= kMaxTaps) {
+                const int row = NMAX + kk - depth[s2];
+                tab.ext[par][kk - kMaxTaps][n] = (unsigned short)(row * 128 + ((row & 7) << 4));
+              }
+          }
+        }
+      }
       __syncwarp();
 
       // ---- the selection matrices and the window rows of unit t - 1 have been consumed (and with them everything
       //      issued before: this parity's tables were last read two units ago) ----
       if (t >= 1) ok = ok && mbar_wait(bar[B_SG], (t - 1) & 1, abort);
-      // with more than four taps the epilogue of unit t - 1 reads the window rows and the V copy as well
-      if (EXT && t >= 1) ok = ok && mbar_wait(bar[B_EPI], (t - 1) & 1, abort);
+      // with more than four taps group Y reads the window rows and the V copy of unit t - 1 as well
+      if (EXT && t >= 1) ok = ok && mbar_wait(bar[B_XT], (t - 1) & 1, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (ok) {
         if (lane == 0) tab.bad[par] = bad_any ? 1 : 0;
@@ -378,22 +418,17 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
               *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + p, (c2 & 63) >> 3) + (c2 & 7) * 2) = wv[i];
           }
         } else {
-          for (int idx = lane; idx < 64 * (W - 1); idx += 32) {
-            const int p = (W - 2) - (idx >> 6), c2 = (idx & 63) * 2;
-            *reinterpret_cast<uint32_t*>(smem + OFF_V + (c2 >> 6) * V_BOX + swz(NMAX + p, (c2 & 63) >> 3) + (c2 & 7) * 2) =
-                *reinterpret_cast<const uint32_t*>(win + (size_t)u * (W - 1) * D + 2 * idx);
-          }
-          // rows that the taps beyond the fourth read: a second walk, now that this parity's table is free
-          for (int s2 = 0; s2 < 2; ++s2) {
-            const int n = lane + 32 * s2;
-            if (n < N && !bad_any) {
-              int m = n, kk = 0;
-              for (; m >= 0 && kk < W; ++kk) {
-                if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned char)m;
-                m = tab.par[m];
-              }
-              for (; kk < W; ++kk)                         // behind the chain: window rows, newest first
-                if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned char)(NMAX + kk - depth[s2]);
+          for (int base = 0; base < wtotal; base += 256) {
+            if (base > 0) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                if (base + lane + 32 * i < wtotal) wq[i] = wsrc[base + lane + 32 * i];
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int idx = base + lane + 32 * i;          // row idx >> 4 of the window (oldest first), channels 8 (idx & 15) ...
+              if (idx < wtotal)
+                *reinterpret_cast<uint4*>(smem + OFF_V + ((idx & 15) >> 3) * V_BOX + swz(NMAX + (W - 2) - (idx >> 4), idx & 7)) = wq[i];
             }
           }
         }
@@ -499,6 +534,19 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
 #pragma unroll
       for (int j = 0; j < kMaxTaps; ++j) wt[j] = w[((size_t)h * D + c) * W + min(j, W - 1)];   // used where j < W
 
+      if (EXT) {
+        // The later taps of this head: its [128][W] block is read as it lies in memory, by all threads.  (Every
+        // thread has left the last unit's sums, which read these; the barrier below publishes the new ones.)
+        float* wext = reinterpret_cast<float*>(smem + OFF_WEXT);
+        const uint32_t pitch = wext_pitch(W);
+        const float* wh = w + (size_t)h * D * W;
+#pragma unroll 4
+        for (int e = ty; e < D * W; e += kThreadsY) {
+          const int cch = e / W, j = e - cch * W;
+          if (j >= kMaxTaps) wext[cch * pitch + j - kMaxTaps] = wh[e];
+        }
+      }
+
       ok = ok && mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) && mbar_wait(bar[B_P], par, abort);
       ok = __all_sync(0xffffffffu, ok);
       tc_fence_after();
@@ -530,6 +578,39 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       mbar_arrive(bar[B_PMDONE]);
       sync_y();
       if (ty < NMAX) tab.rden[ty] = 1.f / (tab.den_part[0][ty] + tab.den_part[1][ty] + eps);
+      float ex[EXT ? 32 : 1];                                // more than four taps: what taps 4 .. W-1 add to nodes n0 .. n0 + 31
+      if (EXT) {
+        // Each thread sums the later taps of its channel over its 32 nodes.  The values come straight from the
+        // shared-memory copy of V (draft rows, then window rows), at the places the tree warp tabulated.  None of this
+        // needs a product of this unit: it runs while the tensor cores work.
+        const float* wext = reinterpret_cast<const float*>(smem + OFF_WEXT);
+        const uint32_t pitch = wext_pitch(W);
+        ok = ok && mbar_wait(bar[B_FULL_V], par, abort);     // the draft rows of V have landed
+        ok = __all_sync(0xffffffffu, ok);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ex[i] = 0.f;
+        if (good && ok) {
+          const unsigned char* vcol = smem + OFF_V + (c >> 6) * V_BOX + (c & 7) * 2;
+          const uint32_t cx = (uint32_t)((c & 63) >> 3) << 4;          // this channel's 16-byte piece, before the swizzle
+          const float* wc = wext + c * pitch;
+#pragma unroll 2
+          for (int j = kMaxTaps; j < W; ++j) {
+            const float wj = wc[j - kMaxTaps];
+#pragma unroll
+            for (int part = 0; part < 4; ++part) {
+              const uint4 o4 = *reinterpret_cast<const uint4*>(&tab.ext[par][j - kMaxTaps][n0 + 8 * part]);   // 8 nodes
+              const uint32_t offs[8] = {o4.x & 0xffffu, o4.x >> 16, o4.y & 0xffffu, o4.y >> 16,
+                                        o4.z & 0xffffu, o4.z >> 16, o4.w & 0xffffu, o4.w >> 16};
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const unsigned short x = *reinterpret_cast<const unsigned short*>(vcol + (offs[i] ^ cx));
+                ex[8 * part + i] = fmaf(wj, __uint_as_float((uint32_t)x << 16), ex[8 * part + i]);
+              }
+            }
+          }
+        }
+        mbar_arrive(bar[B_XT]);
+      }
 
       ok = ok && mbar_wait(bar[B_O], par, abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -563,18 +644,9 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
 #pragma unroll
               for (int i = 0; i < 8; ++i) out[i] = fmaf(wt[j], __uint_as_float(rg[j][i]), out[i]);
             }
-          // taps beyond the fourth: the value comes straight from the shared-memory copy of V (draft rows, then
-          // window rows), at the row the tree warp tabulated
-          for (int j = kMaxTaps; EXT && j < W; ++j) {
-            const float wj = w[((size_t)h * D + c) * W + j];
-            const unsigned char* vcol = smem + OFF_V + (c >> 6) * V_BOX + (c & 7) * 2;
+          if (EXT) {                                         // taps beyond the fourth: summed above
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              if (nb + i < N) {
-                const int row = tab.ext[par][j - kMaxTaps][nb + i];
-                const __nv_bfloat16 x = *reinterpret_cast<const __nv_bfloat16*>(vcol + swz(row, (c & 63) >> 3));
-                out[i] = fmaf(wj, __bfloat162float(x), out[i]);
-              }
+            for (int i = 0; i < 8; ++i) out[i] += ex[8 * part + i];
           }
           // Two neighbouring lanes trade values so that each stores two adjacent channels of one node: the even
           // lane takes node nb + i, the odd lane node nb + i + 1.
@@ -665,9 +737,10 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
   auto kern = c.conv_taps <= vtc::kMaxTaps
                   ? (elu ? vtc::verify_tc_kernel<LA_PHI_ELU1, false> : vtc::verify_tc_kernel<LA_PHI_RELU, false>)
                   : (elu ? vtc::verify_tc_kernel<LA_PHI_ELU1, true> : vtc::verify_tc_kernel<LA_PHI_RELU, true>);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vtc::kSmemBytes);
+  const uint32_t smem = vtc::smem_bytes(c.conv_taps);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(kern, dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), vtc::kSmemBytes, s, ms, mv,
+  e = launch_pdl(kern, dim3(std::min(BH, ctx->sm_count)), dim3(vtc::kThreads), smem, s, ms, mv,
                  (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, parent, w, (const float*)st.z,
                  (const __nv_bfloat16*)st.win, (__nv_bfloat16*)o, ctx->d_status, c.H, N, c.conv_taps, c.eps, BH);
   ctx->launches += 1;
