@@ -449,12 +449,15 @@ def grouped_workload(W: wl.Workload, rank: int, device):
 
 
 FACTORIES = {"llama7b_prefill": prefill_workload, "grouped_block": grouped_workload, "long_prefill": prefill_workload,
-             "batched_decode": decode_workload, "tree_verify": verify_workload, "prompt_gen": promptgen_workload}
+             "batched_decode": decode_workload, "tree_verify": verify_workload, "prompt_gen": promptgen_workload,
+             "prefill_taps32": prefill_workload, "tree_verify_taps8": verify_workload}
 METRICS = {"llama7b_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "long_prefill": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "grouped_block": ("prefill_tokens_per_s_per_layer", "tokens/s"),
            "batched_decode": ("decode_tokens_per_s_per_layer", "tokens/s"),
            "tree_verify": ("verify_nodes_per_s_per_layer", "nodes/s"),
+           "prefill_taps32": ("prefill_tokens_per_s_per_layer", "tokens/s"),
+           "tree_verify_taps8": ("verify_nodes_per_s_per_layer", "nodes/s"),
            "prompt_gen": ("prompt_and_generation_tokens_per_s_per_layer", "tokens/s")}
 
 
@@ -464,7 +467,7 @@ def oracle_samples(W: wl.Workload):
     The primary sample uses the oracle's fastest exact form for the mode (grouped for prefill, the recurrence for
     decode, the tree form for verify + commit); for prefill the quadratic definition is timed beside it."""
     from oracle import la_oracle as orc
-    if W.name in ("llama7b_prefill", "long_prefill"):
+    if W.name in ("llama7b_prefill", "long_prefill", "prefill_taps32"):
         T = W.T
         q, k, v = W.prefill_inputs(B=1, T=T)
         w = W.weights()
@@ -538,13 +541,13 @@ def time_fn(fn, units, repeats: int, warmup: int = 0):
 
 def l2_note(W: wl.Workload) -> str:
     """How the GPU arm keeps the 126 MB L2 from serving a step's inputs (a property of the workload's sizes)."""
-    if W.name in ("llama7b_prefill", "long_prefill", "grouped_block"):
+    if W.name in ("llama7b_prefill", "long_prefill", "grouped_block", "prefill_taps32"):
         per_set = 4 * W.B * W.H * W.T * W.d * 2
         nsets = max(2, -(-2 * L2_BYTES // per_set) + 1) if per_set < 4 * L2_BYTES else 1
         return f"{nsets} input sets of {per_set / 2**20:.0f} MiB rotated (each larger than L2)"
     if W.name == "batched_decode":
         return f"state of {W.B * W.H * W.d * W.d * 4 / 2**20:.0f} MiB streamed every step (larger than L2)"
-    if W.name == "tree_verify":
+    if W.name in ("tree_verify", "tree_verify_taps8"):
         per_state = W.B * W.H * W.d * W.d * 4
         nsets = max(2, -(-2 * L2_BYTES // per_state) + 1)
         return f"{nsets} state sets of {per_state / 2**20:.0f} MiB rotated (together larger than 2x L2)"
@@ -803,9 +806,12 @@ def brief(res, peaks, clocks):
     return out
 
 
-OTHERS = {"llama7b_prefill": ("batched_decode", "tree_verify", "long_prefill", "grouped_block")}
-DEFAULT_STEPS = {"grouped_block": 10, "llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000, "prompt_gen": 20}
-OTHER_STEPS = {"long_prefill": 20, "batched_decode": 400, "tree_verify": 400, "grouped_block": 6}
+OTHERS = {"llama7b_prefill": ("batched_decode", "tree_verify", "long_prefill", "grouped_block", "prefill_taps32",
+                              "tree_verify_taps8")}
+DEFAULT_STEPS = {"grouped_block": 10, "llama7b_prefill": 200, "long_prefill": 50, "batched_decode": 1000, "tree_verify": 1000,
+                 "prompt_gen": 20, "prefill_taps32": 100, "tree_verify_taps8": 1000}
+OTHER_STEPS = {"long_prefill": 20, "batched_decode": 400, "tree_verify": 400, "grouped_block": 6, "prefill_taps32": 100,
+               "tree_verify_taps8": 400}
 
 
 def main():
@@ -870,7 +876,8 @@ def main():
     cpu = None
     if not args.no_cpu_baseline and world == 1:
         samples = oracle_samples(W)
-        reps = {"grouped_block": 1, "llama7b_prefill": 8, "long_prefill": 2, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2}[W.name]
+        reps = {"grouped_block": 1, "llama7b_prefill": 8, "long_prefill": 2, "batched_decode": 3, "tree_verify": 1, "prompt_gen": 2,
+                "prefill_taps32": 4, "tree_verify_taps8": 1}[W.name]
         fn, units, text = samples["primary"]
         v, per = time_fn(fn, units, reps)
         cpu = {"value": v, "unit": unit, "cores": blas_threads(), "kind": "oracle", "sample": text, "seconds": per * reps}

@@ -261,5 +261,17 @@ def grouped_block() -> Workload:
                     extra={"alpha": 1.0, "softmax_scale": 128 ** -0.5})
 
 
+def prefill_taps32() -> Workload:
+    """The LLaMA-2-7B-shaped prefill with the longest tap window: 32 live taps, which is what a convolution kernel of
+    63 (the paper's choice for FLASH) keeps under the causal mask."""
+    return Workload("prefill_taps32", "bf16", 4, 32, 128, 2048, 32, 64, "elu1", 0.0, 7, 128 ** -0.5)
+
+
+def tree_verify_taps8() -> Workload:
+    """The tree_verify shapes with 8 live taps: twice as many as the tensor cores gather."""
+    return Workload("tree_verify_taps8", "bf16", 16, 32, 128, 1024, 8, 64, "elu1", 0.0, 8, 1.0,
+                    tree_nodes=64, max_depth=5, rounds=256)
+
+
 WORKLOADS = {w().name: w for w in (tiny_fp32, llama7b_prefill, batched_decode, tree_verify, long_prefill, prompt_gen,
-                                   grouped_block)}
+                                   grouped_block, prefill_taps32, tree_verify_taps8)}

@@ -49,4 +49,4 @@ def test_workload_shapes():
     cw = w.weights()
     assert cw.shape == (32, 128, 3) and abs(float(cw.var()) - 1 / 3) < 0.02
     assert set(wl.WORKLOADS) == {"tiny_fp32", "llama7b_prefill", "batched_decode", "tree_verify", "long_prefill",
-                                 "prompt_gen", "grouped_block"}
+                                 "prompt_gen", "grouped_block", "prefill_taps32", "tree_verify_taps8"}
