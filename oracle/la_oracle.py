@@ -382,3 +382,40 @@ def accept_greedy(parent, draft_token, pred_root, pred):
         node[b], length[b] = best, best_depth
         nxt[b] = int(pred[b][best]) if best >= 0 else int(pred_root[b])
     return node, length, nxt
+
+
+def accept_threshold(parent, score, thresh):
+    """Acceptance of a draft tree by a per-node score and threshold (Sec. 4.2: the original model accepts or rejects the
+    drafted tokens, resampling if needed).
+
+    The paper names no rule.  Both published families reduce to one comparison per node, and that is what this
+    computes: node n passes when score[n] >= thresh[n] -- rejection sampling: score = p(token) / q(token) and thresh a
+    uniform draw in [0, 1) that the caller supplies; typical acceptance: score = p(token) and thresh the
+    entropy-dependent bound -- and it is accepted when it passes and the node it hangs from is accepted (a child of
+    the committed prefix: when it passes).  A comparison with a NaN fails.  Written as the definition, in node order
+    (parent[n] < n).
+
+    parent [B, N] integers; score, thresh [B, N] float32 (compared as float32, as given).  Returns (accept_node [B],
+    accept_len [B]): the deepest accepted node (the smallest index among equally deep ones, -1 for none) and its
+    depth; the caller resamples after that node.
+    """
+    parent = np.asarray(parent)
+    score = np.asarray(score, dtype=np.float32)
+    thresh = np.asarray(thresh, dtype=np.float32)
+    B, N = parent.shape
+    node = np.full((B,), -1, dtype=np.int32)
+    length = np.zeros((B,), dtype=np.int32)
+    for b in range(B):
+        check_tree(parent[b])
+        accepted = [False] * N
+        depth = [0] * N
+        best, best_depth = -1, 0
+        for n in range(N):
+            p = int(parent[b, n])
+            passes = bool(score[b, n] >= thresh[b, n])
+            accepted[n] = passes and (p < 0 or accepted[p])
+            depth[n] = 1 if p < 0 else depth[p] + 1
+            if accepted[n] and depth[n] > best_depth:      # strict: the first (smallest) index of a depth wins
+                best, best_depth = n, depth[n]
+        node[b], length[b] = best, best_depth
+    return node, length
