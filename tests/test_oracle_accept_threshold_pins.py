@@ -109,8 +109,8 @@ def test_planted_mistakes_are_caught():
         return best, bd
     assert variant() == (g["accept_node"], g["accept_len"])
     assert variant(strict=True) != (g["accept_node"], g["accept_len"])            # node 3 sits exactly on its threshold
-    assert variant(ignore_parent=True) != (g["accept_node"], g["accept_len"])     # node 4 passes on its own
+    assert variant(ignore_parent=True) != (g["accept_node"], g["accept_len"])     # node 8 passes on its own, at depth 4
+    assert variant(last_wins=True) != (g["accept_node"], g["accept_len"])         # nodes 6 and 9 tie at depth 3
     th2 = thresh.copy()
     th2[5] = g["thresh5_second"]
     assert variant(th=th2) == (g["accept_node_second"], g["accept_len_second"])
-    assert variant(last_wins=True, th=th2) != (g["accept_node_second"], g["accept_len_second"])
