@@ -238,6 +238,26 @@ la_status la_accept_greedy(la_ctx* ctx, int32_t B, int32_t N, const int32_t* par
                            const int32_t* pred_root, const int32_t* pred, int32_t* accept_node, int32_t* accept_len,
                            int32_t* next_token, void* stream);
 
+/* Acceptance by a per-node score and threshold: the sampling-based counterpart of la_accept_greedy.  (Sec. 4.2: the
+ * original model accepts or rejects the drafted tokens, "resampling if needed"; the paper names no rule.  Both
+ * published families reduce to one comparison per node, so the caller brings the two numbers: for rejection sampling
+ * score = p(token) / q(token) under the verifier and the draft model and thresh = a uniform draw in [0, 1) -- the
+ * random numbers are inputs, the library draws none; for typical acceptance score = p(token) and thresh = the
+ * entropy-dependent bound.)  Node n passes when score[n] >= thresh[n] as float32 (a NaN on either side fails) and is
+ * accepted when it passes and the node it hangs from is accepted; a child of the committed prefix when it passes.
+ *
+ *   parent       [B, N] int32 device, as for la_verify_tree
+ *   score        [B, N] float32 device
+ *   thresh       [B, N] float32 device
+ *   accept_node  [B]    int32 device, out: the deepest accepted node, the smallest index among equally deep ones;
+ *                       -1 when no child of the prefix passes.  The caller resamples after this node.
+ *   accept_len   [B]    int32 device, out: the depth of accept_node (0 for none)
+ *
+ * Errors as for la_accept_greedy: an invalid parent array gives accept_node = -1, accept_len = 0 and the device
+ * status LA_ERR_BAD_TREE; LA_ERR_INVALID_ARG for null pointers or N outside 1..max_nodes. */
+la_status la_accept_threshold(la_ctx* ctx, int32_t B, int32_t N, const int32_t* parent, const float* score,
+                              const float* thresh, int32_t* accept_node, int32_t* accept_len, void* stream);
+
 /* Self-test of the bounded waits.  (No counterpart in the paper.)  Every wait of a kernel of this library on a
  * shared-memory barrier has a time limit, after which the kernel records LA_ERR_TIMEOUT in the status word and
  * returns instead of hanging the GPU.  This call launches a one-CTA kernel that waits, through the same helper, on a

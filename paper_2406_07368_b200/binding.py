@@ -26,7 +26,7 @@ EXPORTS = ["la_create", "la_destroy", "la_status_str", "la_prefill", "la_decode_
            "la_commit", "la_last_device_status", "la_clear_device_status", "la_set_prefill_kernel",
            "la_launch_count", "la_verify_tree_noalloc", "la_set_workspace", "la_accept_greedy", "la_selftest_wait_timeout",
            "la_prefill_workspace_bytes", "la_prefill_grouped", "la_prefill_grouped_max_group",
-           "la_segment_state", "la_state_prefix"]
+           "la_segment_state", "la_state_prefix", "la_accept_threshold"]
 
 
 class LaError(RuntimeError):
@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
         L.la_verify_tree.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state), vp, vp]
         L.la_commit.argtypes = [vp, i32, i32, vp, vp, vp, vp, C.POINTER(la_state), vp, vp, vp]
         L.la_accept_greedy.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.la_accept_threshold.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
         L.la_selftest_wait_timeout.argtypes = [vp, C.c_uint32, vp, vp]
         L.la_verify_tree_noalloc.argtypes = [C.POINTER(la_config), i32, i32, vp, vp, vp, vp, vp, C.POINTER(la_state),
                                              vp, vp, vp]
@@ -277,6 +278,17 @@ class Context:
             _ptr(accept_len, torch.int32, (B,), "accept_len"), _ptr(next_token, torch.int32, (B,), "next_token"),
             _stream(stream)))
         return accept_node, accept_len, next_token
+
+    def la_accept_threshold(self, parent, score, thresh, accept_node=None, accept_len=None, stream=None):
+        B, N = parent.shape
+        dev = parent.device
+        accept_node = torch.empty(B, dtype=torch.int32, device=dev) if accept_node is None else accept_node
+        accept_len = torch.empty(B, dtype=torch.int32, device=dev) if accept_len is None else accept_len
+        _check("la_accept_threshold", lib().la_accept_threshold(
+            self._h, B, N, _ptr(parent, torch.int32, (B, N), "parent"), _ptr(score, torch.float32, (B, N), "score"),
+            _ptr(thresh, torch.float32, (B, N), "thresh"), _ptr(accept_node, torch.int32, (B,), "accept_node"),
+            _ptr(accept_len, torch.int32, (B,), "accept_len"), _stream(stream)))
+        return accept_node, accept_len
 
     def la_selftest_wait_timeout(self, limit_us: int, stream=None) -> int:
         """Runs the bounded-wait self-test; returns the nanoseconds the wait took (see include/la.h)."""

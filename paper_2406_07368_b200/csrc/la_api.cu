@@ -227,6 +227,18 @@ la_status la_accept_greedy(la_ctx* ctx, int32_t B, int32_t N, const int32_t* par
              : LA_ERR_CUDA;
 }
 
+la_status la_accept_threshold(la_ctx* ctx, int32_t B, int32_t N, const int32_t* parent, const float* score,
+                              const float* thresh, int32_t* accept_node, int32_t* accept_len, void* stream) {
+  if (!ctx || B < 1 || N < 1 || !parent || !score || !thresh || !accept_node || !accept_len) return LA_ERR_INVALID_ARG;
+  if (N > ctx->cfg.max_nodes) return LA_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return LA_ERR_CUDA;
+  return la::launch_accept_threshold(ctx, B, N, parent, score, thresh, accept_node, accept_len,
+                                     static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? LA_OK
+             : LA_ERR_CUDA;
+}
+
 la_status la_last_device_status(la_ctx* ctx, void* stream) {
   if (!ctx) return LA_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);

@@ -143,6 +143,8 @@ cudaError_t launch_verify_tc(la_ctx* ctx, int B, int N, const void* q, const voi
 cudaError_t launch_accept(la_ctx* ctx, int B, int N, const int32_t* parent, const int32_t* draft, const int32_t* pred_root,
                           const int32_t* pred, int32_t* accept_node, int32_t* accept_len, int32_t* next_token,
                           cudaStream_t s);
+cudaError_t launch_accept_threshold(la_ctx* ctx, int B, int N, const int32_t* parent, const float* score, const float* thresh,
+                                    int32_t* accept_node, int32_t* accept_len, cudaStream_t s);
 // The three-branch block (group-exclusive linear attention, softmax inside a group, convolution) on the CUDA cores.
 cudaError_t launch_prefill_grouped(la_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, const float* w,
                                    int group, float alpha, float scale, int init_state, const la_state& st, void* o,
