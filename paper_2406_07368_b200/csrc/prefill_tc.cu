@@ -378,11 +378,13 @@ __device__ __forceinline__ void conv_rows(uint32_t wcol, const uint32_t (&pv)[8]
       conv_block<BLK, ALL_H>(acc, wtap, pv, hend + (8 * (BLK - g) - 7) * (D * 2));
     }
   }
+  uint32_t lav[8];                                // the attention terms of the 8 rows, all loads in flight at once
+#pragma unroll
+  for (int jj = 0; jj < 8; ++jj) lav[jj] = lds32(sthr + (8 * BLK + jj) * 128 + ((cc ^ jj) << 4));
 #pragma unroll
   for (int jj = 0; jj < 8; ++jj) {
-    const uint32_t at = sthr + (8 * BLK + jj) * 128 + ((cc ^ jj) << 4);
-    const float2 la = bf2(lds32(at));
-    sts32(at, pack2(acc[jj].x + la.x, acc[jj].y + la.y));
+    const float2 la = bf2(lav[jj]);
+    sts32(sthr + (8 * BLK + jj) * 128 + ((cc ^ jj) << 4), pack2(acc[jj].x + la.x, acc[jj].y + la.y));
   }
 }
 
