@@ -303,6 +303,35 @@ def test_verify_more_units_than_sms_with_one_bad_tree(W):
     assert rel_err(host(out[good]), want[good]) < TOL[io]
 
 
+@pytest.mark.parametrize("B,H,W", [(50, 4, 3), (149, 1, 3), (37, 8, 4), (51, 4, 8), (64, 8, 3)])
+def test_verify_unit_counts_around_the_number_of_sms(B, H, W):
+    """Unit counts just above, far above and at multiples of the number of SMs (148: 200 units, 149, 296, 204, 512):
+    the persistent grid's last round is partly filled.  Every sequence is compared on its own and by channel half,
+    and a bad tree in one of the last sequences leaves its outputs untouched."""
+    io, d, N = "bf16", 128, 24
+    ost, q, k, v, parent, w = tree_case(io, B, H, d, N, W, seed=300 + B, phi="elu1", eps=0.0)
+    ctx = binding.Context(H, d, W, "elu1", 0.0, io, max_nodes=64, max_depth=64)
+    st = oracle_state_to_dev(ost, io)
+    before = st.clone()
+    want = orc.verify_tree(q, k, v, parent, w, "elu1", 0.0, ost)
+    o = ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(parent).cuda(), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    got = host(o)
+    for b in range(B):
+        assert rel_err(got[b], want[b]) < TOL[io], b
+        for half in (slice(0, 64), slice(64, 128)):
+            assert rel_err(got[b][..., half], want[b][..., half]) < TOL[io], (b, half)
+    assert torch.equal(st.S, before.S) and torch.equal(st.win, before.win)
+    bad = parent.copy()
+    bad[B - 2, 5] = 7                                       # a parent after its child, in one of the last sequences
+    out = torch.full((B, H, N, d), 123.0, dtype=torch.bfloat16, device="cuda")
+    ctx.la_verify_tree(dev(q, io), dev(k, io), dev(v, io), torch.from_numpy(bad).cuda(), dev(w, "f32"), st, out=out)
+    assert ctx.la_last_device_status() == binding.LA_ERR_BAD_TREE
+    assert torch.all(out[B - 2] == 123.0)
+    good = [b for b in range(B) if b != B - 2]
+    assert rel_err(host(out[good]), want[good]) < TOL[io]
+
+
 def test_verify_siblings_are_independent_bitwise():
     io, B, H, d, W = "bf16", 1, 2, 128, 3
     ost, q, k, v, _, w = tree_case(io, B, H, d, 4, W, seed=51)
