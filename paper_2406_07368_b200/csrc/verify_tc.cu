@@ -71,11 +71,9 @@ constexpr uint32_t OFF_SELW = OFF_SEL + 4 * Q_BOX;          // row 64 j + n, col
 constexpr uint32_t OFF_PM = OFF_SELW + Q_BOX;               // masked scores, bf16
 constexpr uint32_t OFF_TAB = OFF_PM + Q_BOX;
 constexpr uint32_t OFF_CTL = OFF_TAB + (uint32_t)sizeof(Tab);
-// Taps 4 .. W-1 of this unit's head, fp32 [128 channels][wext_pitch]: the pitch is odd, so that 32 channels read one
-// tap, and 32 consecutive elements of the head's [128][W] block are written, without bank conflicts.
+// Taps 4 .. W-1 of this unit's head, fp32 [W - 4][128 channels].
 constexpr uint32_t OFF_WEXT = (OFF_CTL + (uint32_t)sizeof(Ctl) + 15u) & ~15u;
-__host__ __device__ constexpr uint32_t wext_pitch(int W) { return (uint32_t)(W - kMaxTaps) | 1u; }
-__host__ __device__ constexpr uint32_t smem_bytes(int W) { return OFF_WEXT + (W > kMaxTaps ? wext_pitch(W) * D * 4 : 0u) + 1024; }
+__host__ __device__ constexpr uint32_t smem_bytes(int W) { return OFF_WEXT + (W > kMaxTaps ? (uint32_t)(W - kMaxTaps) * D * 4 : 0u) + 1024; }
 constexpr uint32_t kSmemBytes = smem_bytes(LA_MAX_TAPS);
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 static_assert(offsetof(Tab, rden) % 16 == 0, "rden is read four at a time");
@@ -316,10 +314,18 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
 #pragma unroll
     for (int i = 0; i < 6; ++i) prev[i / 3][i % 3] = 0xffffffffu;
     bool ok = true;
+    // the parents of this lane's two nodes, requested one unit ahead (right after the previous unit's walk)
+    auto load_par = [&](int t2, int& p0, int& p1) {
+      const int b2 = ((int)blockIdx.x + t2 * (int)gridDim.x) / H;
+      p0 = lane < N ? parent[(size_t)b2 * N + lane] : -1;
+      p1 = lane + 32 < N ? parent[(size_t)b2 * N + lane + 32] : -1;
+    };
+    int pn0 = -1, pn1 = -1;
+    if (nloc > 0) load_par(0, pn0, pn1);
     for (int t = 0; t < nloc; ++t) {
-      const int u = (int)blockIdx.x + t * (int)gridDim.x, b = u / H, par = t & 1;
-      tab.par[lane] = lane < N ? parent[(size_t)b * N + lane] : -1;
-      tab.par[lane + 32] = lane + 32 < N ? parent[(size_t)b * N + lane + 32] : -1;
+      const int u = (int)blockIdx.x + t * (int)gridDim.x, par = t & 1;
+      tab.par[lane] = pn0;
+      tab.par[lane + 32] = pn1;
       uint32_t wv[6];                                       // the committed window (up to three rows: W <= 4) in flight early
 #pragma unroll
       for (int i = 0; i < 6; ++i) {
@@ -335,50 +341,52 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       for (int i = 0; i < 8; ++i)
         if (EXT && lane + 32 * i < wtotal) wq[i] = wsrc[lane + 32 * i];
       __syncwarp();
-      // ---- each lane follows the parents of its two nodes (integer work) ----
+      // ---- each lane follows the parents of its two nodes (integer work), both chains in one loop so that their
+      //      loads overlap.  With more than four taps the walk also notes where taps 4 .. W-1 read: the ancestor at
+      //      distance j while the chain lasts, then rows of the committed window, newest first.  (This parity's table
+      //      was last read two units ago, and the wait for that lies an iteration back.) ----
       unsigned long long mask[2] = {0ull, 0ull};
       int depth[2] = {0, 0}, anc[2][3] = {{0, 0, 0}, {0, 0, 0}};
       bool good = true;
+      int mm[2] = {lane < N ? lane : -1, lane + 32 < N ? lane + 32 : -1};
+      while (mm[0] >= 0 || mm[1] >= 0) {                    // every step lowers the live indices: at most N iterations
 #pragma unroll
-      for (int s2 = 0; s2 < 2; ++s2) {
-        const int n = lane + 32 * s2;
-        if (n < N) {
-          int m = n;
-          while (m >= 0) {                                  // m strictly decreases: at most N iterations
+        for (int s2 = 0; s2 < 2; ++s2) {
+          const int m = mm[s2];
+          if (m >= 0) {
             mask[s2] |= 1ull << m;
             if (depth[s2] == 1) anc[s2][0] = m;
             if (depth[s2] == 2) anc[s2][1] = m;
             if (depth[s2] == 3) anc[s2][2] = m;
+            if (EXT && depth[s2] >= kMaxTaps && depth[s2] < W)
+              tab.ext[par][depth[s2] - kMaxTaps][lane + 32 * s2] = (unsigned short)(m * 128 + ((m & 7) << 4));
             ++depth[s2];
             const int p = tab.par[m];
-            if (p < -1 || p >= m) { good = false; break; }
-            m = p;
+            if (p < -1 || p >= m) {
+              good = false;
+              mm[s2] = -1;
+            } else {
+              mm[s2] = p;
+            }
           }
         }
       }
       const bool bad_any = __any_sync(0xffffffffu, !good);
       if (EXT) {
-        // Where the taps beyond the fourth read: a second walk.  (This parity's table was last read two units ago,
-        // and the wait for that lies an iteration back.)
+#pragma unroll
         for (int s2 = 0; s2 < 2; ++s2) {
           const int n = lane + 32 * s2;
-          if (n >= N)                                        // read like the others, never stored: any row will do
-            for (int kk = kMaxTaps; kk < W; ++kk) tab.ext[par][kk - kMaxTaps][n] = 0;
-          if (n < N && !bad_any) {
-            int m = n, kk = 0;
-            for (; m >= 0 && kk < W; ++kk) {
-              if (kk >= kMaxTaps) tab.ext[par][kk - kMaxTaps][n] = (unsigned short)(m * 128 + ((m & 7) << 4));
-              m = tab.par[m];
-            }
-            for (; kk < W; ++kk)                             // behind the chain: window rows, newest first
-              if (kk >= kMaxTaps) {
-                const int row = NMAX + kk - depth[s2];
-                tab.ext[par][kk - kMaxTaps][n] = (unsigned short)(row * 128 + ((row & 7) << 4));
-              }
+          // behind the chain: window rows; nodes past N are read like the others and never stored: any row will do
+          for (int kk = max(n < N ? depth[s2] : 0, kMaxTaps); kk < W; ++kk) {
+            const int row = n < N ? NMAX + kk - depth[s2] : 0;
+            tab.ext[par][kk - kMaxTaps][n] = (unsigned short)(row * 128 + ((row & 7) << 4));
           }
         }
       }
       __syncwarp();
+      if (t + 1 < nloc) load_par(t + 1, pn0, pn1);           // in flight during the waits and the writes below
+
+      // ---- the selection matrices and the window rows of unit t - 1 have been consumed      __syncwarp();
 
       // ---- the selection matrices and the window rows of unit t - 1 have been consumed (and with them everything
       //      issued before: this parity's tables were last read two units ago) ----
@@ -538,13 +546,10 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         // The later taps of this head: its [128][W] block is read as it lies in memory, by all threads.  (Every
         // thread has left the last unit's sums, which read these; the barrier below publishes the new ones.)
         float* wext = reinterpret_cast<float*>(smem + OFF_WEXT);
-        const uint32_t pitch = wext_pitch(W);
-        const float* wh = w + (size_t)h * D * W;
+        const float* wh = w + (size_t)h * D * W + kMaxTaps;
 #pragma unroll 4
-        for (int e = ty; e < D * W; e += kThreadsY) {
-          const int cch = e / W, j = e - cch * W;
-          if (j >= kMaxTaps) wext[cch * pitch + j - kMaxTaps] = wh[e];
-        }
+        for (int e = ty; e < D * (W - kMaxTaps); e += kThreadsY)   // tap 4 + (e >> 7) of channel e & 127
+          wext[e] = wh[(e & (D - 1)) * W + (e >> 7)];
       }
 
       ok = ok && mbar_wait(bar[B_XDONE0 + par], (t >> 1) & 1, abort) && mbar_wait(bar[B_P], par, abort);
@@ -583,30 +588,46 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
         // Each thread sums the later taps of its channel over its 32 nodes.  The values come straight from the
         // shared-memory copy of V (draft rows, then window rows), at the places the tree warp tabulated.  None of this
         // needs a product of this unit: it runs while the tensor cores work.
+        // For these sums lane 4 g + o of a warp takes channels 4 g ... 4 g + 3 of the warp's 32 and nodes 8 o ... 8 o + 7 of
+        // its 32: one 8-byte load brings four channels of a node's row, so a tap costs 8 loads per thread instead of
+        // 32.  A 4 x 4 transpose inside each group of four lanes (two exchange steps) then hands every lane the sums
+        // of its own channel for all 32 nodes, which is how the epilogue below holds them.
         const float* wext = reinterpret_cast<const float*>(smem + OFF_WEXT);
-        const uint32_t pitch = wext_pitch(W);
         ok = ok && mbar_wait(bar[B_FULL_V], par, abort);     // the draft rows of V have landed
         ok = __all_sync(0xffffffffu, ok);
 #pragma unroll
         for (int i = 0; i < 32; ++i) ex[i] = 0.f;
-        if (good && ok) {
-          const unsigned char* vcol = smem + OFF_V + (c >> 6) * V_BOX + (c & 7) * 2;
-          const uint32_t cx = (uint32_t)((c & 63) >> 3) << 4;          // this channel's 16-byte piece, before the swizzle
-          const float* wc = wext + c * pitch;
-#pragma unroll 2
+        if (good && ok) {                                    // (the same for every lane of the warp)
+          const int cb = 32 * q4 + (lane & ~3), o = lane & 3;             // first of the four channels; node octet
+          const unsigned char* vq = smem + OFF_V + (cb >> 6) * V_BOX + (cb & 7) * 2;
+          const uint32_t cx = (uint32_t)((cb & 63) >> 3) << 4;            // the channels' 16-byte piece, before the swizzle
+#pragma unroll 1
           for (int j = kMaxTaps; j < W; ++j) {
-            const float wj = wc[j - kMaxTaps];
+            const float4 wj = *reinterpret_cast<const float4*>(wext + (j - kMaxTaps) * D + cb);
+            const uint4 o4 = *reinterpret_cast<const uint4*>(&tab.ext[par][j - kMaxTaps][n0 + 8 * o]);   // 8 nodes
+            const uint32_t offs[8] = {o4.x & 0xffffu, o4.x >> 16, o4.y & 0xffffu, o4.y >> 16,
+                                      o4.z & 0xffffu, o4.z >> 16, o4.w & 0xffffu, o4.w >> 16};
 #pragma unroll
-            for (int part = 0; part < 4; ++part) {
-              const uint4 o4 = *reinterpret_cast<const uint4*>(&tab.ext[par][j - kMaxTaps][n0 + 8 * part]);   // 8 nodes
-              const uint32_t offs[8] = {o4.x & 0xffffu, o4.x >> 16, o4.y & 0xffffu, o4.y >> 16,
-                                        o4.z & 0xffffu, o4.z >> 16, o4.w & 0xffffu, o4.w >> 16};
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const unsigned short x = *reinterpret_cast<const unsigned short*>(vcol + (offs[i] ^ cx));
-                ex[8 * part + i] = fmaf(wj, __uint_as_float((uint32_t)x << 16), ex[8 * part + i]);
-              }
+            for (int i = 0; i < 8; ++i) {
+              const uint2 x = *reinterpret_cast<const uint2*>(vq + (offs[i] ^ cx));
+              ex[i] = fmaf(wj.x, __uint_as_float(x.x << 16), ex[i]);
+              ex[8 + i] = fmaf(wj.y, __uint_as_float(x.x & 0xffff0000u), ex[8 + i]);
+              ex[16 + i] = fmaf(wj.z, __uint_as_float(x.y << 16), ex[16 + i]);
+              ex[24 + i] = fmaf(wj.w, __uint_as_float(x.y & 0xffff0000u), ex[24 + i]);
             }
+          }
+          // ex[8 r + i]: channel cb + r, node 8 o + i  ->  ex[8 o' + i]: channel cb + o (this lane's own), node 8 o' + i
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            float a0 = ex[i], a1 = ex[8 + i], a2 = ex[16 + i], a3 = ex[24 + i];
+            const bool odd1 = o & 1, odd2 = o & 2;
+            float t0 = __shfl_xor_sync(0xffffffffu, odd1 ? a0 : a1, 1);
+            float t1 = __shfl_xor_sync(0xffffffffu, odd1 ? a2 : a3, 1);
+            if (odd1) { a0 = t0; a2 = t1; } else { a1 = t0; a3 = t1; }
+            t0 = __shfl_xor_sync(0xffffffffu, odd2 ? a0 : a2, 2);
+            t1 = __shfl_xor_sync(0xffffffffu, odd2 ? a1 : a3, 2);
+            if (odd2) { a0 = t0; a1 = t1; } else { a2 = t0; a3 = t1; }
+            ex[i] = a0; ex[8 + i] = a1; ex[16 + i] = a2; ex[24 + i] = a3;
           }
         }
         mbar_arrive(bar[B_XT]);
@@ -619,7 +640,8 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
       if (good && n0 < N) {                                  // warp-uniform (good implies ok)
         const uint32_t lane_base = tmem + ((uint32_t)(32 * q4) << 16) + n0;
         const int odd = lane & 1;
-        uint32_t pairs[16];                                  // two adjacent channels of node n0 + 2 i + odd
+        uint32_t pairs[EXT ? 1 : 16];                        // two adjacent channels of node n0 + 2 i + odd
+        __nv_bfloat16* orow = o + ((size_t)u * N + n0 + odd) * D + (c - odd);
 #pragma unroll
         for (int part = 0; part < 4; ++part) {               // 8 nodes at a time, all their TMEM loads in flight at once
           const int nb = n0 + 8 * part;
@@ -654,16 +676,20 @@ verify_tc_kernel(const __grid_constant__ CUtensorMap ms, const __grid_constant__
           for (int i = 0; i < 8; i += 2) {
             const float give = odd ? out[i] : out[i + 1];
             const float got = __shfl_xor_sync(0xffffffffu, give, 1);
-            pairs[4 * part + i / 2] = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
+            const uint32_t pr = odd ? pack2(got, out[i + 1]) : pack2(out[i], got);
+            if (EXT) {                                         // (the later taps' sums need the registers: store at once)
+              if (nb + i + odd < N) *reinterpret_cast<uint32_t*>(orow + (size_t)(8 * part + i) * D) = pr;
+            } else {
+              pairs[4 * part + i / 2] = pr;
+            }
           }
         }
         // the accumulators are free again before the outputs leave: the barrier's release would wait for the stores
         tc_fence_before();
         mbar_arrive(bar[B_EPI]);
-        __nv_bfloat16* orow = o + ((size_t)u * N + n0 + odd) * D + (c - odd);
 #pragma unroll
         for (int i = 0; i < 16; ++i)
-          if (n0 + 2 * i + odd < N) *reinterpret_cast<uint32_t*>(orow + (size_t)(2 * i) * D) = pairs[i];
+          if (!EXT && n0 + 2 * i + odd < N) *reinterpret_cast<uint32_t*>(orow + (size_t)(2 * i) * D) = pairs[i];
       } else {
         if (ok && !good && ty == 0) report(status, LA_ERR_BAD_TREE);
         tc_fence_before();
