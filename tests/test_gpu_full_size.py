@@ -72,6 +72,45 @@ def test_llama7b_prefill_full_size():
     assert st.pos.tolist() == [W.T] * W.B
 
 
+def test_prefill_taps32_full_size():
+    """The 32-tap prefill of the bench line (long-window epilogue), full batch, sampled units against the definition."""
+    W = wl.prefill_taps32()
+    q, k, v = W.prefill_inputs()
+    w = W.weights()
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, W.io, chunk=W.chunk)
+    st = ctx.new_state(W.B)
+    o = ctx.la_prefill(dev(q), dev(k), dev(v), dev(w, "f32"), st)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    for b, h in sampled_units(W.B, W.H, 8):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        want, wst = orc.prefill_quadratic(q[sl], k[sl], v[sl], w[h:h + 1], W.phi, W.eps)
+        assert rel_err(host(o[sl]), want) < TOL["bf16"], (b, h)
+        assert rel_err(host(o[sl])[:, :, -128:], want[:, :, -128:]) < TOL["bf16"], (b, h)
+        assert rel_err(host(st.S[sl]), wst.S) < TOL["bf16"] and rel_err(host(st.z[sl]), wst.z) < TOL["bf16"]
+        np.testing.assert_array_equal(host(st.win[sl]), wst.win)
+    assert st.pos.tolist() == [W.T] * W.B
+
+
+def test_grouped_block_full_size():
+    """The three-branch block of the bench line (groups of 64 on the tensor cores), full batch, sampled units."""
+    W = wl.grouped_block()
+    q, k, v = W.prefill_inputs()
+    w = W.weights()
+    alpha, scale = W.extra["alpha"], W.extra["softmax_scale"]
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, W.io, chunk=W.chunk)
+    st = ctx.new_state(W.B)
+    o = ctx.la_prefill_grouped(dev(q), dev(k), dev(v), dev(w, "f32"), st, W.chunk, alpha, scale)
+    assert ctx.la_last_device_status() == binding.LA_OK
+    for b, h in sampled_units(W.B, W.H, 6):
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        want, wst = orc.prefill_grouped_block(q[sl], k[sl], v[sl], w[h:h + 1], W.phi, W.eps, W.chunk, alpha, scale)
+        assert rel_err(host(o[sl]), want) < TOL["bf16"], (b, h)
+        assert rel_err(host(o[sl])[:, :, -128:], want[:, :, -128:]) < TOL["bf16"], (b, h)
+        assert rel_err(host(st.S[sl]), wst.S) < TOL["bf16"] and rel_err(host(st.z[sl]), wst.z) < TOL["bf16"]
+        np.testing.assert_array_equal(host(st.win[sl]), wst.win)
+    assert st.pos.tolist() == [W.T] * W.B
+
+
 def test_long_prefill_full_size_then_decode():
     W = wl.long_prefill()
     q, k, v = W.prefill_inputs()
