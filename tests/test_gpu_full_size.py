@@ -262,6 +262,42 @@ def test_tree_verify_full_size_rounds():
     assert ctx.la_last_device_status() == binding.LA_OK
 
 
+def test_tree_verify_taps8_full_size_rounds():
+    """The 8-tap verify of the bench line at full size (512 units: more than four taps, summed beside the tensor
+    cores): 12 rounds of verify + commit with the state carried, sampled units against the oracle, the window of 7
+    rows bit-exact at the end."""
+    W = wl.tree_verify_taps8()
+    q, k, v = W.prefill_inputs()
+    w = W.weights()
+    ctx = binding.Context(W.H, W.d, W.W, W.phi, W.eps, W.io, max_nodes=W.tree_nodes, max_depth=W.max_depth)
+    st = ctx.new_state(W.B)
+    dw = dev(w, "f32")
+    ctx.la_prefill(dev(q), dev(k), dev(v), dw, st)
+    units = ((0, 0), (5, 9), (9, 30), (15, 31))            # (15, 31): the last unit of the launch's last round
+    ost = {}
+    for b, h in units:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        _, ost[(b, h)] = orc.prefill_chunked(q[sl], k[sl], v[sl], w[h:h + 1], W.phi, W.eps, 256)
+    for rnd in range(12):
+        qd, kd, vd = W.draft_inputs(rnd)
+        parent, accept = W.trees(rnd)
+        par, acc = torch.from_numpy(parent).cuda(), torch.from_numpy(accept).cuda()
+        dq, dk, dv = dev(qd), dev(kd), dev(vd)
+        o = ctx.la_verify_tree(dq, dk, dv, par, dw, st)
+        ctx.la_commit(dk, dv, par, acc, st)
+        for b, h in units:
+            sl = (slice(b, b + 1), slice(h, h + 1))
+            want = orc.verify_tree(qd[sl], kd[sl], vd[sl], parent[b:b + 1], w[h:h + 1], W.phi, W.eps, ost[(b, h)])
+            assert rel_err(host(o[sl]), want) < TOL["bf16"], (rnd, b, h)
+            ost[(b, h)], _, _ = orc.commit(kd[sl], vd[sl], parent[b:b + 1], accept[b:b + 1], W.phi, ost[(b, h)],
+                                           W.max_depth)
+    for b, h in units:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        assert rel_err(host(st.S[sl]), ost[(b, h)].S) < TOL["bf16"]
+        np.testing.assert_array_equal(host(st.win[sl]), ost[(b, h)].win)
+    assert ctx.la_last_device_status() == binding.LA_OK
+
+
 def test_prompt_gen_pairs_prefill_then_generate():
     """The two shorter (prompt, generation) pairs end to end at full head count: every output token and the final
     state against the oracle's quadratic definition over the whole P + G sequence."""
