@@ -737,6 +737,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       mbar_arrive((bar0 + 8u * (B_PHI)));
       float dpart = 0.f;                          // this half of the row sum of the masked P
 
+      // ---- phi on K of the next tile, while the tensor cores form the scores of this one ----
+      if (!GRP && !last) {
+        ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        phi_k(n + 1, ok);
+      }
+
       // ---- P: causal mask, packed bf16 -> TMEM ----
       if (!GRP) ok = ok && mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -843,13 +850,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       }
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PDONE)));
-
-      // ---- phi on K of the next tile while the tensor cores work on this one ----
-      if (!GRP && !last) {
-        ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
-        ok = __all_sync(0xffffffffu, ok);
-        phi_k(n + 1, ok);
-      }
 
       // ---- S_n: bf16 copy for the next tile, or the final state to global memory ----
       // S_n is final after MMA_S; the old copy may be overwritten once O = phi(Q) S_prev has read it
