@@ -571,14 +571,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
           mma_bf16_ts(tmem + O_COL, tmem + P_COL + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), desc64(v_mn + kstep_mnmajor(ks)),
                       idesc(false, true, 128), (has_state && (!GRP || use_glob)) || ks > 0);
         mma_commit((bar0 + 8u * (B_MMA_O0 + par)));
-        if (!LONG && n + 2 < nchunks) {   // the state update was issued long ago: this K buffer is free and takes tile n+2
-          ok = mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort);
-          if (!ok) break;
-          const uint32_t kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
-          mbar_expect_tx(kbar, tile_tx);
-          tma_load(kbuf, &mk, 0, y0 + (n + 2) * tstep, bh, kbar);
-          tma_load(kbuf + KBOX_BYTES, &mk, 64, y0 + (n + 2) * tstep, bh, kbar);
-        }
         // P of the next tile overwrites the columns that the last product of this tile reads
         ok = mbar_wait((bar0 + 8u * (B_MMA_O0 + par)), (n >> 1) & 1, abort);
         if (!ok) break;
@@ -635,6 +627,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         }
       }
       tma_wait_all();                             // every store is complete before the CTA exits
+    } else if (lane == 1 && !LONG) {
+      // A lane of its own for the K reloads (short-window mode): the K buffer of tile n is free the moment its state
+      // update completes, and phi(K) of tile n+2 is wanted early -- neither the issuing lane nor the store lane
+      // should have to stand by for that moment.
+      for (int n = 0; n + 2 < nchunks; ++n) {
+        const uint32_t par = n & 1;
+        if (!mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort)) break;
+        const uint32_t kbuf = sbase + (par ? OFF_K1 : OFF_K0), kbar = bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0);
+        mbar_expect_tx(kbar, tile_tx);
+        tma_load(kbuf, &mk, 0, y0 + (n + 2) * tstep, bh, kbar);
+        tma_load(kbuf + KBOX_BYTES, &mk, 64, y0 + (n + 2) * tstep, bh, kbar);
+      }
     }
   } else if (warp >= 8) {
     // =============================== group A: phi, P, [S|z] snapshot (256 threads) ===============================
