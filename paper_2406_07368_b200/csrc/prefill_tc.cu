@@ -79,12 +79,14 @@ struct Small {
 // waiter is never more than one phase behind.
 enum { B_FULL_K0 = 0, B_FULL_V0 = 1, B_FULL_V1 = 2, B_MMA_P = 3, B_MMA_S = 4, B_MMA_O0 = 5, B_MMA_O1 = 6, B_PHI = 7,
        B_PDONE = 8, B_SB = 9, B_EPI0 = 10, B_EPI1 = 11, B_MMA_Q = 12, B_FULL_Q = 13, B_FULL_K1 = 14, B_STAGED0 = 15,
-       B_STAGED1 = 16, kNumBars = 17 };
+       B_STAGED1 = 16, B_HALO = 17, kNumBars = 18 };
 
 __host__ __device__ constexpr uint32_t off_w() { return OFF_SMALL + (uint32_t)((sizeof(Small) + 15) / 16 * 16); }
 __host__ __device__ inline uint32_t off_halo(int W) { return off_w() + (uint32_t)W * D * 4; }
-// Two halo buffers (the rows of v before a tile, for the convolution): tile n reads one and fills the other.
-__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + 2u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
+// Three halo buffers (the rows of v before a tile, for the convolution).  Where group B fills them itself, tile n reads
+// buffer n & 1 and fills the other; where group A fills them (short windows of the exact layer), tile n reads buffer
+// n % 3 and group A fills (n + 1) % 3 meanwhile, which the epilogue of tile n - 1 no longer reads.
+__host__ __device__ inline uint32_t smem_bytes(int W) { return off_halo(W) + 3u * (uint32_t)(W > 1 ? W - 1 : 1) * D * 2 + 1024; }
 // The three-branch mode keeps 4 KB more behind the halo rows: z before the tile as fp32 [128], the halves of
 // phi(q) . z [2][128], and each half-row's running maximum and sum of the softmax [2][128] x 2.
 constexpr uint32_t kGrpScratch = 4096;
@@ -413,6 +415,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
   const uint32_t sbase = smem_u32(smem);
   Small& sm = *reinterpret_cast<Small*>(smem + OFF_SMALL);
   constexpr bool LONG = WT < 0;                  // the epilogue for longer tap windows
+  constexpr bool HALO_A = !GRP && WT > 0;        // group A copies the rows before the next tile aside (it has the time)
   float* wsm = reinterpret_cast<float*>(smem + off_w());                       // [W][128] ([W up to a multiple of 8][128] if LONG)
   // two halo buffers [W-1][128], oldest row first: tile n reads buffer n&1 and writes buffer (n+1)&1 (LONG: one buffer)
   __nv_bfloat16* halo0 = reinterpret_cast<__nv_bfloat16*>(smem + (LONG ? off_halo_long(W) : off_halo(W)));
@@ -454,6 +457,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     mbar_init((bar0 + 8u * (B_MMA_Q)), 1);
     mbar_init((bar0 + 8u * (B_STAGED0)), kThreadsB);
     mbar_init((bar0 + 8u * (B_STAGED1)), kThreadsB);
+    mbar_init((bar0 + 8u * (B_HALO)), kThreadsA);
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -855,6 +859,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PDONE)));
 
+      // ---- the rows of v before the next tile: the last W-1 of (halo ++ valid rows of this tile's V), 16 bytes per
+      //      thread, in the time this group would otherwise wait for the state update ----
+      if (HALO_A) {
+        ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+          const int valid = min(tstep, T - n * tstep);
+          const __nv_bfloat16* halo = halo0 + (n % 3) * halo_elems;
+          __nv_bfloat16* halo_next = halo0 + ((n + 1) % 3) * halo_elems;
+          const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
+          for (int idx = ta; idx < 16 * (W - 1); idx += kThreadsA) {
+            const int i = idx >> 4, c16 = idx & 15, src = valid + i;
+            uint4 x;
+            if (src < W - 1) x = *reinterpret_cast<const uint4*>(halo + src * D + 8 * c16);
+            else x = *reinterpret_cast<const uint4*>(Vt + (c16 >> 3) * BOX_BYTES + swz(src - (W - 1), c16 & 7));
+            *reinterpret_cast<uint4*>(halo_next + i * D + 8 * c16) = x;
+          }
+        }
+        mbar_arrive((bar0 + 8u * (B_HALO)));
+      }
+
       // ---- S_n: bf16 copy for the next tile, or the final state to global memory ----
       // S_n is final after MMA_S; the old copy may be overwritten once O = phi(Q) S_prev has read it
       ok = ok && mbar_wait((bar0 + 8u * (B_MMA_S)), par, abort) && mbar_wait((bar0 + 8u * (B_MMA_Q)), par, abort);
@@ -987,11 +1012,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       const int valid = min(tstep, T - n * tstep);
       const unsigned char* Vt = smem + OFF_V0 + par * TILE_BYTES;
       // rows before this tile, addressed so that row -1 is the last of W-1 rows
-      const __nv_bfloat16* halo = halo0 + par * halo_elems;
+      const __nv_bfloat16* halo = halo0 + (HALO_A ? n % 3 : (int)par) * halo_elems;
       __nv_bfloat16* halo_next = halo0 + (par ^ 1) * halo_elems;    // rows before the next tile
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_V0 + par)), (n >> 1) & 1, abort);
+      // (HALO_A: group A has read the last rows of this tile's V, and with that filled the halo of the tile before)
+      if (HALO_A) ok = ok && mbar_wait((bar0 + 8u * (B_HALO)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
-      if (ok) {
+      if (ok && !HALO_A) {
         // next halo <- last W-1 rows of (halo ++ valid rows of V), 16 bytes (8 channels) per thread; each half of the
         // group copies its own 64 channels
         const unsigned char* Vc = Vt + hf * BOX_BYTES;
@@ -1016,7 +1043,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         tc_fence_after();
         LA_TMEM_LD32(tmem + lane_addr + O_COL + 64 * hf, v);
       }
-      sync_half_b(hf);                            // the next halo is complete before any row of V is overwritten
+      if (!HALO_A) sync_half_b(hf);               // the next halo is complete before any row of V is overwritten
       float rden = 0.f;
       if (ok) {
         // row sum of the masked P + phi(q) . z_prev, both halves gathered by the masking threads
@@ -1066,7 +1093,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
     sync_group_b();                               // both halves of the last halo are complete
     if (ok && tid < D) {
       // the window to carry on: the last W-1 values of (incoming window ++ this unit's v)
-      const __nv_bfloat16* halo = halo0 + (LONG ? ((int)long_taps(W) - W) * D : (nchunks & 1) * halo_elems);
+      const __nv_bfloat16* halo = halo0 + (LONG ? ((int)long_taps(W) - W) * D : (HALO_A ? nchunks % 3 : nchunks & 1) * halo_elems);
       for (int i = 0; i < W - 1; ++i) win[((size_t)u * (W - 1) + i) * D + tid] = halo[i * D + tid];
       if (tid == 0 && h == 0 && nseg == 1) pos[bh / H] = (init ? pos[bh / H] : 0) + T;
     }
