@@ -745,8 +745,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       mbar_arrive((bar0 + 8u * (B_PHI)));
       float dpart = 0.f;                          // this half of the row sum of the masked P
 
-      // ---- phi on K of the next tile, while the tensor cores form the scores of this one ----
-      if (!GRP && !last) {
+      // ---- phi on K of the next tile, while the tensor cores form the scores of this one.  (Not with the long-window
+      //      epilogue: there the K buffer comes back late, after the outputs staged in it have left, and waiting for
+      //      it here would hold up the mask; see below.) ----
+      if (!GRP && !LONG && !last) {
         ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
         ok = __all_sync(0xffffffffu, ok);
         phi_k(n + 1, ok);
@@ -858,6 +860,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
       }
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PDONE)));
+
+      if (!GRP && LONG && !last) {                // long-window epilogue: phi on K of the next tile after the mask
+        ok = ok && mbar_wait((bar0 + 8u * (((n + 1) & 1) ? B_FULL_K1 : B_FULL_K0)), ((n + 1) >> 1) & 1, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        phi_k(n + 1, ok);
+      }
 
       // ---- the rows of v before the next tile: the last W-1 of (halo ++ valid rows of this tile's V), 16 bytes per
       //      thread, in the time this group would otherwise wait for the state update ----
