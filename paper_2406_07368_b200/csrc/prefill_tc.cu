@@ -713,9 +713,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
 
       // ---- phi on Q in place (phi on K of this tile was done one iteration earlier) ----
       ok = ok && mbar_wait((bar0 + 8u * (B_FULL_Q)), par, abort);
-      if (GRP)   // the score product runs on the raw q and k: phi may touch K only once it is complete
-        ok = ok && mbar_wait((bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0)), (n >> 1) & 1, abort) &&
-             mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
       ok = __all_sync(0xffffffffu, ok);
       if (GRP) sync_group_a();                    // z of the previous snapshot (written by other threads) is in place
       // phi(q) of row r, this thread's 64 channels: 32 packed pairs = 32 TMEM columns of lane r.  (The products of
@@ -739,7 +736,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant_
         }
         tmem_wait_st();
       }
-      if (GRP) phi_k(n, ok);                      // phi on K of this tile, in place, now that the scores are complete
+      if (GRP) {
+        // phi on K of this tile, in place: the score product runs on the raw q and k, so K may be touched only once
+        // that product is complete (phi(Q) above reads the Q buffer and writes TMEM: it ran beside the product)
+        ok = ok && mbar_wait((bar0 + 8u * (par ? B_FULL_K1 : B_FULL_K0)), (n >> 1) & 1, abort) &&
+             mbar_wait((bar0 + 8u * (B_MMA_P)), par, abort);
+        ok = __all_sync(0xffffffffu, ok);
+        phi_k(n, ok);
+      }
       fence_proxy_async();                        // (phi(K) of this tile, written one iteration earlier)
       tc_fence_before();
       mbar_arrive((bar0 + 8u * (B_PHI)));
