@@ -15,15 +15,18 @@
 //   tcgen05  [P | phi(q) . z_prev] = phi(Q) [phi(K); z_prev]^T     (144 columns: 128 tokens, z_prev, 15 unused)
 //            [S | z] += phi(K)^T [V | 1]               (fp32 in TMEM for the whole chain)
 //            O = phi(Q) S_prev                         (S_prev is a bf16 copy in shared memory)
-//   group A  P -> causal mask, row sums (+ the z column), bf16 -> TMEM (the A operand of the next product);
-//            phi on K of tile n+1 (K is double-buffered);  S -> bf16 copy, z -> the K buffer of tile n+1
+//   group A  phi on K of tile n+1 (K is double-buffered), while the tensor cores form the scores;
+//            P -> causal mask, row sums (+ the z column), bf16 -> TMEM (the A operand of the next product);
+//            the rows of v before the next tile -> a halo buffer;  S -> bf16 copy, z -> the K buffer of tile n+1
 //   tcgen05  O += (P o M) V
 //   group B  o = O / (den + eps) + conv(V) -> the tile's V buffer;  TMA stores it to global memory
+// (More than 5 taps: a second epilogue, which forms the tap sums by channel pair and stages the outputs in the tile's
+// K buffer; three-branch mode, GRP: the score product on the raw q and k and a causal softmax instead of the mask.)
 //
 // Four roles run concurrently: group A (warps 8-15), group B (warps 0-7), warp 16, whose elected lane issues
-// every MMA and the Q and K loads, and warp 17, whose elected lane issues the V loads and the output stores (a
-// store has to have read its buffer before the buffer is reloaded: that wait must not hold up the products).
-// While group B finishes tile n, group A already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
+// every MMA and the Q loads, and warp 17, one lane of which issues the V loads and the output stores (a store has
+// to have read its buffer before the buffer is reloaded: that wait must not hold up the products) and another the
+// K reloads.  While group B finishes tile n, group A already works on tile n+1.  Every wait on an mbarrier is bounded; when one runs out the CTA
 // records LA_ERR_TIMEOUT, stops issuing work, frees its TMEM and returns.
 #include <cuda.h>
 
